@@ -1,0 +1,168 @@
+"""SemantiCache oracle -- TEST INFRASTRUCTURE, not the product.
+
+Thin numpy front end of ``semanticache_oracle.c`` (plain C, double accumulators,
+written from the paper's Eq. 1-4 and Algorithm 1).  It shares nothing with the CUDA
+path and must only be used by tests, the smoke check and the benchmark's
+cpu-baseline leg.
+
+Array conventions: bf16 tensors are numpy ``uint16`` arrays holding the raw bits,
+fp32 tensors are ``float32``; K, V are ``[B, Hkv, n, d]`` (any strides with the last
+axis contiguous), cores ``[B, Hkv, cap, d]``, counts ``[B, Hkv, cap]`` int32.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "semanticache_oracle.c")
+_SO = os.path.join(_HERE, "libsemanticache_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP over the outer (b, head) loops only)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
+               _SRC, "-o", _SO, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_chunk.restype = ctypes.c_int64
+        _lib.oracle_sim.restype = ctypes.c_double
+        _lib.oracle_f64_to_bf16.restype = ctypes.c_uint16
+        _lib.oracle_f64_to_bf16.argtypes = [ctypes.c_double]
+    return _lib
+
+
+def _p(a):
+    return ctypes.c_void_p(a.ctypes.data) if a is not None else ctypes.c_void_p(0)
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.uint16:
+        return 0
+    if a.dtype == np.float32:
+        return 1
+    raise TypeError(f"oracle takes uint16 (bf16 bits) or float32, got {a.dtype}")
+
+
+def _kv_strides(K: np.ndarray):
+    assert K.ndim == 4 and K.strides[3] == K.itemsize, "last axis must be contiguous"
+    return tuple(ctypes.c_int64(s // K.itemsize) for s in K.strides[:3])
+
+
+def bf16_bits_to_f64(a: np.ndarray) -> np.ndarray:
+    """Decode raw bf16 bits (uint16) exactly."""
+    return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def f64_to_bf16_bits(x: float) -> int:
+    return int(_load().oracle_f64_to_bf16(float(x)))
+
+
+def num_threads() -> int:
+    """Threads the OpenMP loops will use (the benchmark reports this as 'cores')."""
+    env = os.environ.get("OMP_NUM_THREADS")
+    if env:
+        return int(env)
+    return len(os.sched_getaffinity(0))
+
+
+def chunk(token_ids: np.ndarray, delim_ids, max_chunk_len: int = 256):
+    """Eq. 1.  Returns (seg_off[n_seg+1], seq_seg_off[B+1]) over the flattened token axis."""
+    ids = np.ascontiguousarray(token_ids, dtype=np.int32)
+    assert ids.ndim == 2
+    B, n = ids.shape
+    delim = np.ascontiguousarray(np.asarray(list(delim_ids), dtype=np.int32))
+    seg_off = np.zeros(B * n + 1, dtype=np.int32)
+    seq_seg_off = np.zeros(B + 1, dtype=np.int32)
+    n_seg = _load().oracle_chunk(_p(ids), ctypes.c_int32(B), ctypes.c_int32(n), _p(delim),
+                                 ctypes.c_int32(len(delim)), ctypes.c_int32(max_chunk_len),
+                                 _p(seg_off), _p(seq_seg_off))
+    return seg_off[: n_seg + 1].copy(), seq_seg_off
+
+
+def sim(K2d: np.ndarray, a: int, b: int) -> float:
+    """Eq. 2 between rows a and b of a contiguous [rows, d] array."""
+    K2d = np.ascontiguousarray(K2d)
+    return float(_load().oracle_sim(_p(K2d), ctypes.c_int32(_dtype_code(K2d)), ctypes.c_int64(a),
+                                    ctypes.c_int64(b), ctypes.c_int32(K2d.shape[1])))
+
+
+def gsc(K: np.ndarray, seg_off: np.ndarray, seq_seg_off: np.ndarray, tau: float):
+    """Algorithm 1 per (b, head, segment).  Returns (assign[B,Hkv,n] int32, min |Sim-tau|)."""
+    B, Hkv, n, d = K.shape
+    sb, sh, sn = _kv_strides(K)
+    assign = np.full((B, Hkv, n), -1, dtype=np.int32)
+    margin = ctypes.c_double(0.0)
+    seg_off = np.ascontiguousarray(seg_off, dtype=np.int32)
+    seq_seg_off = np.ascontiguousarray(seq_seg_off, dtype=np.int32)
+    _load().oracle_gsc(_p(K), ctypes.c_int32(_dtype_code(K)), sb, sh, sn, ctypes.c_int32(B),
+                       ctypes.c_int32(Hkv), ctypes.c_int32(n), ctypes.c_int32(d), _p(seg_off),
+                       _p(seq_seg_off), ctypes.c_float(tau), _p(assign), ctypes.byref(margin))
+    return assign, margin.value
+
+
+def merge(K: np.ndarray, V: np.ndarray, assign: np.ndarray, cap: int | None = None,
+          seg_off: np.ndarray | None = None, seq_seg_off: np.ndarray | None = None):
+    """Eq. 3.  Returns (core_k, core_v, count, core_len).
+
+    With seg_off/seq_seg_off given, members of a seed are looked for inside the seed's
+    segment only (same result, far fewer comparisons; used for timing)."""
+    B, Hkv, n, d = K.shape
+    assert V.shape == K.shape and V.dtype == K.dtype and V.strides == K.strides
+    cap = n if cap is None else cap
+    sb, sh, sn = _kv_strides(K)
+    core_k = np.zeros((B, Hkv, cap, d), dtype=K.dtype)
+    core_v = np.zeros((B, Hkv, cap, d), dtype=K.dtype)
+    count = np.zeros((B, Hkv, cap), dtype=np.int32)
+    core_len = np.zeros((B, Hkv), dtype=np.int32)
+    assign = np.ascontiguousarray(assign, dtype=np.int32)
+    common = (_p(K), _p(V), ctypes.c_int32(_dtype_code(K)), sb, sh, sn, ctypes.c_int32(B),
+              ctypes.c_int32(Hkv), ctypes.c_int32(n), ctypes.c_int32(d))
+    tail = (_p(assign), _p(core_k), _p(core_v), _p(count), ctypes.c_int32(cap), _p(core_len))
+    if seg_off is None:
+        _load().oracle_merge(*common, *tail)
+    else:
+        seg_off = np.ascontiguousarray(seg_off, dtype=np.int32)
+        seq_seg_off = np.ascontiguousarray(seq_seg_off, dtype=np.int32)
+        _load().oracle_merge_seg(*common, _p(seg_off), _p(seq_seg_off), *tail)
+    return core_k, core_v, count, core_len
+
+
+def attn(q: np.ndarray, core_k: np.ndarray, core_v: np.ndarray, count: np.ndarray | None,
+         core_len: np.ndarray, scale: float | None = None) -> np.ndarray:
+    """Eq. 4 for one decode step.  q: [B, Hq, d].  Returns float64 [B, Hq, d]."""
+    q = np.ascontiguousarray(q)
+    core_k = np.ascontiguousarray(core_k)
+    core_v = np.ascontiguousarray(core_v)
+    B, Hq, d = q.shape
+    _, Hkv, cap, _ = core_k.shape
+    assert Hq % Hkv == 0 and q.dtype == core_k.dtype == core_v.dtype
+    if count is not None:
+        count = np.ascontiguousarray(count, dtype=np.int32)
+    core_len = np.ascontiguousarray(core_len, dtype=np.int32)
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    out = np.zeros((B, Hq, d), dtype=np.float64)
+    _load().oracle_attn(_p(q), ctypes.c_int32(_dtype_code(q)), ctypes.c_int32(B), ctypes.c_int32(Hq),
+                        ctypes.c_int32(Hkv), ctypes.c_int32(d), _p(core_k), _p(core_v), _p(count),
+                        ctypes.c_int32(cap), _p(core_len), ctypes.c_double(scale), _p(out))
+    return out
+
+
+def compress(token_ids, delim_ids, K, V, tau, max_chunk_len=256, cap=None):
+    """chunk -> gsc -> merge, the whole compress stage.  Returns a dict of every product."""
+    seg_off, seq_seg_off = chunk(token_ids, delim_ids, max_chunk_len)
+    assign, margin = gsc(K, seg_off, seq_seg_off, tau)
+    core_k, core_v, count, core_len = merge(K, V, assign, cap, seg_off, seq_seg_off)
+    return dict(seg_off=seg_off, seq_seg_off=seq_seg_off, assign=assign, margin=margin,
+                core_k=core_k, core_v=core_v, count=count, core_len=core_len)
