@@ -1,0 +1,174 @@
+/*
+ * SemantiCache hot path for NVIDIA B200 (sm_100a) -- C ABI.
+ *
+ * Three calls follow the paper's pipeline:
+ *   sc_chunk        Sec. 2.2, Eq. 1          token ids + delimiter set -> chunk offsets
+ *   sc_compress     Sec. 2.3-2.4, Eq. 2,     per layer: K/V + chunk offsets + GSC parameters ->
+ *                   Algorithm 1, Eq. 3       semantic cores (K, V), member counts, per-head lengths
+ *   sc_decode_attn  Sec. 2.4, Eq. 4          GQA decode queries against the cores with
+ *                                            Proportional Attention (softmax(qK^T/sqrt(d) + ln s) V)
+ *
+ * General rules
+ *   - Every pointer is a DEVICE pointer unless its comment says HOST.  The caller owns all
+ *     buffers; the library allocates nothing and keeps no state between calls.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     Calls return after enqueueing; they never synchronise.
+ *   - The return value reports host-side validation only (SC_OK, SC_ERR_INVALID_ARG,
+ *     SC_ERR_UNSUPPORTED, SC_ERR_CUDA for a failed launch).  Conditions found on the device
+ *     are written to the caller's `status` word (int32, device or pinned host memory, may be
+ *     NULL): it is left untouched on success and set to SC_ERR_CAPACITY / SC_ERR_TIMEOUT
+ *     otherwise (first error wins).  The caller zeroes it beforehand.  Kernels never trap.
+ *   - Tensors are row-major with the head dimension d innermost and contiguous; device
+ *     pointers of K, V, q, cores and out must be 16-byte aligned.  d must be 128 for SC_BF16
+ *     fast paths; the generic path takes any d that is a multiple of 8 up to 256.
+ *   - Results are deterministic: the same inputs give bit-identical outputs.
+ */
+#ifndef SEMANTICACHE_H_
+#define SEMANTICACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SC_API __attribute__((visibility("default")))
+#else
+#define SC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SC_OK = 0,
+    SC_ERR_INVALID_ARG = 1,
+    SC_ERR_UNSUPPORTED = 2,
+    SC_ERR_CAPACITY = 3,
+    SC_ERR_CUDA = 4,
+    SC_ERR_TIMEOUT = 5
+} sc_status;
+
+typedef enum { SC_BF16 = 0, SC_F32 = 1 } sc_dtype;
+
+/* sc_gsc_params.flags */
+#define SC_FLAG_GENERIC 1u     /* force the generic (CUDA-core, any dtype) kernels */
+#define SC_FLAG_TWO_PASS 2u    /* fused compress: count pass + write pass instead of the
+                                  single pass whose tiles look back for their output offset */
+
+typedef struct {
+    float tau;             /* similarity threshold of Algorithm 1; merge iff Sim > tau (strict) */
+    int32_t max_chunk_len; /* must equal the value given to sc_chunk; 1..SC_MAX_CHUNK_LEN */
+    uint32_t flags;        /* SC_FLAG_* */
+} sc_gsc_params;
+
+/* Element strides of a [B, Hkv, n, d] tensor (d contiguous). */
+typedef struct { int64_t b, h, n; } sc_strides;
+
+#define SC_MAX_CHUNK_LEN 256
+#define SC_MAX_DELIMS 64
+#define SC_TILE_ROWS 128       /* rows a compress tile packs (one longer chunk is a tile alone) */
+
+/* Library / build identification: returns a static string. */
+SC_API const char* sc_version(void);
+
+/*
+ * Upper bounds for the outputs of sc_chunk, so a caller can allocate without a sync:
+ * segments <= *n_seg_cap = B*n in total, tiles <= *n_tile_cap per sequence.  Both pointers are HOST.
+ */
+SC_API sc_status sc_chunk_bounds(int32_t B, int32_t n, int32_t* n_seg_cap /*HOST out*/,
+                          int32_t* n_tile_cap /*HOST out*/);
+
+/*
+ * Semantic chunking (Sec. 2.2, Eq. 1).  The token axis of each sequence is cut into the
+ * alternating series (C_1, d_1, C_2, ...): every maximal run of non-delimiter tokens is one
+ * segment, cut every max_chunk_len tokens if longer; every delimiter token is a segment of
+ * length one (clustering a one-token segment returns the token unchanged, which is how the
+ * delimiters' K/V stay unmodified); empty runs produce nothing; no segment spans sequences.
+ * Depends on token ids only, so one call serves every layer and KV head.
+ *
+ *   token_ids    [B, n] int32
+ *   delim_ids    HOST, n_delim <= SC_MAX_DELIMS ids
+ *   seg_off      out [n_seg+1]: start of each segment on the flattened [B*n] axis, then B*n.
+ *                Capacity n_seg_cap+1 entries.
+ *   seq_seg_off  out [B+1]: first segment of each sequence, then n_seg
+ *   n_seg        out [1]
+ *   tile_seg     out [B, n_tile_cap+1]: work partition for sc_compress.  Row b lists the tiles of
+ *                sequence b: tile t covers segments [tile_seg[b][t], tile_seg[b][t+1]) -- as many
+ *                consecutive segments as fit in SC_TILE_ROWS tokens, or one longer segment
+ *                alone.  n_tile_cap from sc_chunk_bounds always suffices.
+ *   seq_tile_cnt out [B]: number of tiles of each sequence
+ *   workspace    scratch of at least sc_chunk_workspace_bytes(B, n) bytes
+ *   status       SC_ERR_CAPACITY if n_seg > n_seg_cap or a sequence needs more than n_tile_cap
+ *                tiles (writes clamped; n_seg and seq_tile_cnt still report the needed sizes)
+ * B == 0 or n == 0 is valid and yields empty offsets.
+ */
+SC_API size_t sc_chunk_workspace_bytes(int32_t B, int32_t n);
+
+SC_API sc_status sc_chunk(const int32_t* token_ids, int32_t B, int32_t n,
+                   const int32_t* delim_ids /*HOST*/, int32_t n_delim, int32_t max_chunk_len,
+                   int32_t* seg_off, int32_t n_seg_cap, int32_t* seq_seg_off, int32_t* n_seg,
+                   int32_t* tile_seg, int32_t n_tile_cap, int32_t* seq_tile_cnt,
+                   void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
+ * Compress one layer (Sec. 2.3-2.4).  For every (sequence b, KV head h, segment) independently:
+ * Greedy Seed-Based Clustering (Algorithm 1) on the cosine similarity of the keys (Eq. 2; a
+ * zero-norm key has similarity 0 to everything), then each cluster S_t is mean-pooled into one
+ * core k_hat = mean(k_i), v_hat = mean(v_i) (Eq. 3; fp32 sums in token order, rounded once to
+ * the storage dtype) with count = |S_t|.  Cores are written compactly in position order of
+ * their seeds; a delimiter is a core of count 1 carrying its K/V bits unchanged.
+ *
+ *   K, V        [B, Hkv, n, d] with element strides kv_strides (both tensors), dtype dt
+ *   seg_off .. seq_tile_cnt, n_tile_cap   as produced by / given to sc_chunk for the same B, n,
+ *               max_chunk_len
+ *   params      HOST
+ *   core_k/v    out [B, Hkv, cap, d] contiguous, dtype dt; rows < core_len[b,h] are valid
+ *   count       out [B, Hkv, cap] int32, >= 1 on valid rows
+ *   core_len    out [B, Hkv]: number of cores of each head (the needed length even when it
+ *               exceeds cap; then status = SC_ERR_CAPACITY and rows >= cap are not written).
+ *               cap = n always suffices.
+ *   assign      optional out [B, Hkv, n] int32: for each token the position (within its
+ *               sequence) of the seed of its cluster; NULL to skip
+ *   workspace   at least sc_compress_workspace_bytes(B, Hkv, n) bytes
+ */
+SC_API size_t sc_compress_workspace_bytes(int32_t B, int32_t Hkv, int32_t n);
+
+SC_API sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dtype dt,
+                      int32_t B, int32_t Hkv, int32_t n, int32_t d,
+                      const int32_t* seg_off, const int32_t* seq_seg_off, const int32_t* n_seg,
+                      const int32_t* tile_seg, const int32_t* seq_tile_cnt, int32_t n_tile_cap,
+                      const sc_gsc_params* params /*HOST*/,
+                      void* core_k, void* core_v, int32_t* count, int32_t cap, int32_t* core_len,
+                      int32_t* assign, void* workspace, size_t workspace_bytes,
+                      int32_t* status, void* stream);
+
+/*
+ * One decode step of Proportional Attention (Sec. 2.4, Eq. 4) for one layer.  For every query
+ * head hq of sequence b, with KV head h = hq / (Hq/Hkv):
+ *     x_t = scale * <q, k_hat_t> + ln(count_t),  out = sum_t softmax(x)_t * v_hat_t
+ * over rows t < core_len[b, h].  The whole query group of a KV head is served in one pass over
+ * that head's cores; long heads are split along t and the partial (max, sum, acc) triples are
+ * combined by the last block to finish.
+ *
+ *   q          [B, Hq, d] contiguous, dtype dt
+ *   core_k/v   [B, Hkv, cap, d] contiguous, dtype dt;  count [B, Hkv, cap] int32, or NULL for
+ *              all ones (plain attention over an uncompressed cache)
+ *   core_len   [B, Hkv] int32 (device), each <= cap
+ *   scale      0 means 1/sqrt(d)
+ *   out        [B, Hq, d] contiguous, dtype dt; a head with core_len 0 gets zeros
+ *   flags      SC_FLAG_GENERIC forces the generic kernels; 0 otherwise
+ *   workspace  at least sc_decode_workspace_bytes(B, Hq, Hkv, d, cap) bytes.  It holds the
+ *              split partials and a few arrival counters; the counters must be zero on entry
+ *              and are left zero on exit, so zero the workspace once after allocating it.
+ */
+SC_API size_t sc_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap);
+
+SC_API sc_status sc_decode_attn(const void* q, sc_dtype dt, int32_t B, int32_t Hq, int32_t Hkv, int32_t d,
+                         const void* core_k, const void* core_v, const int32_t* count, int32_t cap,
+                         const int32_t* core_len, float scale, uint32_t flags, void* out,
+                         void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SEMANTICACHE_H_ */

@@ -1,0 +1,137 @@
+// C-ABI entry points: argument validation and dispatch.  See include/semanticache.h.
+#include "common.cuh"
+
+using namespace sc;
+
+namespace sc {
+// fused bf16 paths (compress_fused.cu, decode_mma.cu)
+bool compress_fused_supported(const CompressArgs& a);
+cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st);
+size_t compress_fused_ws_bytes(int32_t B, int32_t Hkv, int32_t n);
+bool decode_mma_supported(const DecodeArgs& a);
+cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);
+size_t decode_mma_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap);
+}  // namespace sc
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline int tile_cap_for(int32_t n) { return 2 * div_up(n, SC_TILE_ROWS) + 1; }
+
+extern "C" {
+
+const char* sc_version(void) { return "semanticache-b200 0.1 (sm_100a)"; }
+
+sc_status sc_chunk_bounds(int32_t B, int32_t n, int32_t* n_seg_cap, int32_t* n_tile_cap) {
+    if (B < 0 || n < 0 || (int64_t)B * n > 0x7fffffff - 1) return SC_ERR_INVALID_ARG;
+    if (n_seg_cap) *n_seg_cap = B * n;
+    if (n_tile_cap) *n_tile_cap = tile_cap_for(n);
+    return SC_OK;
+}
+
+size_t sc_chunk_workspace_bytes(int32_t B, int32_t n) {
+    if (B <= 0 || n <= 0) return 256;
+    return chunk_ws_bytes(B, n);
+}
+
+sc_status sc_chunk(const int32_t* token_ids, int32_t B, int32_t n, const int32_t* delim_ids, int32_t n_delim,
+                   int32_t max_chunk_len, int32_t* seg_off, int32_t n_seg_cap, int32_t* seq_seg_off,
+                   int32_t* n_seg, int32_t* tile_seg, int32_t n_tile_cap, int32_t* seq_tile_cnt,
+                   void* workspace, size_t workspace_bytes, int32_t* status, void* stream) {
+    if (B < 0 || n < 0 || (int64_t)B * n > 0x7fffffff - 1) return SC_ERR_INVALID_ARG;
+    if (n_delim < 0 || n_delim > SC_MAX_DELIMS || (n_delim > 0 && !delim_ids)) return SC_ERR_INVALID_ARG;
+    if (max_chunk_len < 1 || max_chunk_len > SC_MAX_CHUNK_LEN) return SC_ERR_INVALID_ARG;
+    if (!seg_off || !seq_seg_off || !n_seg || !tile_seg || !seq_tile_cnt) return SC_ERR_INVALID_ARG;
+    if (n_seg_cap < 0 || n_tile_cap < 0) return SC_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (B == 0 || n == 0) {  // nothing to chunk: empty offsets
+        cudaError_t e = cudaMemsetAsync(n_seg, 0, sizeof(int32_t), st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(seq_seg_off, 0, sizeof(int32_t) * (B + 1), st);
+        if (e == cudaSuccess) e = cudaMemsetAsync(seg_off, 0, sizeof(int32_t), st);
+        if (e == cudaSuccess && B > 0) e = cudaMemsetAsync(seq_tile_cnt, 0, sizeof(int32_t) * B, st);
+        for (int b = 0; e == cudaSuccess && b < B; ++b)
+            e = cudaMemsetAsync(tile_seg + (int64_t)b * (n_tile_cap + 1), 0, sizeof(int32_t), st);
+        return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+    }
+    if (!token_ids || !workspace || workspace_bytes < chunk_ws_bytes(B, n)) return SC_ERR_INVALID_ARG;
+    ChunkArgs a;
+    a.token_ids = token_ids; a.B = B; a.n = n;
+    for (int i = 0; i < SC_MAX_DELIMS; ++i) a.delim[i] = i < n_delim ? delim_ids[i] : 0;
+    a.n_delim = n_delim; a.max_chunk_len = max_chunk_len;
+    a.seg_off = seg_off; a.n_seg_cap = n_seg_cap; a.seq_seg_off = seq_seg_off; a.n_seg = n_seg;
+    a.tile_seg = tile_seg; a.n_tile_cap = n_tile_cap; a.seq_tile_cnt = seq_tile_cnt;
+    a.ws = (int32_t*)workspace; a.status = status;
+    return launch_chunk(a, st) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
+size_t sc_compress_workspace_bytes(int32_t B, int32_t Hkv, int32_t n) {
+    if (B <= 0 || Hkv <= 0 || n <= 0) return 256;
+    size_t a = compress_generic_ws_bytes(B, Hkv, n), b = compress_fused_ws_bytes(B, Hkv, n);
+    return a > b ? a : b;
+}
+
+sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dtype dt, int32_t B, int32_t Hkv,
+                      int32_t n, int32_t d, const int32_t* seg_off, const int32_t* seq_seg_off,
+                      const int32_t* n_seg, const int32_t* tile_seg, const int32_t* seq_tile_cnt,
+                      int32_t n_tile_cap, const sc_gsc_params* params, void* core_k, void* core_v, int32_t* count,
+                      int32_t cap, int32_t* core_len, int32_t* assign, void* workspace, size_t workspace_bytes,
+                      int32_t* status, void* stream) {
+    if (B < 0 || Hkv <= 0 || n < 0 || cap < 0 || !params || !core_len) return SC_ERR_INVALID_ARG;
+    if (dt != SC_BF16 && dt != SC_F32) return SC_ERR_UNSUPPORTED;
+    if (d < 8 || d > 256 || (d % 8) != 0) return SC_ERR_UNSUPPORTED;
+    if (params->max_chunk_len < 1 || params->max_chunk_len > SC_MAX_CHUNK_LEN) return SC_ERR_INVALID_ARG;
+    if (!(params->tau == params->tau)) return SC_ERR_INVALID_ARG;  // NaN threshold
+    cudaStream_t st = (cudaStream_t)stream;
+    if (B == 0 || n == 0) {
+        if (B == 0) return SC_OK;
+        return cudaMemsetAsync(core_len, 0, sizeof(int32_t) * (size_t)B * Hkv, st) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+    }
+    if (!K || !V || !seg_off || !seq_seg_off || !n_seg || !tile_seg || !seq_tile_cnt) return SC_ERR_INVALID_ARG;
+    if (!core_k || !core_v || !count || !workspace) return SC_ERR_INVALID_ARG;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(core_k) || !aligned16(core_v)) return SC_ERR_INVALID_ARG;
+    const size_t esz = dt == SC_BF16 ? 2 : 4;
+    if ((kv_strides.b * esz) % 16 || (kv_strides.h * esz) % 16 || (kv_strides.n * esz) % 16) return SC_ERR_INVALID_ARG;
+    if (kv_strides.n < d) return SC_ERR_INVALID_ARG;
+    if ((int64_t)B * n > 0x7fffffff - 1) return SC_ERR_INVALID_ARG;
+    if (workspace_bytes < sc_compress_workspace_bytes(B, Hkv, n)) return SC_ERR_INVALID_ARG;
+    CompressArgs a;
+    a.K = K; a.V = V; a.st = kv_strides; a.dt = dt; a.B = B; a.Hkv = Hkv; a.n = n; a.d = d;
+    a.seg_off = seg_off; a.seq_seg_off = seq_seg_off; a.n_seg = n_seg;
+    a.tile_seg = tile_seg; a.seq_tile_cnt = seq_tile_cnt; a.n_tile_cap = n_tile_cap;
+    a.tau = params->tau; a.max_chunk_len = params->max_chunk_len; a.flags = params->flags;
+    a.core_k = core_k; a.core_v = core_v; a.count = count; a.cap = cap; a.core_len = core_len;
+    a.assign = assign; a.ws = workspace; a.status = status;
+    cudaError_t e;
+    if (!(a.flags & SC_FLAG_GENERIC) && compress_fused_supported(a)) e = launch_compress_fused(a, st);
+    else e = launch_compress_generic(a, st);
+    return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
+size_t sc_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || cap < 0) return 256;
+    size_t a = decode_generic_ws_bytes(B, Hq, Hkv, d, cap), b = decode_mma_ws_bytes(B, Hq, Hkv, d, cap);
+    return a > b ? a : b;
+}
+
+sc_status sc_decode_attn(const void* q, sc_dtype dt, int32_t B, int32_t Hq, int32_t Hkv, int32_t d,
+                         const void* core_k, const void* core_v, const int32_t* count, int32_t cap,
+                         const int32_t* core_len, float scale, uint32_t flags, void* out, void* workspace,
+                         size_t workspace_bytes, int32_t* status, void* stream) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || cap < 0 || (Hq % Hkv) != 0) return SC_ERR_INVALID_ARG;
+    if (dt != SC_BF16 && dt != SC_F32) return SC_ERR_UNSUPPORTED;
+    if (d < 8 || d > 256 || (d % 8) != 0) return SC_ERR_UNSUPPORTED;
+    if (!(scale == scale) || scale < 0.f) return SC_ERR_INVALID_ARG;
+    if (B == 0) return SC_OK;
+    if (!q || !out || !core_len || !workspace) return SC_ERR_INVALID_ARG;
+    if (cap > 0 && (!core_k || !core_v)) return SC_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(core_k) || !aligned16(core_v)) return SC_ERR_INVALID_ARG;
+    if (workspace_bytes < sc_decode_workspace_bytes(B, Hq, Hkv, d, cap)) return SC_ERR_INVALID_ARG;
+    DecodeArgs a;
+    a.q = q; a.dt = dt; a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.d = d; a.core_k = core_k; a.core_v = core_v;
+    a.count = count; a.cap = cap; a.core_len = core_len; a.scale = scale; a.out = out; a.ws = workspace;
+    a.status = status;
+    cudaError_t e;
+    if (!(flags & SC_FLAG_GENERIC) && decode_mma_supported(a)) e = launch_decode_mma(a, (cudaStream_t)stream);
+    else e = launch_decode_generic(a, (cudaStream_t)stream);
+    return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,271 @@
+"""GPU parity: every product of the CUDA path against the CPU oracle on the same seeded bytes.
+
+All calls go through the C-ABI library (via the ctypes binding).  Offsets, assignments, counts
+and lengths are compared bit-exactly; merged K/V and attention outputs with the tolerance in
+helpers.py.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import (TOL, assert_close_vectors, compare_compressed, compare_plan, layer_from_oracle,
+                     oracle_compress, to_f64)
+from paper_2603_14303_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+DELIMS = synth.DELIMS
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ---------------------------------------------------------------------------------- sc_chunk
+
+
+def _chunk_both(ids_np, max_len):
+    ids = torch.from_numpy(ids_np).to(DEV)
+    plan = binding.chunk(ids, DELIMS, max_len)
+    seg_off, seq_seg_off = oracle.chunk(ids_np, DELIMS, max_len)
+    compare_plan(plan, seg_off, seq_seg_off)
+    return plan
+
+
+def test_chunk_hand_worked_cases():
+    for line in open(os.path.join(GOLDEN, "chunk_cases.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        ids, max_len, expect = [p.split() for p in line.split(";")]
+        plan = _chunk_both(np.array([[int(x) for x in ids]], dtype=np.int32), int(max_len[0]))
+        n_seg = int(plan.n_seg.item())
+        assert plan.seg_off[: n_seg + 1].tolist() == [int(x) for x in expect]
+
+
+@pytest.mark.parametrize("B,n,p_delim,max_len", [
+    (1, 1, 0.0, 256), (1, 1, 1.0, 256), (1, 2047, 0.05, 256), (1, 2048, 0.05, 256), (2, 2049, 0.05, 256),
+    (3, 5000, 0.0, 256), (3, 5000, 1.0, 256), (2, 6000, 0.0, 7), (2, 4500, 0.3, 3), (1, 10000, 0.002, 100),
+    (4, 4096, 0.04, 1), (1, 70000, 0.045, 256), (1, 9000, 0.0005, 256)])
+def test_chunk_matches_oracle(B, n, p_delim, max_len):
+    rng = np.random.default_rng(B * 1000 + n)
+    ids = rng.integers(100, 30000, size=(B, n)).astype(np.int32)
+    mask = rng.random((B, n)) < p_delim
+    ids[mask] = rng.choice(DELIMS, size=int(mask.sum()))
+    _chunk_both(ids, max_len)
+
+
+def test_chunk_empty_input_and_capacity_error():
+    ids = torch.zeros((2, 0), dtype=torch.int32, device=DEV)
+    plan = binding.chunk(ids, DELIMS, 256)
+    assert int(plan.n_seg.item()) == 0 and plan.seq_seg_off.tolist() == [0, 0, 0] and plan.seq_tile_cnt.tolist() == [0, 0]
+    # too-small segment capacity: status says so, n_seg still reports the need, nothing out of bounds
+    ids_np = np.full((1, 300), 13, dtype=np.int32)
+    t = torch.from_numpy(ids_np).to(DEV)
+    i32 = dict(dtype=torch.int32, device=DEV)
+    canary = 0x5A5A5A5A
+    seg_off = torch.full((100 + 1 + 8,), canary, **i32)
+    tile_seg = torch.full((1, 7 + 8), canary, **i32)
+    st = torch.zeros(1, **i32)
+    ws = torch.empty(binding.lib().sc_chunk_workspace_bytes(1, 300), dtype=torch.uint8, device=DEV)
+    n_seg, sso, stc = torch.zeros(1, **i32), torch.zeros(2, **i32), torch.zeros(1, **i32)
+    binding.sc_chunk(t, DELIMS, 256, seg_off[:101], sso, n_seg, tile_seg[:, :7], stc, ws, st)
+    assert int(st.item()) == binding.SC_ERR_CAPACITY and int(n_seg.item()) == 300
+    assert torch.all(seg_off[101:] == canary) and torch.all(tile_seg[:, 7:] == canary)
+    assert seg_off[:100].tolist() == list(range(100))
+
+
+# ------------------------------------------------------------------------------- sc_compress
+
+
+def _compress_both(w, layer=0, flags=0, cap=None, strided=False, tau=None):
+    tau = w.tau if tau is None else tau
+    ids, run_id, run_lens = synth.token_ids(w)
+    K, V = synth.layer_kv(w, layer, run_id, run_lens)          # CPU bytes, shared by both sides
+    ref = oracle_compress(ids, K, V, w.delims, tau, w.max_chunk_len, cap)
+    Kd, Vd = K.to(DEV), V.to(DEV)
+    if strided:  # [B, n, Hkv, d] storage viewed as [B, Hkv, n, d]
+        Kd = Kd.transpose(1, 2).contiguous().transpose(1, 2)
+        Vd = Vd.transpose(1, 2).contiguous().transpose(1, 2)
+    plan = binding.chunk(ids.to(DEV), w.delims, w.max_chunk_len)
+    got = binding.compress(Kd, Vd, plan, tau, cap=cap, want_assign=True, flags=flags)
+    return ref, got, plan, (K, V)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC, binding.SC_FLAG_TWO_PASS])
+def test_compress_cfg0_matches_oracle(dtype, flags):
+    w = synth.config(0, dtype=dtype)
+    ref, got, plan, _ = _compress_both(w, flags=flags)
+    assert ref["margin"] > 1e-3
+    binding.check_status(plan.status)
+    compare_compressed(got, ref, torch.bfloat16 if dtype == "bf16" else torch.float32)
+    kept = ref["core_len"].sum() / (w.Hkv * w.n)
+    assert 0.1 < kept < 0.5
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC, binding.SC_FLAG_TWO_PASS])
+@pytest.mark.parametrize("length", [1, 2, 31, 32, 33, 63, 64, 65, 127, 128, 129, 200, 255, 256])
+def test_compress_fixed_chunk_lengths(length, flags):
+    w = synth.config(0, n=3000, Hkv=2, Hq=8, gap=("fixed", length), centroids=("uniform", 5), seed=length)
+    ref, got, plan, _ = _compress_both(w, flags=flags)
+    assert ref["margin"] > 1e-4
+    binding.check_status(plan.status)
+    compare_compressed(got, ref, torch.bfloat16)
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+def test_compress_ragged_lognormal_batch(flags):
+    w = synth.config(2, B=3, n=5000, Hkv=2, Hq=8, L=1)
+    ref, got, plan, _ = _compress_both(w, flags=flags)
+    assert ref["margin"] > 1e-4
+    compare_compressed(got, ref, torch.bfloat16)
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+@pytest.mark.parametrize("max_len", [256, 16, 5])
+def test_compress_hard_cut_and_no_delimiters(flags, max_len):
+    w = synth.config(0, n=1500, Hkv=2, Hq=8, gap=("fixed", 100000), max_chunk_len=max_len, centroids=("uniform", 3))
+    ref, got, plan, _ = _compress_both(w, flags=flags)
+    compare_compressed(got, ref, torch.bfloat16)
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+def test_compress_threshold_extremes(flags):
+    w = synth.config(0, n=1024, Hkv=2, Hq=8)
+    for tau in (2.0, -2.0, 1.0):
+        ref, got, plan, (K, V) = _compress_both(w, flags=flags, tau=tau)
+        compare_compressed(got, ref, torch.bfloat16)
+        if tau >= 1.0:  # nothing merges: the compressed cache is the cache, bit for bit
+            assert torch.equal(got.core_k.cpu(), K) and torch.equal(got.core_v.cpu(), V)
+            assert torch.all(got.count == 1) and torch.all(got.core_len == w.n)
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+def test_compress_all_identical_and_zero_keys(flags):
+    w = synth.config(0, n=700, Hkv=2, Hq=8)
+    ids, run_id, run_lens = synth.token_ids(w)
+    K, V = synth.layer_kv(w, 0, run_id, run_lens)
+    K[:, 0] = K[:, 0, :1]            # head 0: every key identical -> one cluster per segment
+    K[:, 1, 100:140] = 0             # head 1: a stretch of zero-norm keys (Sim := 0 < tau)
+    ref = oracle_compress(ids, K, V, w.delims, 0.7)
+    plan = binding.chunk(ids.to(DEV), w.delims)
+    got = binding.compress(K.to(DEV), V.to(DEV), plan, 0.7, want_assign=True, flags=flags)
+    compare_compressed(got, ref, torch.bfloat16)
+    n_seg = int(plan.n_seg.item())
+    assert int(got.core_len[0, 0]) == n_seg
+    # zero keys with a negative threshold: Sim = 0 > tau merges them
+    ref = oracle_compress(ids, K, V, w.delims, -0.5)
+    got = binding.compress(K.to(DEV), V.to(DEV), plan, -0.5, want_assign=True, flags=flags)
+    compare_compressed(got, ref, torch.bfloat16)
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+def test_compress_strided_layout_and_determinism(flags):
+    w = synth.config(0, n=2048, B=2)
+    ref, got, plan, (K, V) = _compress_both(w, flags=flags, strided=True)
+    compare_compressed(got, ref, torch.bfloat16)
+    again = binding.compress(K.to(DEV), V.to(DEV), plan, w.tau, want_assign=True, flags=flags)
+    L = got.core_len.cpu().numpy()
+    assert torch.equal(again.core_len, got.core_len) and torch.equal(again.assign, got.assign)
+    for b in range(w.B):
+        for h in range(w.Hkv):
+            assert torch.equal(again.core_k[b, h, : L[b, h]], got.core_k[b, h, : L[b, h]])
+            assert torch.equal(again.core_v[b, h, : L[b, h]], got.core_v[b, h, : L[b, h]])
+            assert torch.equal(again.count[b, h, : L[b, h]], got.count[b, h, : L[b, h]])
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+def test_compress_capacity_overflow_is_reported_not_written(flags):
+    w = synth.config(0, n=1024, Hkv=2, Hq=8)
+    ids, run_id, run_lens = synth.token_ids(w)
+    K, V = synth.layer_kv(w, 0, run_id, run_lens)
+    full = oracle_compress(ids, K, V, w.delims, w.tau)
+    cap = int(full["core_len"].min()) - 5
+    plan = binding.chunk(ids.to(DEV), w.delims)
+    canary = 12345
+    # carve the [1, 2, cap, *] outputs out of larger buffers whose tails hold a canary
+    flat_k = torch.full((2 * cap * 128 + 4096,), 7.0, dtype=torch.bfloat16, device=DEV)
+    flat_v = torch.full((2 * cap * 128 + 4096,), 7.0, dtype=torch.bfloat16, device=DEV)
+    flat_c = torch.full((2 * cap + 4096,), canary, dtype=torch.int32, device=DEV)
+    view = binding.CompressedLayer(flat_k[: 2 * cap * 128].view(1, 2, cap, 128), flat_v[: 2 * cap * 128].view(1, 2, cap, 128),
+                                   flat_c[: 2 * cap].view(1, 2, cap), torch.zeros((1, 2), dtype=torch.int32, device=DEV))
+    binding.compress(K.to(DEV), V.to(DEV), plan, w.tau, cap=cap, out=view, flags=flags)
+    assert int(plan.status.item()) == binding.SC_ERR_CAPACITY
+    assert np.array_equal(view.core_len.cpu().numpy(), full["core_len"])
+    assert np.array_equal(view.count.cpu().numpy(), full["count"][:, :, :cap])
+    assert torch.all(flat_c[2 * cap:] == canary)
+    assert torch.all(flat_k[2 * cap * 128:] == 7.0) and torch.all(flat_v[2 * cap * 128:] == 7.0)
+    # head 0 overflowed too: its surplus rows must not have spilled into head 1's first rows
+    ref_cap = oracle_compress(ids, K, V, w.delims, w.tau, cap=cap)
+    compare_compressed(view, ref_cap, torch.bfloat16)
+
+
+# ---------------------------------------------------------------------------- sc_decode_attn
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+def test_decode_cfg0_end_to_end_and_on_oracle_cores(dtype, flags):
+    w = synth.config(0, dtype=dtype)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    ref, got, plan, _ = _compress_both(w)
+    ref_layer = layer_from_oracle(ref, tdt, DEV)
+    ws = binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, w.n, DEV)
+    for step in range(w.decode_steps):
+        q = synth.queries(w, step, 0)
+        want = oracle.attn(synth.to_numpy_bits(q), ref["core_k"], ref["core_v"], ref["count"], ref["core_len"])
+        out_e2e = binding.decode_attn(q.to(DEV), got, workspace=ws, flags=flags)
+        out_iso = binding.decode_attn(q.to(DEV), ref_layer, workspace=ws, flags=flags)
+        assert_close_vectors(to_f64(out_iso), want, TOL[tdt], f"decode on oracle cores, step {step}")
+        assert_close_vectors(to_f64(out_e2e), want, TOL[tdt], f"decode end to end, step {step}")
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+@pytest.mark.parametrize("Hkv,G", [(4, 7), (2, 1), (2, 8), (3, 2)])
+def test_decode_gqa_shapes_ragged_lengths_and_plain_attention(Hkv, G, flags):
+    rng = np.random.default_rng(Hkv * 10 + G)
+    B, d, cap = 3, 128, 1500
+    ck = torch.from_numpy(rng.normal(size=(B, Hkv, cap, d)).astype(np.float32)).to(torch.bfloat16)
+    cv = torch.from_numpy(rng.normal(size=(B, Hkv, cap, d)).astype(np.float32)).to(torch.bfloat16)
+    cnt = torch.from_numpy(rng.integers(1, 40, size=(B, Hkv, cap)).astype(np.int32))
+    clen = torch.from_numpy(rng.integers(0, cap + 1, size=(B, Hkv)).astype(np.int32))
+    clen[0, 0], clen[1, 0], clen[2, Hkv - 1] = 0, 1, cap           # empty, single row, full
+    if Hkv > 1:
+        clen[0, 1] = 17
+    q = torch.from_numpy(rng.normal(size=(B, Hkv * G, d)).astype(np.float32)).to(torch.bfloat16)
+    layer = binding.CompressedLayer(ck.to(DEV), cv.to(DEV), cnt.to(DEV), clen.to(DEV))
+    for use_count in (True, False):
+        want = oracle.attn(synth.to_numpy_bits(q), synth.to_numpy_bits(ck), synth.to_numpy_bits(cv),
+                           cnt.numpy() if use_count else None, clen.numpy())
+        out = binding.decode_attn(q.to(DEV), layer, flags=flags, use_count=use_count)
+        assert_close_vectors(to_f64(out), want, 1e-2, f"decode G={G} count={use_count}")
+        assert torch.all(out[0, :G] == 0), "a head without cores yields zeros"
+
+
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+def test_decode_is_deterministic_and_scale_is_honoured(flags):
+    w = synth.config(0, n=4096)
+    ref, got, plan, _ = _compress_both(w)
+    q = synth.queries(w, 0, 0).to(DEV)
+    ws = binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, w.n, DEV)
+    a = binding.decode_attn(q, got, workspace=ws, flags=flags)
+    b = binding.decode_attn(q, got, workspace=ws, flags=flags)
+    assert torch.equal(a, b)
+    c = binding.decode_attn(q, got, workspace=ws, flags=flags, scale=0.05)
+    want = oracle.attn(synth.to_numpy_bits(q), ref["core_k"], ref["core_v"], ref["count"], ref["core_len"], scale=0.05)
+    assert_close_vectors(to_f64(c), want, 1e-2, "custom scale")
+
+
+def test_no_merge_compress_then_decode_equals_exact_attention():
+    """tau >= 1: the whole path must reproduce exact softmax attention over the raw cache."""
+    w = synth.config(0, n=1536)
+    ref, got, plan, (K, V) = _compress_both(w, tau=2.0)
+    q = synth.queries(w, 0, 0)
+    out = binding.decode_attn(q.to(DEV), got)
+    Kf, Vf, qf = K.double(), V.double(), q.double()
+    G = w.G
+    for hq in range(w.Hq):
+        s = (Kf[0, hq // G] @ qf[0, hq]) / np.sqrt(w.d)
+        want = torch.softmax(s, 0) @ Vf[0, hq // G]
+        assert_close_vectors(to_f64(out[0, hq]), want.numpy(), 1e-2, f"exact attention head {hq}")
