@@ -72,6 +72,12 @@ typedef struct { int64_t b, h, n; } sc_strides;
 SC_API const char* sc_version(void);
 
 /*
+ * Statistics: number of kernels this library has launched (or recorded into a CUDA graph under
+ * stream capture) since it was loaded.  The only state the library keeps; it affects nothing.
+ */
+SC_API uint64_t sc_launch_counter(void);
+
+/*
  * Upper bounds for the outputs of sc_chunk, so a caller can allocate without a sync:
  * segments <= *n_seg_cap = B*n in total, tiles <= *n_tile_cap per sequence.  Both pointers are HOST.
  */

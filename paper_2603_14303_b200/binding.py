@@ -22,7 +22,7 @@ SC_MAX_CHUNK_LEN, SC_MAX_DELIMS, SC_TILE_ROWS = 256, 64, 128
 _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CAPACITY", "SC_ERR_CUDA",
                  "SC_ERR_TIMEOUT"]
 
-EXPORTS = ["sc_version", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
+EXPORTS = ["sc_version", "sc_launch_counter", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
            "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn"]
 
 
@@ -53,6 +53,7 @@ def lib() -> ctypes.CDLL:
                                "(there is no fallback implementation)")
         L = ctypes.CDLL(LIB_PATH)
         L.sc_version.restype = ctypes.c_char_p
+        L.sc_launch_counter.restype = ctypes.c_uint64
         L.sc_chunk_bounds.restype = _i32
         L.sc_chunk_bounds.argtypes = [_i32, _i32, ctypes.POINTER(_i32), ctypes.POINTER(_i32)]
         for f in (L.sc_chunk_workspace_bytes, L.sc_compress_workspace_bytes, L.sc_decode_workspace_bytes):
@@ -98,6 +99,11 @@ def _need_cuda(*ts):
     for t in ts:
         if t is not None and not t.is_cuda:
             raise ValueError("device tensors required")
+
+
+def launch_counter() -> int:
+    """Kernels launched (or captured into a graph) by the library since it was loaded."""
+    return int(lib().sc_launch_counter())
 
 
 def chunk_bounds(B: int, n: int):

@@ -13,12 +13,18 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);
 size_t decode_mma_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap);
 }  // namespace sc
 
+#include <atomic>
+static std::atomic<uint64_t> g_launches{0};
+namespace sc { void note_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); } }
+
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline int tile_cap_for(int32_t n) { return 2 * div_up(n, SC_TILE_ROWS) + 1; }
 
 extern "C" {
 
 const char* sc_version(void) { return "semanticache-b200 0.1 (sm_100a)"; }
+
+uint64_t sc_launch_counter(void) { return g_launches.load(std::memory_order_relaxed); }
 
 sc_status sc_chunk_bounds(int32_t B, int32_t n, int32_t* n_seg_cap, int32_t* n_tile_cap) {
     if (B < 0 || n < 0 || (int64_t)B * n > 0x7fffffff - 1) return SC_ERR_INVALID_ARG;

@@ -273,6 +273,7 @@ cudaError_t launch_chunk(const ChunkArgs& a, cudaStream_t st) {
                                                  a.seg_off, a.n_seg_cap);
     chunk_pack_tiles<<<a.B, kChunkThreads, 0, st>>>(a.seg_off, a.seq_seg_off, a.n_seg_cap, a.tile_seg,
                                                     a.n_tile_cap, a.seq_tile_cnt, a.status);
+    note_launches(5);
     return cudaGetLastError();
 }
 

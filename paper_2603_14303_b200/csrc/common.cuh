@@ -68,6 +68,9 @@ __device__ __forceinline__ int warp_scan_max(int v, int lane) {
 
 inline int div_up(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
+// Statistics only: kernels launched (or captured into a graph) by this library since load.
+void note_launches(int n);
+
 // --- launch entry points implemented in the .cu files (host side) ---------------------------
 
 struct ChunkArgs {

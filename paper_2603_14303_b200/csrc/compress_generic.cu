@@ -181,6 +181,7 @@ static cudaError_t run(const CompressArgs& a, cudaStream_t st) {
     merge_generic<T><<<grid, kGenWarps * 32, 0, st>>>((const T*)a.K, (const T*)a.V, a.st, a.B, a.Hkv, a.n, a.d,
                                                       a.seg_off, a.n_seg, seg_stride, assign, seg_core_off,
                                                       (T*)a.core_k, (T*)a.core_v, a.count, a.cap);
+    note_launches(3);
     return cudaGetLastError();
 }
 

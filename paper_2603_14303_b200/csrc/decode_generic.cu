@@ -119,6 +119,7 @@ static cudaError_t run(const DecodeArgs& a, cudaStream_t st) {
     const int64_t heads = (int64_t)a.B * a.Hq;
     combine_generic<T><<<div_up(heads, kDecWarps), kDecWarps * 32, 0, st>>>(heads, a.d, n_split, (const float*)a.ws,
                                                                           (T*)a.out);
+    note_launches(2);
     return cudaGetLastError();
 }
 
