@@ -111,11 +111,14 @@ class Pipeline:
                                                torch.zeros((w.B, w.Hkv, self.cap), **i32),
                                                torch.zeros((w.B, w.Hkv), **i32)) for _ in range(w.L)]
         self.cws = binding.compress_workspace(w.B, w.Hkv, w.n, device)
-        self.dws = binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, self.cap, device)
+        # one workspace per layer: consecutive layer launches overlap and must not share scratch
+        self.dws = [binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, self.cap, device) for _ in range(w.L)]
         self.q = torch.stack([torch.stack([synth.queries(w, s, l, device) for l in range(w.L)])
                               for s in range(w.decode_steps)])            # [steps, L, B, Hq, d]
         self.out = torch.empty_like(self.q)
         self.plan = None
+        self.decode_flags = 0
+        self.status = torch.zeros((w.L, 1), **i32)
         self.launches_compress = self.launches_decode = 0
         self.g_compress = self.g_decode = None
 
@@ -136,8 +139,10 @@ class Pipeline:
         b, w = self.b, self.w
         for s in range(w.decode_steps):
             for l in range(w.L):
-                b.decode_attn(self.q[s, l], self.layers[l], out=self.out[s, l], workspace=self.dws,
-                              status=self.plan.status)
+                # layer 0 of each step is an ordinary launch (ordered after all earlier work); the other
+                # layers share no buffer with their predecessor and may overlap it
+                b.decode_attn(self.q[s, l], self.layers[l], out=self.out[s, l], workspace=self.dws[l],
+                              status=self.status[l], flags=self.decode_flags if l > 0 else 0)
 
     def capture(self):
         self.run_compress()   # allocates the plan outside capture
@@ -180,9 +185,13 @@ def run_ours(args):
     w = synth.config(args.config)
     if args.decode_steps:
         w = w.replace(decode_steps=args.decode_steps)
+    if args.layers:
+        w = w.replace(L=args.layers)
     if distributed:
         w = w.replace(seed=w.seed + 1000 * rank)    # every rank owns an independent batch (weak scaling)
     pipe = Pipeline(w, dev)
+    # the per-layer decode calls of a step are independent (own q, out, workspace): let them overlap
+    pipe.decode_flags = 0 if args.no_overlap else binding.SC_FLAG_OVERLAP_PREV
     pipe.capture()
     cbytes, dbytes, per_layer, kept = pipe.algorithmic_bytes()
 
@@ -214,6 +223,8 @@ def run_ours(args):
     t_wall = time.perf_counter() - t_wall
     clocks = sampler.stop() if rank == 0 else None
     binding.check_status(pipe.plan.status, "timed region")
+    if int(pipe.status.abs().max().item()) != 0:
+        raise RuntimeError("sc_decode_attn reported a device-side error")
     ms_c = [e[0].elapsed_time(e[1]) for e in ev]
     ms_d = [e[1].elapsed_time(e[2]) for e in ev]
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
@@ -250,7 +261,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "n_ctx": w.n, "layers": w.L, "kv_heads": w.Hkv, "q_heads": w.Hq,
                    "head_dim": w.d, "tau": w.tau, "decode_steps": w.decode_steps, "kept_fraction": round(kept, 4),
-                   "l2": "inputs larger than L2 (every step streams all layers)", "launch": "cuda graphs",
+                   "l2": "inputs larger than L2 (every step streams all layers)", "launch": "cuda graphs" + ("" if args.no_overlap else "; the independent per-layer decode launches of a step overlap (programmatic stream serialization, no wait)"),
                    "parallelism": f"replicas x{args.gpus}" if distributed else "single gpu"},
         "decode_tokens_per_s": w.B * w.decode_steps * args.gpus / (sum_d / args.steps * 1e-3),
         "decode_bytes_per_step": dbytes,
@@ -382,8 +393,10 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="workload 0..4 (1 = Llama-3-8B, 32K context, batch 1)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps per step")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small profiling cases)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic dependent launch)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--traffic", type=float, default=None,

@@ -54,6 +54,14 @@ typedef enum { SC_BF16 = 0, SC_F32 = 1 } sc_dtype;
 #define SC_FLAG_GENERIC 1u     /* force the generic (CUDA-core, any dtype) kernels */
 #define SC_FLAG_TWO_PASS 2u    /* fused compress: count pass + write pass instead of the
                                   single pass whose tiles look back for their output offset */
+#define SC_FLAG_OVERLAP_PREV 4u /* sc_decode_attn: launch with programmatic stream serialization and
+                                  do not wait for the kernel enqueued just before on this stream.
+                                  The caller promises that that kernel and this call share no
+                                  buffer that either of them writes (q, out, workspace, status and
+                                  the cores all count).  Independent calls, e.g. the layers of an
+                                  attention-only benchmark with one workspace per layer, then run
+                                  back to back without the launch gap.  A call without the flag
+                                  orders itself after everything enqueued before it, as usual. */
 
 typedef struct {
     float tau;             /* similarity threshold of Algorithm 1; merge iff Sim > tau (strict) */
@@ -162,7 +170,7 @@ SC_API sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides
  *   core_len   [B, Hkv] int32 (device), each <= cap
  *   scale      0 means 1/sqrt(d)
  *   out        [B, Hq, d] contiguous, dtype dt; a head with core_len 0 gets zeros
- *   flags      SC_FLAG_GENERIC forces the generic kernels; 0 otherwise
+ *   flags      SC_FLAG_GENERIC forces the generic kernels; SC_FLAG_OVERLAP_PREV (see above); else 0
  *   workspace  at least sc_decode_workspace_bytes(B, Hq, Hkv, d, cap) bytes.  It holds the
  *              split partials and a few arrival counters; the counters must be zero on entry
  *              and are left zero on exit, so zero the workspace once after allocating it.

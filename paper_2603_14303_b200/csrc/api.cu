@@ -132,7 +132,7 @@ sc_status sc_decode_attn(const void* q, sc_dtype dt, int32_t B, int32_t Hq, int3
     if (workspace_bytes < sc_decode_workspace_bytes(B, Hq, Hkv, d, cap)) return SC_ERR_INVALID_ARG;
     DecodeArgs a;
     a.q = q; a.dt = dt; a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.d = d; a.core_k = core_k; a.core_v = core_v;
-    a.count = count; a.cap = cap; a.core_len = core_len; a.scale = scale; a.out = out; a.ws = workspace;
+    a.count = count; a.cap = cap; a.core_len = core_len; a.scale = scale; a.flags = flags; a.out = out; a.ws = workspace;
     a.status = status;
     cudaError_t e;
     if (!(flags & SC_FLAG_GENERIC) && decode_mma_supported(a)) e = launch_decode_mma(a, (cudaStream_t)stream);

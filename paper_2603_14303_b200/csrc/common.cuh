@@ -98,7 +98,7 @@ size_t compress_generic_ws_bytes(int32_t B, int32_t Hkv, int32_t n);
 struct DecodeArgs {
     const void* q; sc_dtype dt; int32_t B, Hq, Hkv, d;
     const void* core_k; const void* core_v; const int32_t* count; int32_t cap;
-    const int32_t* core_len; float scale; void* out; void* ws; int32_t* status;
+    const int32_t* core_len; float scale; uint32_t flags; void* out; void* ws; int32_t* status;
 };
 cudaError_t launch_decode_generic(const DecodeArgs& a, cudaStream_t st);
 size_t decode_generic_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap);

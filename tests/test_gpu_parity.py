@@ -269,3 +269,39 @@ def test_no_merge_compress_then_decode_equals_exact_attention():
         s = (Kf[0, hq // G] @ qf[0, hq]) / np.sqrt(w.d)
         want = torch.softmax(s, 0) @ Vf[0, hq // G]
         assert_close_vectors(to_f64(out[0, hq]), want.numpy(), 1e-2, f"exact attention head {hq}")
+
+
+def test_overlapped_independent_layer_launches_match_ordinary_ones():
+    """SC_FLAG_OVERLAP_PREV: layers with their own q/out/workspace launched back to back."""
+    w = synth.config(0, n=4096, L=4)
+    ids, run_id, run_lens = synth.token_ids(w)
+    plan = binding.chunk(ids.to(DEV), w.delims)
+    layers, refs = [], []
+    for l in range(w.L):
+        K, V = synth.layer_kv(w, l, run_id, run_lens)
+        refs.append(oracle_compress(ids, K, V, w.delims, w.tau))
+        layers.append(binding.compress(K.to(DEV), V.to(DEV), plan, w.tau))
+    steps = 6
+    q = torch.stack([torch.stack([synth.queries(w, s, l) for l in range(w.L)]) for s in range(steps)]).to(DEV)
+    plain, fast = torch.empty_like(q), torch.empty_like(q)
+    ws = [binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, w.n, DEV) for _ in range(w.L)]
+    st = torch.zeros((w.L, 1), dtype=torch.int32, device=DEV)
+    for s in range(steps):
+        for l in range(w.L):
+            binding.decode_attn(q[s, l], layers[l], out=plain[s, l], workspace=ws[l], status=st[l])
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for s in range(steps):
+            for l in range(w.L):
+                binding.decode_attn(q[s, l], layers[l], out=fast[s, l], workspace=ws[l], status=st[l],
+                                    flags=binding.SC_FLAG_OVERLAP_PREV if l > 0 else 0)
+        torch.cuda.synchronize()
+        assert torch.equal(plain, fast)
+        fast.zero_()
+    assert int(st.abs().max()) == 0
+    for l in range(w.L):
+        want = oracle.attn(synth.to_numpy_bits(q[2, l].cpu()), refs[l]["core_k"], refs[l]["core_v"], refs[l]["count"],
+                           refs[l]["core_len"])
+        assert_close_vectors(to_f64(plain[2, l]), want, 1e-2, f"layer {l}")
+    for x in ws:
+        assert int(x.view(torch.int32)[:64].abs().max()) == 0, "arrival counters are left at zero"
