@@ -97,6 +97,7 @@ sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dt
     if ((kv_strides.b * esz) % 16 || (kv_strides.h * esz) % 16 || (kv_strides.n * esz) % 16) return SC_ERR_INVALID_ARG;
     if (kv_strides.n < d) return SC_ERR_INVALID_ARG;
     if ((int64_t)B * n > 0x7fffffff - 1) return SC_ERR_INVALID_ARG;
+    if (n_tile_cap < 1 || n_tile_cap > tile_cap_for(n)) return SC_ERR_INVALID_ARG;
     if (workspace_bytes < sc_compress_workspace_bytes(B, Hkv, n)) return SC_ERR_INVALID_ARG;
     CompressArgs a;
     a.K = K; a.V = V; a.st = kv_strides; a.dt = dt; a.B = B; a.Hkv = Hkv; a.n = n; a.d = d;
