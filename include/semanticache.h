@@ -182,6 +182,39 @@ SC_API sc_status sc_decode_attn(const void* q, sc_dtype dt, int32_t B, int32_t H
                          const int32_t* core_len, float scale, uint32_t flags, void* out,
                          void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
 
+/*
+ * sc_decode_attn for callers that cannot allocate device memory.  (A convenience of this
+ * library; the paper has no counterpart.)
+ *
+ * Who needs it: a server that handed all free HBM to its KV-cache pool at start-up, so that any
+ * later cudaMalloc fails; a plug-in whose host runtime forbids allocation inside its step
+ * callback; a loop that cannot tolerate the device-wide synchronisation an allocation may
+ * bring.  Such callers have nowhere to get the workspace sc_decode_attn asks for.
+ *
+ * Same arguments, results and error codes as sc_decode_attn, minus the workspace: the split
+ * partials and arrival counters live in a fixed array of SC_STATIC_SCRATCH_BYTES that is part of
+ * the library image.  Every GPU on which the library is loaded holds that array until the
+ * process exits, whether or not this entry point is ever called.  The call itself performs no
+ * cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ *   - Shapes whose workspace (sc_decode_workspace_bytes) exceeds SC_STATIC_SCRATCH_BYTES are
+ *     rejected with SC_ERR_CAPACITY before anything is enqueued; use sc_decode_attn for those.
+ *     For d = 128 the limit admits B * Hq * min(64, ceil(cap / 512)) up to about 16000, e.g.
+ *     16 sequences of 32 query heads with 8K rows of capacity each.
+ *   - The first call on each GPU looks up the array's device address (a short host-side set-up,
+ *     done with that GPU current).  Make that first call outside any stream capture.
+ *   - All calls on a GPU share the one array, which keeps the previous call's contents; each
+ *     call clears the part it uses, in stream order, before its kernel runs.  Two calls that may
+ *     execute concurrently on the same GPU (different streams, or SC_FLAG_OVERLAP_PREV, which is
+ *     refused here with SC_ERR_INVALID_ARG) would race on it: keep them on one stream.
+ */
+#define SC_STATIC_SCRATCH_BYTES (8u << 20)
+
+SC_API sc_status sc_decode_attn_static(const void* q, sc_dtype dt, int32_t B, int32_t Hq, int32_t Hkv, int32_t d,
+                                const void* core_k, const void* core_v, const int32_t* count, int32_t cap,
+                                const int32_t* core_len, float scale, uint32_t flags, void* out,
+                                int32_t* status, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

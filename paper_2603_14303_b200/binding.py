@@ -23,7 +23,9 @@ _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CA
                  "SC_ERR_TIMEOUT"]
 
 EXPORTS = ["sc_version", "sc_launch_counter", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
-           "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn"]
+           "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn",
+           "sc_decode_attn_static"]
+SC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class ScError(RuntimeError):
@@ -70,6 +72,9 @@ def lib() -> ctypes.CDLL:
         L.sc_decode_attn.restype = _i32
         L.sc_decode_attn.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, ctypes.c_float,
                                      ctypes.c_uint32, _vp, _vp, _sz, _vp, _vp]
+        L.sc_decode_attn_static.restype = _i32
+        L.sc_decode_attn_static.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp,
+                                            ctypes.c_float, ctypes.c_uint32, _vp, _vp, _vp]
         _lib = L
     return _lib
 
@@ -158,6 +163,23 @@ def sc_decode_attn(q, core_k, core_v, count, core_len, out, workspace, scale=0.0
                                 _ptr(core_len), float(scale), int(flags), _ptr(out), _ptr(workspace),
                                 workspace.numel() * workspace.element_size(), _ptr(status), _stream(q))
     _check("sc_decode_attn", code)
+
+
+def sc_decode_attn_static(q, core_k, core_v, count, core_len, out, scale=0.0, status=None, flags=0):
+    """Raw sc_decode_attn_static: one decode step with the scratch inside the library image.
+
+    For callers that cannot allocate device memory (see the header); nothing is allocated here
+    either -- every buffer, ``out`` included, is the caller's.  Calls on one GPU share the
+    library's scratch array, so keep them on one stream.
+    """
+    _need_cuda(q, core_k, core_v, count, core_len, out)
+    B, Hq, d = q.shape
+    _, Hkv, cap, _ = core_k.shape
+    assert q.is_contiguous() and out.is_contiguous() and core_k.is_contiguous() and core_v.is_contiguous()
+    code = lib().sc_decode_attn_static(_ptr(q), _dt(q), B, Hq, Hkv, d, _ptr(core_k), _ptr(core_v), _ptr(count),
+                                       cap, _ptr(core_len), float(scale), int(flags), _ptr(out), _ptr(status),
+                                       _stream(q))
+    _check("sc_decode_attn_static", code)
 
 
 # ------------------------------------------------------------------------- convenience wrappers
