@@ -173,13 +173,13 @@ class Pipeline:
 
 
 def run_ours(args):
+    from paper_2603_14303_b200 import dist as scdist
     distributed = args.gpus > 1
-    rank, local = int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0))
-    if distributed:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    rank, local, _ = scdist.env_rank()
     dev = torch.device(f"cuda:{local}")
     torch.cuda.set_device(dev)
+    if distributed:
+        scdist.init("nccl", dev)
     from paper_2603_14303_b200 import binding, build
     build.build()
     w = synth.config(args.config)
@@ -188,7 +188,7 @@ def run_ours(args):
     if args.layers:
         w = w.replace(L=args.layers)
     if distributed:
-        w = w.replace(seed=w.seed + 1000 * rank)    # every rank owns an independent batch (weak scaling)
+        w = scdist.rank_workload(w, rank)           # every rank owns an independent batch (weak scaling)
     pipe = Pipeline(w, dev)
     # the per-layer decode calls of a step are independent (own q, out, workspace): let them overlap
     pipe.decode_flags = 0 if args.no_overlap else binding.SC_FLAG_OVERLAP_PREV
@@ -196,9 +196,7 @@ def run_ours(args):
     cbytes, dbytes, per_layer, kept = pipe.algorithmic_bytes()
 
     def barrier():
-        if distributed:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
+        scdist.barrier(dev)
 
     def one_step():
         pipe.g_compress.replay()
@@ -228,21 +226,14 @@ def run_ours(args):
     ms_c = [e[0].elapsed_time(e[1]) for e in ev]
     ms_d = [e[1].elapsed_time(e[2]) for e in ev]
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
-    if distributed:
-        t = torch.tensor([total_ms, sum(ms_c), sum(ms_d)], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, sum_c, sum_d = t.tolist()
-    else:
-        sum_c, sum_d = sum(ms_c), sum(ms_d)
-    tokens = w.B * w.decode_steps * args.steps * args.gpus
-    value = tokens / (total_ms * 1e-3)
+    total_ms, sum_c, sum_d = scdist.max_over_ranks([total_ms, sum(ms_c), sum(ms_d)], dev)
+    value = scdist.whole_job_rate(w.B * w.decode_steps * args.steps, args.gpus, total_ms)
 
     # end to end through the public API with HOST buffers (copies inside the timed region)
     e2e = run_e2e(pipe, args, barrier) if not args.no_e2e else None
     if distributed and e2e is not None:
-        t = torch.tensor([e2e["_ms"]], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e["value"] = w.B * w.decode_steps * e2e["_steps"] * args.gpus / (t.item() * 1e-3)
+        e2e["value"] = scdist.whole_job_rate(w.B * w.decode_steps * e2e["_steps"], args.gpus,
+                                             scdist.max_over_ranks([e2e["_ms"]], dev)[0])
     if e2e is not None:
         e2e = {k: v for k, v in e2e.items() if not k.startswith("_")}
 
@@ -388,7 +379,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=1, help="workload 0..4 (1 = Llama-3-8B, 32K context, batch 1)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
