@@ -128,7 +128,7 @@ SC_API sc_status sc_chunk(const int32_t* token_ids, int32_t B, int32_t n,
  * Compress one layer (Sec. 2.3-2.4).  For every (sequence b, KV head h, segment) independently:
  * Greedy Seed-Based Clustering (Algorithm 1) on the cosine similarity of the keys (Eq. 2; a
  * zero-norm key has similarity 0 to everything), then each cluster S_t is mean-pooled into one
- * core k_hat = mean(k_i), v_hat = mean(v_i) (Eq. 3; fp32 sums in token order, rounded once to
+ * core k_hat = mean(k_i), v_hat = mean(v_i) (Eq. 3; fp32 accumulation, rounded once to
  * the storage dtype) with count = |S_t|.  Cores are written compactly in position order of
  * their seeds; a delimiter is a core of count 1 carrying its K/V bits unchanged.
  *
@@ -143,7 +143,10 @@ SC_API sc_status sc_chunk(const int32_t* token_ids, int32_t B, int32_t n,
  *               cap = n always suffices.
  *   assign      optional out [B, Hkv, n] int32: for each token the position (within its
  *               sequence) of the seed of its cluster; NULL to skip
- *   workspace   at least sc_compress_workspace_bytes(B, Hkv, n) bytes
+ *   workspace   at least sc_compress_workspace_bytes(B, Hkv, n) bytes.  It holds per-tile status
+ *               words and two counters that must be zero on entry and are left zero on exit, so
+ *               zero the workspace once after allocating it (and again after a call that
+ *               reported SC_ERR_TIMEOUT).  Calls that share a workspace must not overlap.
  */
 SC_API size_t sc_compress_workspace_bytes(int32_t B, int32_t Hkv, int32_t n);
 

@@ -233,7 +233,8 @@ def chunk(token_ids: torch.Tensor, delim_ids, max_chunk_len: int = SC_MAX_CHUNK_
 
 
 def compress_workspace(B, Hkv, n, device) -> torch.Tensor:
-    return torch.empty(lib().sc_compress_workspace_bytes(B, Hkv, n), dtype=torch.uint8, device=device)
+    """Zero-initialised workspace for sc_compress (its status words and counters must start at zero)."""
+    return torch.zeros(lib().sc_compress_workspace_bytes(B, Hkv, n), dtype=torch.uint8, device=device)
 
 
 def compress(K, V, plan: ChunkPlan, tau: float, cap: int | None = None, want_assign: bool = False,

@@ -19,6 +19,9 @@ namespace sc { void note_launches(int n) { g_launches.fetch_add((uint64_t)n, std
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline int tile_cap_for(int32_t n) { return 2 * div_up(n, SC_TILE_ROWS) + 1; }
+static inline size_t fused_region_bytes(int32_t B, int32_t Hkv, int32_t n) {
+    return (compress_fused_ws_bytes(B, Hkv, n) + 255) / 256 * 256;
+}
 
 extern "C" {
 
@@ -70,8 +73,8 @@ sc_status sc_chunk(const int32_t* token_ids, int32_t B, int32_t n, const int32_t
 
 size_t sc_compress_workspace_bytes(int32_t B, int32_t Hkv, int32_t n) {
     if (B <= 0 || Hkv <= 0 || n <= 0) return 256;
-    size_t a = compress_generic_ws_bytes(B, Hkv, n), b = compress_fused_ws_bytes(B, Hkv, n);
-    return a > b ? a : b;
+    // [status words and counters of the fused kernel (zero between calls)] [scratch of the generic kernels]
+    return fused_region_bytes(B, Hkv, n) + compress_generic_ws_bytes(B, Hkv, n);
 }
 
 sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dtype dt, int32_t B, int32_t Hkv,
@@ -107,8 +110,12 @@ sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dt
     a.core_k = core_k; a.core_v = core_v; a.count = count; a.cap = cap; a.core_len = core_len;
     a.assign = assign; a.ws = workspace; a.status = status;
     cudaError_t e;
-    if (!(a.flags & SC_FLAG_GENERIC) && compress_fused_supported(a)) e = launch_compress_fused(a, st);
-    else e = launch_compress_generic(a, st);
+    if (!(a.flags & SC_FLAG_GENERIC) && compress_fused_supported(a)) {
+        e = launch_compress_fused(a, st);
+    } else {
+        a.ws = (char*)workspace + fused_region_bytes(B, Hkv, n);   // never touches the fused kernel's words
+        e = launch_compress_generic(a, st);
+    }
     return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
 

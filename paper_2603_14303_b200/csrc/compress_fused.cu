@@ -1,22 +1,29 @@
-// Fused bf16 compress kernel (d = 128, token stride of 256 bytes or more), sm_100a.
+// Fused bf16 compress kernel (d = 128), sm_100a: Eq. 2 + Algorithm 1 + Eq. 3 in one pass over K, V.
 //
-// One block per (sequence, KV head, work tile).  A tile is a run of whole segments of at most
-// SC_TILE_ROWS tokens (K and V staged in shared memory), or one longer segment alone (K staged,
-// V streamed from global memory).  Steps inside a block:
-//   1. cp.async the tile's K (and V) rows into shared memory, 16-byte chunks XOR-swizzled;
-//   2. Gram blocks K.K^T of 32x32 rows on the tensor cores (mma.m16n8k16, bf16 products are exact
-//      in fp32) for exactly the block pairs a segment spans; the diagonal gives the norms, then
-//      Sim > tau (Eq. 2) is decided as G_ij > tau*|k_i|*|k_j| and packed into one adjacency bit
-//      row per token (later tokens of the same segment only);
-//   3. Algorithm 1 per segment on those bit rows: lowest unassigned token becomes a seed and
+// Persistent blocks (as many as fit on the GPU at once) draw work tiles from a global ticket
+// counter.  A tile is a run of whole segments of at most SC_TILE_ROWS tokens of one (sequence, KV
+// head) -- K and V both staged in shared memory -- or one longer segment alone (K staged, then V
+// in a second pass over the same buffer).  Per tile:
+//   1. the rows are brought in with one bulk asynchronous copy per row (cp.async.bulk, completion
+//      on an mbarrier) into rows of 272 bytes: the 16-byte pad makes ldmatrix conflict free
+//      without address swizzling.  While a tile is processed the block already holds its next
+//      ticket and has asked L2 to prefetch that tile, so DRAM stays busy during the compute phases;
+//   2. Gram blocks K.K^T of 32x32 rows on the tensor cores (mma.m16n8k16; bf16 products are exact
+//      in fp32) for exactly the block pairs a segment spans; the diagonal gives the norms and
+//      Sim > tau (Eq. 2) is decided as G_ij > tau*|k_i|*|k_j|, packed into adjacency bit rows
+//      (later tokens of the same segment only, stored as an upper triangle of 32-bit words);
+//   3. Algorithm 1 per segment on those bit rows: the lowest unassigned token becomes a seed and
 //      takes every unassigned adjacent token -- a few word operations per seed, one warp per
-//      segment with one lane per 32-token word;
-//   4. the tile's cluster count feeds a prefix sum over the tiles of the (sequence, head): either
-//      a separate count pass (two-pass mode) or a decoupled look-back over per-tile status words
-//      (single pass; tiles are taken in ticket order so every predecessor is already running,
-//      and the wait is bounded);
-//   5. Eq. 3: one warp per cluster sums the member rows of K and V in token order in fp32,
-//      scales by 1/|S|, rounds once to bf16 and writes the core row and its count compactly.
+//      segment with one lane per 32-token word; the seed's row then holds its member mask;
+//   4. the tile's cluster count enters a prefix sum over the tiles of its (sequence, head): a
+//      decoupled look-back over per-tile status words (tickets are handed out in order, so every
+//      predecessor is held by a running block and the bounded wait cannot starve), or, in
+//      two-pass mode, a count pass followed by a write pass;
+//   5. Eq. 3 as a product on the tensor cores: member masks expanded to a 0/1 bf16 matrix times
+//      the staged K (V) rows, fp32 accumulation, one multiply by 1/|S|, one rounding to bf16; the
+//      cores are compacted in place in shared memory and leave with 16-byte coalesced stores.
+// The last block to finish zeroes the status words and counters, so a workspace that was zero
+// before the call is zero again after it.
 #include "common.cuh"
 
 namespace sc {
@@ -26,34 +33,90 @@ namespace cf {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kD = 128;
-constexpr int kRowBytes = 256;
+constexpr int kRowBytes = 256;                    // one K or V row in global memory
+constexpr int kPitch = 272;                       // its pitch in shared memory (16-byte pad)
 constexpr int kMaxRows = SC_MAX_CHUNK_LEN;        // 256: a long tile
 constexpr int kShortRows = SC_TILE_ROWS;          // 128
-constexpr int kNW = 8;                            // 32-bit words per adjacency row
-constexpr int kKvBytes = kMaxRows * kRowBytes;    // 65536: short = K 32K | V 32K, long = K 64K
+constexpr int kNW = 8;                            // 32-bit words per (full) adjacency row
+constexpr int kKvBytes = kMaxRows * kPitch;       // 69632: short = K | V halves, long = one tensor
+constexpr int kVOff = kShortRows * kPitch;        // 34816
 constexpr int kAdjOff = kKvBytes;
-constexpr int kAdjBytes = kMaxRows * kNW * 4;     // 8192
-constexpr int kNormOff = kAdjOff + kAdjBytes;     // float[256]
-constexpr int kSendOff = kNormOff + kMaxRows * 4; // uint16[256]: segment end per row
-constexpr int kSegsOff = kSendOff + kMaxRows * 2; // int16[130]: segment starts in the tile
-constexpr int kItemOff = kSegsOff + 272;          // uint8[48]: (row block << 4 | col block) pairs
-constexpr int kMiscOff = kItemOff + 48;           // uint32 seedmask[8], int misc[8]
-constexpr int kSmemBytes = kMiscOff + 64;
+constexpr int kAdjWords = 32 * (8 + 7 + 6 + 5 + 4 + 3 + 2 + 1);   // rows of block k keep words k..7
+constexpr int kNormOff = kAdjOff + kAdjWords * 4; // float[256]; later uint16 seed row per cluster
+constexpr int kSendOff = kNormOff + kMaxRows * 4; // uint16[256]: end of the segment a row is in
+constexpr int kSegsOff = kSendOff + kMaxRows * 2; // 2 x int16[132]: segment starts (this tile, next tile)
+constexpr int kSegsStride = 132;
+constexpr int kMiscOff = kSegsOff + 2 * kSegsStride * 2;   // uint32 seedmask[8]; int geo[2][8]; int misc[4]
+constexpr int kBarOff = kMiscOff + 32 + 64 + 16;  // two mbarriers (rows of K; rows of V)
+constexpr int kSmemBytes = kBarOff + 16;
+static_assert(kBarOff % 8 == 0, "mbarrier alignment");
+static_assert(kSmemBytes <= 76800, "three blocks per SM need <= 75 KB each");
 
 enum Mode { kCountOnly = 0, kWriteWithCounts = 1, kLookBack = 2 };
+enum Geo { gB = 0, gH = 1, gT = 2, gNseg = 3, gRow0 = 4, gR = 5, gLast = 6 };
+
+// Per-phase cycle totals for a debugging harness; compiled out of the library.
+#ifdef SC_PHASE_TIMING
+__device__ unsigned long long g_phase_cycles[16];
+#define CF_T(i)                                                                 \
+    do {                                                                        \
+        if (threadIdx.x == 0) {                                                 \
+            const long long now_ = clock64();                                   \
+            atomicAdd(&g_phase_cycles[i], (unsigned long long)(now_ - t_prev)); \
+            t_prev = now_;                                                      \
+        }                                                                       \
+    } while (0)
+#else
+#define CF_T(i)
+#endif
 
 constexpr uint32_t kFlagAggregate = 1u << 30, kFlagPrefix = 2u << 30, kValueMask = (1u << 30) - 1;
-constexpr int kSpinLimit = 1 << 22;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every wait gives up after 2 s
+constexpr int kCtlWords = 64;                                // ticket, done counter, padding
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+    return t;
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0u;
+}
+// Bounded wait for a phase of an mbarrier; false if it gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > kWaitLimitNs) return false;
+    }
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -62,7 +125,6 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ uint32_t swz(int row, int chunk) { return row * kRowBytes + ((chunk ^ (row & 7)) << 4); }
 __device__ __forceinline__ uint32_t bits_between(int lo, int hi, int word) {   // bits [lo, hi) that fall in `word`
     lo = max(lo, word * 32); hi = min(hi, word * 32 + 32);
     if (hi <= lo) return 0u;
@@ -73,29 +135,36 @@ __device__ __forceinline__ uint32_t ld_volatile(const uint32_t* p) {
     asm volatile("ld.volatile.global.u32 %0, [%1];\n" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
+// Word offset of adjacency word (row i, word i>>5) in the triangular store; word w >= i>>5 of the
+// same row follows at + (w - (i>>5)).
+__device__ __forceinline__ int adj_row(int i) {
+    const int k = i >> 5;
+    return 256 * k - 16 * k * (k - 1) + (i & 31) * (kNW - k);
+}
+// Two mask bits -> two bf16 (0.0 or 1.0) packed as an mma operand register.
+__device__ __forceinline__ uint32_t expand2(uint32_t two_bits) {
+    return ((two_bits * 0x8001u) & 0x00010001u) * 0x3F80u;
+}
 
-// 32x32 block of K.K^T: rows of block rb against rows of block cb.
+// 32x32 block of K.K^T: rows of block rb against rows of block cb (rows staged at pitch kPitch).
 __device__ __forceinline__ void gram_block(uint32_t kbase, int rb, int cb, int lane, float (&acc)[2][4][4]) {
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = acc[mt][nt][2] = acc[mt][nt][3] = 0.f;
     const int j = lane >> 3, r8 = lane & 7;
-    const int a_row = r8 + ((j & 1) << 3), a_c = j >> 1;      // (r0-7,c) (r8-15,c) (r0-7,c+1) (r8-15,c+1)
-    const int b_row = r8 + ((j >> 1) << 3), b_c = j & 1;      // (r0-7,c) (r0-7,c+1) (r8-15,c) (r8-15,c+1)
+    // A: matrices (r0-7,c) (r8-15,c) (r0-7,c+1) (r8-15,c+1);  B: (r0-7,c) (r0-7,c+1) (r8-15,c) (r8-15,c+1)
+    const uint32_t a_addr = kbase + (rb * 32 + r8 + ((j & 1) << 3)) * kPitch + ((j >> 1) << 4);
+    const uint32_t b_addr = kbase + (cb * 32 + r8 + ((j >> 1) << 3)) * kPitch + ((j & 1) << 4);
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
         uint32_t a[2][4], bq[2][4];
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-            const int row = rb * 32 + mt * 16 + a_row;
-            ldmatrix_x4(kbase + swz(row, 2 * ks + a_c), a[mt][0], a[mt][1], a[mt][2], a[mt][3]);
-        }
+        for (int mt = 0; mt < 2; ++mt)
+            ldmatrix_x4(a_addr + mt * 16 * kPitch + ks * 32, a[mt][0], a[mt][1], a[mt][2], a[mt][3]);
 #pragma unroll
-        for (int p = 0; p < 2; ++p) {
-            const int row = cb * 32 + p * 16 + b_row;
-            ldmatrix_x4(kbase + swz(row, 2 * ks + b_c), bq[p][0], bq[p][1], bq[p][2], bq[p][3]);
-        }
+        for (int p = 0; p < 2; ++p)
+            ldmatrix_x4(b_addr + p * 16 * kPitch + ks * 32, bq[p][0], bq[p][1], bq[p][2], bq[p][3]);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
@@ -104,16 +173,32 @@ __device__ __forceinline__ void gram_block(uint32_t kbase, int rb, int cb, int l
     }
 }
 
-// Turns a Gram block into adjacency words: bit j of adj[i][cb] = Sim(i, 32cb + j) > tau, limited
+// Diagonal of a diagonal Gram block = squared norms of its 32 rows.
+__device__ __forceinline__ void store_norms(const float (&acc)[2][4][4], int rb, int lane, float* norm) {
+    const int g = lane >> 2, tig = lane & 3;
+    if ((g >> 1) == tig) {
+        const int e = g & 1;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+                norm[rb * 32 + mt * 16 + hh * 8 + g] =
+                    sqrtf(e ? acc[mt][2 * mt + hh][hh * 2 + 1] : acc[mt][2 * mt + hh][hh * 2]);
+    }
+}
+
+// Turns a Gram block into adjacency words: bit j of word (i, cb) = Sim(i, 32cb + j) > tau, limited
 // to later tokens of i's own segment.
+template <bool kNegTau>
 __device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int rb, int cb, int lane, float tau,
                                                 const float* norm, const uint16_t* send, uint32_t* adj) {
     const int g = lane >> 2, tig = lane & 3;
     float tn[4][2];
 #pragma unroll
     for (int nt = 0; nt < 4; ++nt) {
-        tn[nt][0] = tau * norm[cb * 32 + nt * 8 + 2 * tig];
-        tn[nt][1] = tau * norm[cb * 32 + nt * 8 + 2 * tig + 1];
+        const float2 nn = *reinterpret_cast<const float2*>(norm + cb * 32 + nt * 8 + 2 * tig);
+        tn[nt][0] = tau * nn.x;
+        tn[nt][1] = tau * nn.y;
     }
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
@@ -121,326 +206,518 @@ __device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int
         for (int hh = 0; hh < 2; ++hh) {
             const int i = rb * 32 + mt * 16 + hh * 8 + g;
             const float ni = norm[i];
-            uint32_t w = 0;
+            uint32_t w = 0;   // bit nt*8 + e, moved to nt*8 + 2*tig + e afterwards
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const float thr = ni * tn[nt][e];
                     bool hit = acc[mt][nt][hh * 2 + e] > thr;
-                    if (tau < 0.f) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
-                    w |= (hit ? 1u : 0u) << (nt * 8 + 2 * tig + e);
+                    if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
+                    if (hit) w |= 1u << (nt * 8 + e);
                 }
+            w <<= 2 * tig;
             w |= __shfl_xor_sync(kFull, w, 1);
             w |= __shfl_xor_sync(kFull, w, 2);
-            if (tig == 0) adj[i * kNW + cb] = w & bits_between(i + 1, (int)send[i], cb);
+            if (tig == 0) adj[adj_row(i) + (cb - rb)] = w & bits_between(i + 1, (int)send[i], cb);
         }
 }
 
+// Off-diagonal block pairs (row block << 4 | column block), nearest diagonals first.
+__constant__ uint8_t kOffDiag[28] = {0x01, 0x12, 0x23, 0x34, 0x45, 0x56, 0x67, 0x02, 0x13, 0x24, 0x35, 0x46, 0x57, 0x03,
+                                     0x14, 0x25, 0x36, 0x47, 0x04, 0x15, 0x26, 0x37, 0x05, 0x16, 0x27, 0x06, 0x17, 0x07};
+
+struct Params {
+    const __nv_bfloat16* K; const __nv_bfloat16* V; sc_strides st;
+    int B, Hkv, n;
+    const int32_t* seg_off; const int32_t* tile_seg; const int32_t* seq_tile_cnt; int n_tile_cap;
+    float tau;
+    __nv_bfloat16* core_k; __nv_bfloat16* core_v; int32_t* count; int cap; int32_t* core_len;
+    int32_t* assign;
+    int32_t* ctl;            // [0] ticket counter, [1] blocks finished
+    uint32_t* tile_state;    // [B*Hkv][n_tile_cap]
+    int32_t* status;
+};
+
+// Warp 0 draws the next ticket, turns it into a tile (sequence, head, tile index, rows), copies the
+// tile's segment starts into shared memory and asks L2 to prefetch the tile's K and V rows.
+// Tickets walk the tiles of head 0 of sequence 0 in order, then head 1, ...; a block's tickets only
+// grow, so the sequence it last decoded (dec_b, with dec_pref tickets before it) is where the search
+// resumes.  geo[gT] = -1 when no work is left.
 template <int kMode>
-__global__ void __launch_bounds__(kThreads, 3)
-compress_fused_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V, sc_strides st,
-                      int Hkv, int n, const int32_t* __restrict__ seg_off, const int32_t* __restrict__ tile_seg,
-                      const int32_t* __restrict__ seq_tile_cnt, int n_tile_cap, float tau,
-                      __nv_bfloat16* __restrict__ core_k, __nv_bfloat16* __restrict__ core_v,
-                      int32_t* __restrict__ count, int cap, int32_t* __restrict__ core_len,
-                      int32_t* __restrict__ assign, uint32_t* __restrict__ tile_state, int32_t* __restrict__ tickets,
-                      int32_t* status) {
+__device__ __forceinline__ void fetch_tile(const Params& p, int lane, int& dec_b, int& dec_pref, int* geo,
+                                           int16_t* segs) {
+    int w = 0;
+    if (lane == 0) w = atomicAdd(&p.ctl[0], 1);
+    w = __shfl_sync(kFull, w, 0);
+    int nt = 0;
+    while (dec_b < p.B) {
+        nt = min(p.seq_tile_cnt[dec_b], p.n_tile_cap);
+        const int span = p.Hkv * nt;
+        if (w < dec_pref + span) break;
+        dec_pref += span;
+        ++dec_b;
+    }
+    if (dec_b >= p.B) {
+        if (lane == 0) geo[gT] = -1;
+        return;
+    }
+    const int r = w - dec_pref, h = r / nt, t = r - h * nt, b = dec_b;
+    const int32_t* ts = p.tile_seg + (size_t)b * (p.n_tile_cap + 1);
+    const int s_begin = ts[t], s_end = ts[t + 1];
+    const int nseg = max(min(s_end - s_begin, kShortRows), 1);
+    const int g_row0 = p.seg_off[s_begin];
+    for (int i = lane; i <= nseg; i += 32) segs[i] = (int16_t)min(p.seg_off[s_begin + i] - g_row0, kMaxRows);
+    const int R = min(p.seg_off[s_begin + nseg] - g_row0, kMaxRows);
+    const int row0 = g_row0 - b * p.n;
+    if (lane == 0) {
+        geo[gB] = b; geo[gH] = h; geo[gT] = t; geo[gNseg] = nseg; geo[gRow0] = row0; geo[gR] = R;
+        geo[gLast] = (t == nt - 1);
+    }
+    // L2 prefetch: one request per tensor when rows are contiguous, else one per row
+    const int64_t off = b * p.st.b + h * p.st.h + (int64_t)row0 * p.st.n;
+    if (p.st.n == kD) {
+        if (lane == 0) l2_prefetch(p.K + off, (uint32_t)R * kRowBytes);
+        if (lane == 1 && kMode != kCountOnly) l2_prefetch(p.V + off, (uint32_t)R * kRowBytes);
+    } else {
+        for (int i = lane; i < R; i += 32) {
+            l2_prefetch(p.K + off + (int64_t)i * p.st.n, kRowBytes);
+            if (kMode != kCountOnly) l2_prefetch(p.V + off + (int64_t)i * p.st.n, kRowBytes);
+        }
+    }
+}
+
+// Eq. 3 on the tensor cores for one staged tensor (K or V rows at `area`, pitch kPitch).
+// Cluster c (in seed order) has its member mask in the adjacency row of its seed seedrow[c].  A
+// warp owns one tile of 16 clusters (mt_in_round of a round of mts_per_round tiles) and 64 of the
+// 128 columns (col_off bytes): acc[16 x 64] = mask[16 x rows] . rows[rows x 64].  The scaled,
+// rounded cores overwrite rows [0, P) of the same area: cluster c only reads rows >= its seed
+// >= c, rounds go up in c, and inside a round every warp has finished reading before any writes.
+__device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_ptr, int col_off, int mt_in_round,
+                                             int mts_per_round, int P, const uint16_t* seedrow, const uint16_t* send,
+                                             const uint32_t* adj, int lane, bool write_counts) {
+    const int g = lane >> 2, tig = lane & 3;
+    const uint32_t b_lane = area + ((lane & 7) + ((lane >> 3) & 1) * 8) * kPitch + col_off + (lane >> 4) * 16;
+    for (int c0 = 0; c0 < P; c0 += 16 * mts_per_round) {
+        const int cbase = c0 + 16 * mt_in_round;
+        const bool active = cbase < P;
+        float acc[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+        int cnt0 = 0, cnt1 = 0;
+        if (active) {
+            const int c_lo = cbase + g, c_hi = cbase + g + 8;
+            const int i0 = c_lo < P ? (int)seedrow[c_lo] : -1, i1 = c_hi < P ? (int)seedrow[c_hi] : -1;
+            const int lo0 = i0 >> 5, hi0 = i0 >= 0 ? ((int)send[i0] - 1) >> 5 : -2;   // word range of the masks
+            const int lo1 = i1 >> 5, hi1 = i1 >= 0 ? ((int)send[i1] - 1) >> 5 : -2;
+            const uint32_t* r0 = adj + (i0 >= 0 ? adj_row(i0) - lo0 : 0);
+            const uint32_t* r1 = adj + (i1 >= 0 ? adj_row(i1) - lo1 : 0);
+            const int w_first = (int)seedrow[cbase] >> 5;
+            const int w_last = ((int)send[seedrow[min(cbase + 15, P - 1)]] - 1) >> 5;
+            for (int w = w_first; w <= w_last; ++w) {
+                const uint32_t m0w = (w >= lo0 && w <= hi0) ? r0[w] : 0u;
+                const uint32_t m1w = (w >= lo1 && w <= hi1) ? r1[w] : 0u;
+                cnt0 += __popc(m0w);
+                cnt1 += __popc(m1w);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const uint32_t m0 = (m0w >> (16 * hh)) & 0xffffu, m1 = (m1w >> (16 * hh)) & 0xffffu;
+                    if (!__any_sync(kFull, (m0 | m1) != 0u)) continue;
+                    const uint32_t a0 = expand2((m0 >> (2 * tig)) & 3u), a2 = expand2((m0 >> (2 * tig + 8)) & 3u);
+                    const uint32_t a1 = expand2((m1 >> (2 * tig)) & 3u), a3 = expand2((m1 >> (2 * tig + 8)) & 3u);
+                    const uint32_t b_addr = b_lane + (w * 32 + hh * 16) * kPitch;
+#pragma unroll
+                    for (int np = 0; np < 4; ++np) {
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4_trans(b_addr + np * 32, b0, b1, b2, b3);
+                        mma_bf16(acc[2 * np], a0, a1, a2, a3, b0, b1);
+                        mma_bf16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+                    }
+                }
+            }
+        }
+        __syncthreads();   // every warp has read what it needs of rows [c0, ...)
+        if (active) {
+            const float inv0 = 1.0f / (float)max(cnt0, 1), inv1 = 1.0f / (float)max(cnt1, 1);
+            unsigned char* o_lo = area_ptr + (cbase + g) * kPitch + col_off + tig * 4;
+            unsigned char* o_hi = o_lo + 8 * kPitch;
+            const bool ok_lo = cbase + g < P, ok_hi = cbase + g + 8 < P;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(acc[nt][0] * inv0, acc[nt][1] * inv0);
+                __nv_bfloat162 hi = __floats2bfloat162_rn(acc[nt][2] * inv1, acc[nt][3] * inv1);
+                if (ok_lo) *reinterpret_cast<__nv_bfloat162*>(o_lo + nt * 16) = lo;
+                if (ok_hi) *reinterpret_cast<__nv_bfloat162*>(o_hi + nt * 16) = hi;
+            }
+            if (write_counts && tig == 0) {   // the row's 16-byte pad carries its member count
+                if (ok_lo) *reinterpret_cast<int*>(area_ptr + (cbase + g) * kPitch + kRowBytes) = cnt0;
+                if (ok_hi) *reinterpret_cast<int*>(area_ptr + (cbase + g + 8) * kPitch + kRowBytes) = cnt1;
+            }
+        }
+    }
+}
+
+template <int kMode>
+__global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Params p) {
     extern __shared__ __align__(128) unsigned char smem[];
     uint32_t* adj = reinterpret_cast<uint32_t*>(smem + kAdjOff);
     float* norm = reinterpret_cast<float*>(smem + kNormOff);
+    uint16_t* seedrow = reinterpret_cast<uint16_t*>(smem + kNormOff);   // reuses the norms once they are spent
     uint16_t* send = reinterpret_cast<uint16_t*>(smem + kSendOff);
-    int16_t* segs = reinterpret_cast<int16_t*>(smem + kSegsOff);
-    uint8_t* items = reinterpret_cast<uint8_t*>(smem + kItemOff);
+    int16_t* segs_buf = reinterpret_cast<int16_t*>(smem + kSegsOff);
     uint32_t* seedmask = reinterpret_cast<uint32_t*>(smem + kMiscOff);
-    int* misc = reinterpret_cast<int*>(smem + kMiscOff + 32);   // [0] tile index, [1] n items, [2] base offset
+    int* geo_buf = reinterpret_cast<int*>(smem + kMiscOff + 32);        // [2][8]
+    int* misc = reinterpret_cast<int*>(smem + kMiscOff + 96);           // [0] output offset of the tile, [1] last block
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_k = sbase + kBarOff, bar_v = sbase + kBarOff + 8;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int h = blockIdx.y, b = blockIdx.z;
-    const int bh = b * Hkv + h;
-    const int n_tiles = min(seq_tile_cnt[b], n_tile_cap);
+    const int rwarp = kWarps - 1 - warp;   // work is dealt from the last warp down: warp 0 also scouts ahead
+    int dec_b = 0, dec_pref = 0;           // ticket decoding state (warp 0)
 
-    // ---- which tile ----
-    int t;
-    if (kMode == kLookBack) {   // ticket order: every earlier tile of this head is held by a running block
-        if (tid == 0) misc[0] = atomicAdd(&tickets[bh], 1);
-        __syncthreads();
-        t = misc[0];
-    } else {
-        t = blockIdx.x;
+    if (tid == 0) {
+        mbar_init(bar_k, 1);
+        mbar_init(bar_v, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (t >= n_tiles) return;
-
-    const int32_t* ts = tile_seg + (size_t)b * (n_tile_cap + 1);
-    const int s_begin = ts[t], s_end = ts[t + 1];
-    const int nseg = min(s_end - s_begin, kShortRows);
-    const int g_row0 = seg_off[s_begin];                       // on the flattened [B*n] axis
-    const int R = min(seg_off[s_begin + nseg] - g_row0, kMaxRows);
-    const int row0 = g_row0 - b * n;                           // within the sequence
-    const bool long_tile = R > kShortRows;
-    const int nrb = (R + 31) >> 5;
-
-    // ---- 1. stage K (and V) ----
-    const uint32_t sbase = smem_u32(smem);
-    const __nv_bfloat16* Kt = K + b * st.b + h * st.h + (int64_t)row0 * st.n;
-    const __nv_bfloat16* Vt = V + b * st.b + h * st.h + (int64_t)row0 * st.n;
-    {
-        const int c = tid & 15;
-        for (int r = tid >> 4; r < R; r += kThreads / 16) cp_async16(sbase + swz(r, c), Kt + (int64_t)r * st.n + c * 8);
-        cp_async_commit();
-        if (kMode != kCountOnly && !long_tile)
-            for (int r = tid >> 4; r < R; r += kThreads / 16)
-                cp_async16(sbase + kShortRows * kRowBytes + swz(r, c), Vt + (int64_t)r * st.n + c * 8);
-        cp_async_commit();
-    }
-
-    // ---- segment bookkeeping (while the copies fly) ----
-    for (int i = tid; i <= nseg; i += kThreads) segs[i] = (int16_t)min(seg_off[s_begin + i] - g_row0, kMaxRows);
-    if (tid < kNW) seedmask[tid] = 0u;
+    if (warp == 0) fetch_tile<kMode>(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
+    fence_async_proxy();
     __syncthreads();
-    for (int r = tid; r < nrb * 32; r += kThreads) {   // end of the segment each row belongs to (0 past the tile)
-        int lo = 0, hi = nseg;                         // find s with segs[s] <= r < segs[s+1]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (segs[mid] <= r) lo = mid; else hi = mid;
+
+    uint32_t phase_k = 0, phase_v = 0;
+    int buf = 0;
+    bool failed = false;
+#ifdef SC_PHASE_TIMING
+    long long t_prev = clock64();
+#endif
+    for (;;) {
+        const int* geo = geo_buf + buf * 8;
+        const int16_t* segs = segs_buf + buf * kSegsStride;
+        const int t = geo[gT];
+        if (t < 0) break;
+        const int b = geo[gB], h = geo[gH], nseg = geo[gNseg], row0 = geo[gRow0], R = geo[gR];
+        const int bh = b * p.Hkv + h;
+        const bool long_tile = R > kShortRows;
+        const bool two_tensors = (kMode != kCountOnly) && !long_tile;   // V staged beside K
+        const int nrb = (R + 31) >> 5;
+        const int64_t goff = b * p.st.b + h * p.st.h + (int64_t)row0 * p.st.n;
+
+        // ---- 1. stage the rows ----
+        if (tid == 0) {
+            mbar_expect_tx(bar_k, (uint32_t)R * kRowBytes);
+            if (two_tensors) mbar_expect_tx(bar_v, (uint32_t)R * kRowBytes);
         }
-        send[r] = (r < R) ? (uint16_t)segs[lo + 1] : (uint16_t)0;
-    }
-    __syncthreads();
-    if (tid == 0) {   // list the Gram blocks: diagonals first, then the blocks right of them a segment reaches
-        int k = 0;
-        for (int rb = 0; rb < nrb; ++rb) items[k++] = (uint8_t)((rb << 4) | rb);
-        for (int rb = 0; rb < nrb; ++rb) {
-            const int last = min(rb * 32 + 31, R - 1);
-            const int cbmax = ((int)send[last] - 1) >> 5;
-            for (int cb = rb + 1; cb <= cbmax; ++cb) items[k++] = (uint8_t)((rb << 4) | cb);
+        if (long_tile) {
+            if (tid < R) bulk_g2s(sbase + tid * kPitch, p.K + goff + (int64_t)tid * p.st.n, kRowBytes, bar_k);
+        } else if (tid < kShortRows) {
+            if (tid < R) bulk_g2s(sbase + tid * kPitch, p.K + goff + (int64_t)tid * p.st.n, kRowBytes, bar_k);
+        } else if (two_tensors) {
+            const int r = tid - kShortRows;
+            if (r < R) bulk_g2s(sbase + kVOff + r * kPitch, p.V + goff + (int64_t)r * p.st.n, kRowBytes, bar_v);
         }
-        misc[1] = k;
-    }
-    cp_async_wait<1>();   // K has landed (this thread's copies); the barrier publishes everyone's
-    __syncthreads();
-
-    // ---- 2. Gram blocks -> norms -> adjacency bits ----
-    const int n_items = misc[1];
-    {
-        float acc[2][4][4];
-        const bool have = warp < n_items;
-        int rb = 0, cb = 0;
-        if (have) {
-            rb = items[warp] >> 4; cb = items[warp] & 15;
-            gram_block(sbase, rb, cb, lane, acc);
-            if (rb == cb) {   // diagonal of the Gram block = squared norms
-                const int g = lane >> 2, tig = lane & 3;
-                if ((g >> 1) == tig) {
-                    const int e = g & 1;
-#pragma unroll
-                    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-                        for (int hh = 0; hh < 2; ++hh)
-                            norm[rb * 32 + mt * 16 + hh * 8 + g] =
-                                sqrtf(e ? acc[mt][2 * mt + hh][hh * 2 + 1] : acc[mt][2 * mt + hh][hh * 2]);
-                }
+        {   // rows [R, next multiple of 16) take part in the Eq. 3 product with zero weight: keep them finite
+            const int pad_chunks = (((R + 15) & ~15) - R) * 16;
+            for (int i = tid; i < pad_chunks; i += kThreads) {
+                unsigned char* dst = smem + (R + (i >> 4)) * kPitch + (i & 15) * 16;
+                *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
+                if (two_tensors) *reinterpret_cast<uint4*>(dst + kVOff) = make_uint4(0, 0, 0, 0);
             }
         }
-        __syncthreads();
-        if (have) threshold_block(acc, rb, cb, lane, tau, norm, send, adj);
-        for (int k = warp + kWarps; k < n_items; k += kWarps) {
-            rb = items[k] >> 4; cb = items[k] & 15;
-            gram_block(sbase, rb, cb, lane, acc);
-            threshold_block(acc, rb, cb, lane, tau, norm, send, adj);
-        }
-    }
-    __syncthreads();
+        CF_T(0);
 
-    // ---- 3. Algorithm 1 per segment: one warp per segment, lane c owns word c ----
-    int32_t* as = assign ? assign + (size_t)bh * n + row0 : nullptr;
-    for (int s = warp; s < nseg; s += kWarps) {
-        const int a = segs[s], e = segs[s + 1];
-        if (e - a == 1) {   // a delimiter or a one-token run: its own cluster
-            if (lane == 0) {
-                adj[a * kNW + (a >> 5)] = 1u << (a & 31);
-                atomicOr(&seedmask[a >> 5], 1u << (a & 31));
-                if (as) as[a] = row0 + a;
-            }
-            continue;
-        }
-        const int w0 = a >> 5, w1 = (e - 1) >> 5;
-        uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
-        uint32_t seeds = 0u;
-        for (;;) {
-            const uint32_t any = __ballot_sync(kFull, U != 0u);
-            if (any == 0u) break;
-            const int wf = __ffs(any) - 1;
-            const int i = wf * 32 + __ffs(__shfl_sync(kFull, U, wf)) - 1;   // lowest unassigned token: a seed
-            uint32_t mem = 0u;
-            if (lane >= w0 && lane <= w1) {
-                mem = adj[i * kNW + lane] & U;
-                if (lane == wf) { mem |= 1u << (i & 31); seeds |= 1u << (i & 31); }
-                adj[i * kNW + lane] = mem;            // the row now lists the cluster's members
-                U &= ~mem;
-                if (as) {
-                    uint32_t mm = mem;
-                    while (mm) { const int j = lane * 32 + __ffs(mm) - 1; mm &= mm - 1; as[j] = row0 + i; }
-                }
-            }
-        }
-        if (seeds) atomicOr(&seedmask[lane], seeds);
-    }
-    __syncthreads();
-
-    // ---- 4. output offset of this tile ----
-    int P = 0;
-#pragma unroll
-    for (int w = 0; w < kNW; ++w) P += __popc(seedmask[w]);
-    if (kMode == kCountOnly) {
-        if (tid == 0) tile_state[(size_t)bh * n_tile_cap + t] = (uint32_t)P;
-        return;
-    }
-    if (warp == 0) {
-        int base = 0;
-        uint32_t* stt = tile_state + (size_t)bh * n_tile_cap;
-        if (kMode == kWriteWithCounts) {
-            for (int k = lane; k < t; k += 32) base += (int)stt[k];
-            base = warp_sum_i(base);
+        // ---- scout: next ticket, its geometry, L2 prefetch (warp 0); segment bookkeeping (others) ----
+        if (warp == 0) {
+            fetch_tile<kMode>(p, lane, dec_b, dec_pref, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
         } else {
-            if (lane == 0) atomicExch(&stt[t], (t == 0 ? kFlagPrefix : kFlagAggregate) | (uint32_t)P);
-            // look back over the predecessors, 32 at a time, nearest first
-            int upto = t;      // tiles [0, upto) still to be accounted for
-            int spins = 0;
-            bool gave_up = false;
-            while (upto > 0) {
-                const int k = upto - 1 - lane;
-                uint32_t v = (k >= 0) ? ld_volatile(&stt[k]) : kFlagPrefix;   // before tile 0: prefix 0
-                const uint32_t ready = __ballot_sync(kFull, (v >> 30) != 0u);
-                const uint32_t pref = __ballot_sync(kFull, (v >> 30) == 2u);
-                // usable run: lanes 0..m-1 all ready, stopping at the first that holds a full prefix
-                const int first_unready = (ready == kFull) ? 32 : __ffs(~ready) - 1;
-                const int first_pref = pref ? __ffs(pref) - 1 : 32;
-                const int take = min(first_unready, first_pref + 1);
-                int contrib = (lane < take) ? (int)(v & kValueMask) : 0;
-                base += warp_sum_i(contrib);
-                if (first_pref < first_unready) break;        // reached an inclusive prefix
-                upto -= take;
-                if (take == 0) {
-                    if (++spins > kSpinLimit) { gave_up = true; break; }
-                    __nanosleep(40);
+            if (tid - 32 < kNW) seedmask[tid - 32] = 0u;
+            for (int r = tid - 32; r < nrb * 32; r += kThreads - 32) {   // end of the segment each row is in
+                int lo = 0, hi = nseg;                                    // segs[lo] <= r < segs[hi]
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (segs[mid] <= r) lo = mid; else hi = mid;
                 }
-            }
-            if (gave_up) { set_status(status, SC_ERR_TIMEOUT); base = 0; }
-            if (lane == 0 && t > 0) atomicExch(&stt[t], kFlagPrefix | (uint32_t)(base + P));
-        }
-        if (lane == 0) {
-            misc[2] = base;
-            if (t == n_tiles - 1) {
-                core_len[bh] = base + P;
-                if (base + P > cap) set_status(status, SC_ERR_CAPACITY);
+                send[r] = (r < R) ? (uint16_t)segs[lo + 1] : (uint16_t)0;
             }
         }
-    }
-    cp_async_wait<0>();   // V
-    __syncthreads();
-    const int base = misc[2];
+        CF_T(1);
+        failed = !mbar_wait(bar_k, phase_k);
+        phase_k ^= 1u;
+        if (__syncthreads_or(failed)) { failed = true; break; }
+        CF_T(2);
 
-    // ---- 5. Eq. 3: one warp per cluster ----
-    const unsigned char* ksm = smem;
-    const unsigned char* vsm = smem + kShortRows * kRowBytes;
-    const size_t obase = (size_t)bh * cap;
-    int rank_base = 0;
-    for (int w = 0; w < nrb; ++w) {
-        const uint32_t sm = seedmask[w];
-        uint32_t m = sm;
-        while (m) {
-            const int bit = __ffs(m) - 1;
-            m &= m - 1;
-            const int rank = rank_base + __popc(sm & ((1u << bit) - 1u));
-            if ((rank & (kWarps - 1)) != warp) continue;
-            const int i = w * 32 + bit;
-            const int w1 = ((int)send[i] - 1) >> 5;
-            float ak[4] = {0.f, 0.f, 0.f, 0.f}, av[4] = {0.f, 0.f, 0.f, 0.f};
-            int cnt = 0;
-            for (int ww = w; ww <= w1; ++ww) {
-                uint32_t mm = adj[i * kNW + ww];
-                cnt += __popc(mm);
-                while (mm) {
-                    const int j = ww * 32 + __ffs(mm) - 1;
-                    mm &= mm - 1;
-                    const uint32_t off = swz(j, lane >> 1) + (lane & 1) * 8;
-                    const uint2 kk = *reinterpret_cast<const uint2*>(ksm + off);
-                    uint2 vv;
-                    if (!long_tile) vv = *reinterpret_cast<const uint2*>(vsm + off);
-                    else vv = __ldg(reinterpret_cast<const uint2*>(Vt + (int64_t)j * st.n + lane * 4));
-                    ak[0] += __uint_as_float(kk.x << 16); ak[1] += __uint_as_float(kk.x & 0xffff0000u);
-                    ak[2] += __uint_as_float(kk.y << 16); ak[3] += __uint_as_float(kk.y & 0xffff0000u);
-                    av[0] += __uint_as_float(vv.x << 16); av[1] += __uint_as_float(vv.x & 0xffff0000u);
-                    av[2] += __uint_as_float(vv.y << 16); av[3] += __uint_as_float(vv.y & 0xffff0000u);
+        // ---- 2. Gram blocks -> norms -> adjacency bits ----
+        {
+            float acc[2][4][4];
+            const bool have = rwarp < nrb;
+            if (have) {
+                gram_block(sbase, rwarp, rwarp, lane, acc);
+                store_norms(acc, rwarp, lane, norm);
+            }
+            __syncthreads();
+            CF_T(3);
+            if (have) {
+                if (p.tau < 0.f) threshold_block<true>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
+                else threshold_block<false>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
+            }
+            if (nrb > 1) {
+                for (int k = rwarp; k < 28; k += kWarps) {
+                    const int rb = kOffDiag[k] >> 4, cb = kOffDiag[k] & 15;
+                    if (cb >= nrb) continue;
+                    const int reach = ((int)send[min(rb * 32 + 31, R - 1)] - 1) >> 5;   // last block a segment of rb spans
+                    if (cb > reach) continue;
+                    gram_block(sbase, rb, cb, lane, acc);
+                    if (p.tau < 0.f) threshold_block<true>(acc, rb, cb, lane, p.tau, norm, send, adj);
+                    else threshold_block<false>(acc, rb, cb, lane, p.tau, norm, send, adj);
                 }
             }
-            const int row = base + rank;
-            if (row < cap) {
-                const float inv = 1.0f / (float)cnt;
-                __nv_bfloat162 k01 = __floats2bfloat162_rn(ak[0] * inv, ak[1] * inv);
-                __nv_bfloat162 k23 = __floats2bfloat162_rn(ak[2] * inv, ak[3] * inv);
-                __nv_bfloat162 v01 = __floats2bfloat162_rn(av[0] * inv, av[1] * inv);
-                __nv_bfloat162 v23 = __floats2bfloat162_rn(av[2] * inv, av[3] * inv);
-                uint2 ko, vo;
-                ko.x = *reinterpret_cast<uint32_t*>(&k01); ko.y = *reinterpret_cast<uint32_t*>(&k23);
-                vo.x = *reinterpret_cast<uint32_t*>(&v01); vo.y = *reinterpret_cast<uint32_t*>(&v23);
-                *reinterpret_cast<uint2*>(core_k + (obase + row) * kD + lane * 4) = ko;
-                *reinterpret_cast<uint2*>(core_v + (obase + row) * kD + lane * 4) = vo;
-                if (lane == 0) count[obase + row] = cnt;
+        }
+        __syncthreads();
+        CF_T(4);
+
+        // ---- 3. Algorithm 1 per segment: one warp per segment, lane c owns word c ----
+        int32_t* as = p.assign ? p.assign + (size_t)bh * p.n + row0 : nullptr;
+        for (int s = rwarp; s < nseg; s += kWarps) {
+            const int a = segs[s], e = segs[s + 1];
+            if (e - a == 1) {   // a delimiter or a one-token run: its own cluster
+                if (lane == 0) {
+                    adj[adj_row(a)] = 1u << (a & 31);
+                    atomicOr(&seedmask[a >> 5], 1u << (a & 31));
+                    if (as) as[a] = row0 + a;
+                }
+                continue;
+            }
+            const int w1 = (e - 1) >> 5;
+            uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
+            uint32_t seeds = 0u;
+            for (;;) {
+                const uint32_t any = __ballot_sync(kFull, U != 0u);
+                if (any == 0u) break;
+                const int wf = __ffs(any) - 1;
+                const int i = wf * 32 + __ffs(__shfl_sync(kFull, U, wf)) - 1;   // lowest unassigned token: a seed
+                if (lane >= wf && lane <= w1) {
+                    uint32_t* slot = adj + adj_row(i) + (lane - wf);
+                    uint32_t mem = *slot & U;
+                    if (lane == wf) { mem |= 1u << (i & 31); seeds |= 1u << (i & 31); }
+                    *slot = mem;            // the row now lists the cluster's members
+                    U &= ~mem;
+                    if (as) {
+                        uint32_t mm = mem;
+                        while (mm) { const int j = lane * 32 + __ffs(mm) - 1; mm &= mm - 1; as[j] = row0 + i; }
+                    }
+                }
+            }
+            if (seeds) atomicOr(&seedmask[lane], seeds);
+        }
+        __syncthreads();
+        CF_T(5);
+
+        // ---- 4. cluster count of the tile; publish it; seed row of every cluster ----
+        int P = 0;
+#pragma unroll
+        for (int w = 0; w < kNW; ++w) P += __popc(seedmask[w]);
+        uint32_t* stt = p.tile_state + (size_t)bh * p.n_tile_cap;
+        if (kMode == kCountOnly) {
+            if (tid == 0) stt[t] = (uint32_t)P;
+        } else {
+            if (kMode == kLookBack && tid == 0)
+                atomicExch(&stt[t], (t == 0 ? kFlagPrefix : kFlagAggregate) | (uint32_t)P);
+            if (tid < R) {
+                const uint32_t wbits = seedmask[tid >> 5];
+                if ((wbits >> (tid & 31)) & 1u) {
+                    int rank = __popc(wbits & ((1u << (tid & 31)) - 1u));
+                    for (int w = 0; w < (tid >> 5); ++w) rank += __popc(seedmask[w]);
+                    seedrow[rank] = (uint16_t)tid;
+                }
+            }
+            if (two_tensors) {
+                failed = !mbar_wait(bar_v, phase_v);
+                phase_v ^= 1u;
+            }
+            if (__syncthreads_or(failed)) { failed = true; break; }
+            CF_T(6);
+
+            // ---- 5. Eq. 3 (K, and V when it is staged) ----
+            if (long_tile)
+                merge_rounds(sbase, smem, (warp & 1) * 128, warp >> 1, 4, P, seedrow, send, adj, lane, (warp & 1) == 0);
+            else
+                merge_rounds(sbase + ((warp >> 1) & 1) * kVOff, smem + ((warp >> 1) & 1) * kVOff, (warp & 1) * 128,
+                             warp >> 2, 2, P, seedrow, send, adj, lane, (warp & 3) == 0);
+            CF_T(7);
+
+            // ---- output offset of the tile (warp 0) ----
+            if (warp == 0) {
+                int base = 0;
+                if (kMode == kWriteWithCounts) {
+                    for (int k = lane; k < t; k += 32) base += (int)stt[k];
+                    base = warp_sum_i(base);
+                } else {
+                    // look back over the predecessors, 32 at a time, nearest first
+                    int upto = t;      // tiles [0, upto) still to be accounted for
+                    bool gave_up = false;
+                    unsigned long long t0 = 0;
+                    while (upto > 0) {
+                        const int k = upto - 1 - lane;
+                        const uint32_t v = (k >= 0) ? ld_volatile(&stt[k]) : kFlagPrefix;   // before tile 0: prefix 0
+                        const uint32_t ready = __ballot_sync(kFull, (v >> 30) != 0u);
+                        const uint32_t pref = __ballot_sync(kFull, (v >> 30) == 2u);
+                        // usable run: lanes 0..m-1 all ready, stopping at the first that holds a full prefix
+                        const int first_unready = (ready == kFull) ? 32 : __ffs(~ready) - 1;
+                        const int first_pref = pref ? __ffs(pref) - 1 : 32;
+                        const int take = min(first_unready, first_pref + 1);
+                        const int contrib = (lane < take) ? (int)(v & kValueMask) : 0;
+                        base += warp_sum_i(contrib);
+                        if (first_pref < first_unready) break;        // reached an inclusive prefix
+                        upto -= take;
+                        if (take == 0) {
+                            if (t0 == 0) t0 = global_ns();
+                            else if (global_ns() - t0 > kWaitLimitNs) { gave_up = true; break; }
+                            __nanosleep(64);
+                        }
+                    }
+                    if (gave_up) { set_status(p.status, SC_ERR_TIMEOUT); base = 0; }
+                    if (lane == 0 && t > 0) atomicExch(&stt[t], kFlagPrefix | (uint32_t)(base + P));
+                }
+                if (lane == 0) {
+                    misc[0] = base;
+                    if (geo[gLast]) {
+                        p.core_len[bh] = base + P;
+                        if (base + P > p.cap) set_status(p.status, SC_ERR_CAPACITY);
+                    }
+                }
+            }
+            __syncthreads();
+            CF_T(8);
+
+            // ---- compact, coalesced stores of the cores ----
+            const int base = misc[0];
+            const size_t obase = (size_t)bh * p.cap;
+            for (int idx = tid; idx < P * 16; idx += kThreads) {
+                const int row = idx >> 4, c = idx & 15;
+                if (base + row < p.cap) {
+                    const size_t o = (obase + base + row) * kD + c * 8;
+                    *reinterpret_cast<uint4*>(p.core_k + o) = *reinterpret_cast<const uint4*>(smem + row * kPitch + c * 16);
+                    if (!long_tile)
+                        *reinterpret_cast<uint4*>(p.core_v + o) =
+                            *reinterpret_cast<const uint4*>(smem + kVOff + row * kPitch + c * 16);
+                }
+            }
+            for (int row = tid; row < P; row += kThreads)
+                if (base + row < p.cap)
+                    p.count[obase + base + row] = *reinterpret_cast<const int*>(smem + row * kPitch + kRowBytes);
+
+            // ---- a long segment: V takes the place of K and goes through the same product ----
+            if (long_tile) {
+                fence_async_proxy();
+                __syncthreads();
+                if (tid == 0) mbar_expect_tx(bar_v, (uint32_t)R * kRowBytes);
+                if (tid < R) bulk_g2s(sbase + tid * kPitch, p.V + goff + (int64_t)tid * p.st.n, kRowBytes, bar_v);
+                failed = !mbar_wait(bar_v, phase_v);
+                phase_v ^= 1u;
+                if (__syncthreads_or(failed)) { failed = true; break; }
+                merge_rounds(sbase, smem, (warp & 1) * 128, warp >> 1, 4, P, seedrow, send, adj, lane, false);
+                __syncthreads();
+                for (int idx = tid; idx < P * 16; idx += kThreads) {
+                    const int row = idx >> 4, c = idx & 15;
+                    if (base + row < p.cap)
+                        *reinterpret_cast<uint4*>(p.core_v + (obase + base + row) * kD + c * 8) =
+                            *reinterpret_cast<const uint4*>(smem + row * kPitch + c * 16);
+                }
             }
         }
-        rank_base += __popc(sm);
+
+        // the next tile's bulk copies overwrite what this one read and wrote through ordinary accesses
+        fence_async_proxy();
+        __syncthreads();
+        CF_T(9);
+        buf ^= 1;
+    }
+
+    // ---- exit: the last block to finish leaves the workspace zeroed for the next call ----
+    if (failed) {
+        if (tid == 0) set_status(p.status, SC_ERR_TIMEOUT);
+        mbar_wait(bar_k, phase_k ^ 1u);   // bounded: let copies that may still be in flight land before leaving
+        mbar_wait(bar_v, phase_v ^ 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const int done = atomicAdd(&p.ctl[1], 1);
+        misc[1] = (done == (int)gridDim.x - 1);
+    }
+    __syncthreads();
+    if (misc[1]) {
+        __threadfence();
+        if (kMode != kCountOnly) {
+            const size_t words = (size_t)p.B * p.Hkv * p.n_tile_cap;
+            for (size_t i = tid; i < words; i += kThreads) p.tile_state[i] = 0u;
+        }
+        if (tid == 0) { p.ctl[0] = 0; p.ctl[1] = 0; }
     }
 }
 
 }  // namespace cf
 
 bool compress_fused_supported(const CompressArgs& a) {
-    return a.dt == SC_BF16 && a.d == cf::kD && a.Hkv <= 65535 && a.B <= 65535 && a.n_tile_cap >= 1;
+    // ticket arithmetic is 32-bit
+    return a.dt == SC_BF16 && a.d == cf::kD && a.n_tile_cap >= 1 &&
+           (int64_t)a.B * a.Hkv * (int64_t)a.n_tile_cap < (int64_t)1 << 30;
 }
 
 size_t compress_fused_ws_bytes(int32_t B, int32_t Hkv, int32_t n) {
     const size_t tiles = 2 * (size_t)div_up(n, SC_TILE_ROWS) + 1;
-    return sizeof(uint32_t) * (size_t)B * Hkv * (tiles + 1) + 256;
+    return sizeof(uint32_t) * ((size_t)B * Hkv * tiles + cf::kCtlWords) + 256;
 }
 
 cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
-    static bool attr_set[64] = {false};
+    static int grid_of[64] = {0};   // per device: blocks that are resident at once
     int dev = 0;
     cudaGetDevice(&dev);
     dev &= 63;
-    if (!attr_set[dev]) {
+    if (grid_of[dev] == 0) {
         cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kCountOnly>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
         cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kWriteWithCounts>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
         cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kLookBack>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
-        attr_set[dev] = true;
+        int sms = 0, per_sm = 0;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cf::compress_fused_kernel<cf::kLookBack>, cf::kThreads,
+                                                      cf::kSmemBytes);
+        grid_of[dev] = (sms < 1 ? 1 : sms) * (per_sm < 1 ? 1 : per_sm);
     }
-    const size_t heads = (size_t)a.B * a.Hkv;
-    uint32_t* tile_state = (uint32_t*)a.ws;
-    int32_t* tickets = (int32_t*)(tile_state + heads * a.n_tile_cap);
-    dim3 grid(a.n_tile_cap, a.Hkv, a.B);
-    const __nv_bfloat16* K = (const __nv_bfloat16*)a.K;
-    const __nv_bfloat16* V = (const __nv_bfloat16*)a.V;
-    __nv_bfloat16* ck = (__nv_bfloat16*)a.core_k;
-    __nv_bfloat16* cv = (__nv_bfloat16*)a.core_v;
+    cf::Params p;
+    p.K = (const __nv_bfloat16*)a.K; p.V = (const __nv_bfloat16*)a.V; p.st = a.st;
+    p.B = a.B; p.Hkv = a.Hkv; p.n = a.n;
+    p.seg_off = a.seg_off; p.tile_seg = a.tile_seg; p.seq_tile_cnt = a.seq_tile_cnt; p.n_tile_cap = a.n_tile_cap;
+    p.tau = a.tau;
+    p.core_k = (__nv_bfloat16*)a.core_k; p.core_v = (__nv_bfloat16*)a.core_v; p.count = a.count; p.cap = a.cap;
+    p.core_len = a.core_len; p.assign = a.assign;
+    p.ctl = (int32_t*)a.ws;
+    p.tile_state = (uint32_t*)a.ws + cf::kCtlWords;
+    p.status = a.status;
+    // no more blocks than there can be tiles
+    const int64_t max_tiles = (int64_t)a.B * a.Hkv * a.n_tile_cap;
+    const int grid = (int)(max_tiles < grid_of[dev] ? max_tiles : grid_of[dev]);
     if (a.flags & SC_FLAG_TWO_PASS) {
-        cf::compress_fused_kernel<cf::kCountOnly><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(
-            K, V, a.st, a.Hkv, a.n, a.seg_off, a.tile_seg, a.seq_tile_cnt, a.n_tile_cap, a.tau, ck, cv, a.count, a.cap,
-            a.core_len, nullptr, tile_state, tickets, a.status);
-        cf::compress_fused_kernel<cf::kWriteWithCounts><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(
-            K, V, a.st, a.Hkv, a.n, a.seg_off, a.tile_seg, a.seq_tile_cnt, a.n_tile_cap, a.tau, ck, cv, a.count, a.cap,
-            a.core_len, a.assign, tile_state, tickets, a.status);
+        cf::Params pc = p;
+        pc.assign = nullptr;
+        cf::compress_fused_kernel<cf::kCountOnly><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(pc);
+        cf::compress_fused_kernel<cf::kWriteWithCounts><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
         note_launches(2);
     } else {
-        cudaError_t e = cudaMemsetAsync(a.ws, 0, sizeof(uint32_t) * heads * (a.n_tile_cap + 1), st);
-        if (e != cudaSuccess) return e;
-        cf::compress_fused_kernel<cf::kLookBack><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(
-            K, V, a.st, a.Hkv, a.n, a.seg_off, a.tile_seg, a.seq_tile_cnt, a.n_tile_cap, a.tau, ck, cv, a.count, a.cap,
-            a.core_len, a.assign, tile_state, tickets, a.status);
+        cf::compress_fused_kernel<cf::kLookBack><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
         note_launches(1);
     }
     return cudaGetLastError();
 }
 
 }  // namespace sc
+
+#ifdef SC_PHASE_TIMING
+extern "C" __attribute__((visibility("default"))) int sc_debug_phase_cycles(unsigned long long* host16, int reset) {
+    cudaError_t e = cudaMemcpyFromSymbol(host16, sc::cf::g_phase_cycles, 16 * sizeof(unsigned long long));
+    if (e == cudaSuccess && reset) {
+        unsigned long long z[16] = {0};
+        e = cudaMemcpyToSymbol(sc::cf::g_phase_cycles, z, sizeof(z));
+    }
+    return (int)e;
+}
+#endif

@@ -201,6 +201,72 @@ def test_compress_capacity_overflow_is_reported_not_written(flags):
     compare_compressed(view, ref_cap, torch.bfloat16)
 
 
+@pytest.mark.parametrize("cfg,kw", [(1, {}), (3, dict(tau=0.9, sigma=0.15)), (4, dict(B=1, gap=("poisson", 128.0))),
+                                    (4, dict(B=2, n=32768, gap=("poisson", 8.0), centroids=("ratio", 2.0)))])
+def test_compress_full_size_layer_of_the_benchmark_shapes(cfg, kw):
+    """One whole layer at the benchmark's sizes (every block walks many tiles; cfg4 with mean chunk
+    length 128 is mostly tiles longer than SC_TILE_ROWS), compared in full with the oracle."""
+    w = synth.config(cfg, L=1, **kw)
+    ref, got, plan, _ = _compress_both(w, layer=0)
+    binding.check_status(plan.status)
+    assert ref["margin"] > 1e-4
+    compare_compressed(got, ref, torch.bfloat16)
+
+
+def test_compress_near_ties_are_decided_consistently():
+    """Noise 0.3 at tau = 0.9 puts similarities on both sides of the threshold, some within rounding of
+    it, where fp32 (GPU) and fp64 (oracle) may decide differently and both partitions are valid runs of
+    Algorithm 1.  What is unique is checked exactly: replaying Algorithm 1 along the GPU's partition,
+    every comparison whose similarity is clear of tau (by 1e-5) must have been decided as Eq. 2 says;
+    the merged cores must then equal Eq. 3 applied to the GPU's own partition."""
+    w = synth.config(3, L=1, n=8192, Hkv=2, Hq=14, tau=0.9, sigma=0.3)
+    ids, run_id, run_lens = synth.token_ids(w)
+    K, V = synth.layer_kv(w, 0, run_id, run_lens)
+    Kb, Vb = synth.to_numpy_bits(K), synth.to_numpy_bits(V)
+    seg_off, seq_seg_off = oracle.chunk(ids.numpy(), w.delims, w.max_chunk_len)
+    assert oracle.gsc(Kb, seg_off, seq_seg_off, w.tau)[1] < 1e-4      # the oracle does meet near-ties here
+    plan = binding.chunk(ids.to(DEV), w.delims, w.max_chunk_len)
+    got = binding.compress(K.to(DEV), V.to(DEV), plan, w.tau, want_assign=True)
+    binding.check_status(plan.status)
+    assign = got.assign.cpu().numpy()
+    for h in range(w.Hkv):
+        for s in range(len(seg_off) - 1):
+            a, e = int(seg_off[s]), int(seg_off[s + 1])
+            taken = np.zeros(e - a, dtype=bool)
+            for i in range(a, e):
+                if taken[i - a]:
+                    continue
+                assert assign[0, h, i] == i, "the lowest unassigned token must be a seed"
+                taken[i - a] = True
+                for j in range(i + 1, e):
+                    if taken[j - a]:
+                        continue
+                    joined = assign[0, h, j] == i
+                    sim = oracle.sim(Kb[0, h], i, j)
+                    if abs(sim - w.tau) > 1e-5:
+                        assert joined == (sim > w.tau), (h, i, j, sim)
+                    taken[j - a] |= joined
+            assert taken.all()
+    ck, cv, cnt, clen = oracle.merge(Kb, Vb, assign, None, seg_off, seq_seg_off)
+    compare_compressed(got, dict(core_k=ck, core_v=cv, count=cnt, core_len=clen, assign=assign), torch.bfloat16)
+
+
+def test_compress_workspace_is_left_clean_and_can_be_shared_by_consecutive_calls():
+    w = synth.config(0, n=6000, L=3, gap=("poisson", 40.0))
+    ids, run_id, run_lens = synth.token_ids(w)
+    plan = binding.chunk(ids.to(DEV), w.delims)
+    ws = binding.compress_workspace(w.B, w.Hkv, w.n, DEV)
+    for rep in range(2):
+        for layer, flags in enumerate((0, binding.SC_FLAG_GENERIC, binding.SC_FLAG_TWO_PASS, 0)):
+            K, V = synth.layer_kv(w, layer % w.L, run_id, run_lens)
+            ref = oracle_compress(ids, K, V, w.delims, w.tau)
+            got = binding.compress(K.to(DEV), V.to(DEV), plan, w.tau, want_assign=True, workspace=ws, flags=flags)
+            binding.check_status(plan.status)
+            compare_compressed(got, ref, torch.bfloat16)
+            n_words = 64 + w.B * w.Hkv * plan.n_tile_cap
+            assert int(ws.view(torch.int32)[:n_words].abs().max()) == 0, "status words and counters are zero again"
+
+
 # ---------------------------------------------------------------------------- sc_decode_attn
 
 
