@@ -4,10 +4,11 @@
 // counter.  A tile is a run of whole segments of at most SC_TILE_ROWS tokens of one (sequence, KV
 // head) -- K and V both staged in shared memory -- or one longer segment alone (K staged, then V
 // in a second pass over the same buffer).  Per tile:
-//   1. the rows are brought in with one bulk asynchronous copy per row (cp.async.bulk, completion
-//      on an mbarrier) into rows of 272 bytes: the 16-byte pad makes ldmatrix conflict free
-//      without address swizzling.  While a tile is processed the block already holds its next
-//      ticket and has asked L2 to prefetch that tile, so DRAM stays busy during the compute phases;
+//   1. the rows are staged with 16-byte cp.async copies into rows of 272 bytes (the 16-byte pad
+//      makes ldmatrix conflict free without address swizzling).  Tickets walk the cache in memory
+//      order, so each block also asks L2 to prefetch the rows a fixed distance ahead of its tile
+//      (about what all resident blocks hold together): DRAM stays busy during the compute phases
+//      and the copies into shared memory mostly hit L2;
 //   2. Gram blocks K.K^T of 32x32 rows on the tensor cores (mma.m16n8k16; bf16 products are exact
 //      in fp32) for exactly the block pairs a segment spans; the diagonal gives the norms and
 //      Sim > tau (Eq. 2) is decided as G_ij > tau*|k_i|*|k_j|, packed into adjacency bit rows
@@ -19,9 +20,10 @@
 //      decoupled look-back over per-tile status words (tickets are handed out in order, so every
 //      predecessor is held by a running block and the bounded wait cannot starve), or, in
 //      two-pass mode, a count pass followed by a write pass;
-//   5. Eq. 3 as a product on the tensor cores: member masks expanded to a 0/1 bf16 matrix times
-//      the staged K (V) rows, fp32 accumulation, one multiply by 1/|S|, one rounding to bf16; the
-//      cores are compacted in place in shared memory and leave with 16-byte coalesced stores.
+//   5. Eq. 3 as a product on the tensor cores (warps 4-7): member masks expanded to a 0/1 bf16
+//      matrix times the staged K (V) rows, fp32 accumulation, one multiply by 1/|S|, one rounding
+//      to bf16; the cores are compacted in place in shared memory and leave with 16-byte
+//      coalesced stores.  Meanwhile warp 0 draws the block's next ticket and warp 1 looks back.
 // The last block to finish zeroes the status words and counters, so a workspace that was zero
 // before the call is zero again after it.
 #include "common.cuh"
@@ -47,9 +49,7 @@ constexpr int kSendOff = kNormOff + kMaxRows * 4; // uint16[256]: end of the seg
 constexpr int kSegsOff = kSendOff + kMaxRows * 2; // 2 x int16[132]: segment starts (this tile, next tile)
 constexpr int kSegsStride = 132;
 constexpr int kMiscOff = kSegsOff + 2 * kSegsStride * 2;   // uint32 seedmask[8]; int geo[2][8]; int misc[4]
-constexpr int kBarOff = kMiscOff + 32 + 64 + 16;  // two mbarriers (rows of K; rows of V)
-constexpr int kSmemBytes = kBarOff + 16;
-static_assert(kBarOff % 8 == 0, "mbarrier alignment");
+constexpr int kSmemBytes = kMiscOff + 32 + 64 + 16;
 static_assert(kSmemBytes <= 76800, "three blocks per SM need <= 75 KB each");
 
 enum Mode { kCountOnly = 0, kWriteWithCounts = 1, kLookBack = 2 };
@@ -71,7 +71,8 @@ __device__ unsigned long long g_phase_cycles[16];
 #endif
 
 constexpr uint32_t kFlagAggregate = 1u << 30, kFlagPrefix = 2u << 30, kValueMask = (1u << 30) - 1;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every wait gives up after 2 s
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // the look-back gives up after 2 s
+constexpr int kMergeWarp0 = 4;                               // warps 4..7 run the Eq. 3 product
 constexpr int kCtlWords = 64;                                // ticket, done counter, padding
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -80,37 +81,19 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+// 16-byte asynchronous copy; src_bytes = 0 fills the destination with zeros instead.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0u;
-}
-// Bounded wait for a phase of an mbarrier; false if it gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > kWaitLimitNs) return false;
-    }
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void merge_warps_sync() {   // the four warps of the Eq. 3 product
+    asm volatile("bar.sync 1, 128;\n" ::: "memory");
 }
 __device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -147,6 +130,7 @@ __device__ __forceinline__ uint32_t expand2(uint32_t two_bits) {
 }
 
 // 32x32 block of K.K^T: rows of block rb against rows of block cb (rows staged at pitch kPitch).
+template <bool kDiag>
 __device__ __forceinline__ void gram_block(uint32_t kbase, int rb, int cb, int lane, float (&acc)[2][4][4]) {
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
@@ -168,8 +152,10 @@ __device__ __forceinline__ void gram_block(uint32_t kbase, int rb, int cb, int l
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt)
+            for (int nt = 0; nt < 4; ++nt) {
+                if (kDiag && nt < 2 * mt) continue;   // wholly below the diagonal: never read
                 mma_bf16(acc[mt][nt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], bq[nt >> 1][(nt & 1) * 2], bq[nt >> 1][(nt & 1) * 2 + 1]);
+            }
     }
 }
 
@@ -189,7 +175,7 @@ __device__ __forceinline__ void store_norms(const float (&acc)[2][4][4], int rb,
 
 // Turns a Gram block into adjacency words: bit j of word (i, cb) = Sim(i, 32cb + j) > tau, limited
 // to later tokens of i's own segment.
-template <bool kNegTau>
+template <bool kNegTau, bool kDiag>
 __device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int rb, int cb, int lane, float tau,
                                                 const float* norm, const uint16_t* send, uint32_t* adj) {
     const int g = lane >> 2, tig = lane & 3;
@@ -208,7 +194,8 @@ __device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int
             const float ni = norm[i];
             uint32_t w = 0;   // bit nt*8 + e, moved to nt*8 + 2*tig + e afterwards
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt)
+            for (int nt = 0; nt < 4; ++nt) {
+                if (kDiag && nt < 2 * mt + hh) continue;   // columns before the row's own: masked out anyway
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const float thr = ni * tn[nt][e];
@@ -216,6 +203,7 @@ __device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int
                     if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
                     if (hit) w |= 1u << (nt * 8 + e);
                 }
+            }
             w <<= 2 * tig;
             w |= __shfl_xor_sync(kFull, w, 1);
             w |= __shfl_xor_sync(kFull, w, 2);
@@ -237,14 +225,15 @@ struct Params {
     int32_t* ctl;            // [0] ticket counter, [1] blocks finished
     uint32_t* tile_state;    // [B*Hkv][n_tile_cap]
     int32_t* status;
+    int ahead_rows;          // L2 prefetch distance in rows; 0 = the cache is not one contiguous [B*Hkv*n, d] array
+    int64_t total_rows;      // B*Hkv*n
 };
 
-// Warp 0 draws the next ticket, turns it into a tile (sequence, head, tile index, rows), copies the
-// tile's segment starts into shared memory and asks L2 to prefetch the tile's K and V rows.
-// Tickets walk the tiles of head 0 of sequence 0 in order, then head 1, ...; a block's tickets only
-// grow, so the sequence it last decoded (dec_b, with dec_pref tickets before it) is where the search
-// resumes.  geo[gT] = -1 when no work is left.
-template <int kMode>
+
+// Warp 0 draws the next ticket, turns it into a tile (sequence, head, tile index, rows) and copies
+// the tile's segment starts into shared memory.  Tickets walk the tiles of head 0 of sequence 0 in
+// order, then head 1, ...; a block's tickets only grow, so the sequence it last decoded (dec_b,
+// with dec_pref tickets before it) is where the search resumes.  geo[gT] = -1 when no work is left.
 __device__ __forceinline__ void fetch_tile(const Params& p, int lane, int& dec_b, int& dec_pref, int* geo,
                                            int16_t* segs) {
     int w = 0;
@@ -269,51 +258,60 @@ __device__ __forceinline__ void fetch_tile(const Params& p, int lane, int& dec_b
     const int g_row0 = p.seg_off[s_begin];
     for (int i = lane; i <= nseg; i += 32) segs[i] = (int16_t)min(p.seg_off[s_begin + i] - g_row0, kMaxRows);
     const int R = min(p.seg_off[s_begin + nseg] - g_row0, kMaxRows);
-    const int row0 = g_row0 - b * p.n;
     if (lane == 0) {
-        geo[gB] = b; geo[gH] = h; geo[gT] = t; geo[gNseg] = nseg; geo[gRow0] = row0; geo[gR] = R;
+        geo[gB] = b; geo[gH] = h; geo[gT] = t; geo[gNseg] = nseg; geo[gRow0] = g_row0 - b * p.n; geo[gR] = R;
         geo[gLast] = (t == nt - 1);
-    }
-    // L2 prefetch: one request per tensor when rows are contiguous, else one per row
-    const int64_t off = b * p.st.b + h * p.st.h + (int64_t)row0 * p.st.n;
-    if (p.st.n == kD) {
-        if (lane == 0) l2_prefetch(p.K + off, (uint32_t)R * kRowBytes);
-        if (lane == 1 && kMode != kCountOnly) l2_prefetch(p.V + off, (uint32_t)R * kRowBytes);
-    } else {
-        for (int i = lane; i < R; i += 32) {
-            l2_prefetch(p.K + off + (int64_t)i * p.st.n, kRowBytes);
-            if (kMode != kCountOnly) l2_prefetch(p.V + off + (int64_t)i * p.st.n, kRowBytes);
-        }
     }
 }
 
-// Eq. 3 on the tensor cores for one staged tensor (K or V rows at `area`, pitch kPitch).
-// Cluster c (in seed order) has its member mask in the adjacency row of its seed seedrow[c].  A
-// warp owns one tile of 16 clusters (mt_in_round of a round of mts_per_round tiles) and 64 of the
-// 128 columns (col_off bytes): acc[16 x 64] = mask[16 x rows] . rows[rows x 64].  The scaled,
-// rounded cores overwrite rows [0, P) of the same area: cluster c only reads rows >= its seed
-// >= c, rounds go up in c, and inside a round every warp has finished reading before any writes.
-__device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_ptr, int col_off, int mt_in_round,
-                                             int mts_per_round, int P, const uint16_t* seedrow, const uint16_t* send,
-                                             const uint32_t* adj, int lane, bool write_counts) {
+// Stages rows [0, R) of one tensor (row r at src + r*stride elements) at `dst`, pitch kPitch, and
+// zero-fills up to the next multiple of 16 rows (those rows enter the Eq. 3 product with weight 0).
+__device__ __forceinline__ void stage_rows(uint32_t dst, const __nv_bfloat16* src, int64_t stride, int R, int tid) {
+    const int c = tid & 15, r0 = tid >> 4;
+    const char* s = reinterpret_cast<const char*>(src + (int64_t)r0 * stride) + c * 16;
+    uint32_t d = dst + r0 * kPitch + c * 16;
+    const int64_t s_step = stride * (2 * (kThreads / 16));
+    for (int r = r0; r < R; r += kThreads / 16) {
+        cp_async16(d, s, 16);
+        s += s_step;
+        d += (kThreads / 16) * kPitch;
+    }
+    const int r = R + r0;   // at most 15 rows of padding
+    if (r < ((R + 15) & ~15)) cp_async16(dst + r * kPitch + c * 16, src, 0);
+}
+
+// Eq. 3 on the tensor cores for one staged tensor (K or V rows at `area`, pitch kPitch), run by the
+// four warps kMergeWarp0..+3.  Cluster c (in seed order) has its member mask in the adjacency row
+// of its seed seedrow[c].  A warp owns one tile of 16 clusters (mt_in_round of a round of
+// mts_per_round tiles) and does the 128 columns in two halves:
+//     acc[16 x 64] = mask[16 x rows] . rows[rows x 64].
+// The scaled, rounded cores overwrite rows [0, P) of the same area: cluster c only reads rows >=
+// its seed >= c, rounds go up in c, and inside a half every warp has finished reading before any
+// of them writes.  The 16-byte pad of row c receives the cluster's member count.
+__device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_ptr, int mt_in_round, int mts_per_round,
+                                             int P, const uint16_t* seedrow, const uint16_t* send, const uint32_t* adj,
+                                             int lane, bool write_counts) {
     const int g = lane >> 2, tig = lane & 3;
-    const uint32_t b_lane = area + ((lane & 7) + ((lane >> 3) & 1) * 8) * kPitch + col_off + (lane >> 4) * 16;
+    const uint32_t b_lane = area + ((lane & 7) + ((lane >> 3) & 1) * 8) * kPitch + (lane >> 4) * 16;
     for (int c0 = 0; c0 < P; c0 += 16 * mts_per_round) {
         const int cbase = c0 + 16 * mt_in_round;
         const bool active = cbase < P;
-        float acc[8][4];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-        int cnt0 = 0, cnt1 = 0;
+        const bool ok_lo = cbase + g < P, ok_hi = cbase + g + 8 < P;
+        int lo0 = 0, hi0 = -2, lo1 = 0, hi1 = -2, w_first = 0, w_last = -1;
+        const uint32_t* r0 = adj;
+        const uint32_t* r1 = adj;
         if (active) {
-            const int c_lo = cbase + g, c_hi = cbase + g + 8;
-            const int i0 = c_lo < P ? (int)seedrow[c_lo] : -1, i1 = c_hi < P ? (int)seedrow[c_hi] : -1;
-            const int lo0 = i0 >> 5, hi0 = i0 >= 0 ? ((int)send[i0] - 1) >> 5 : -2;   // word range of the masks
-            const int lo1 = i1 >> 5, hi1 = i1 >= 0 ? ((int)send[i1] - 1) >> 5 : -2;
-            const uint32_t* r0 = adj + (i0 >= 0 ? adj_row(i0) - lo0 : 0);
-            const uint32_t* r1 = adj + (i1 >= 0 ? adj_row(i1) - lo1 : 0);
-            const int w_first = (int)seedrow[cbase] >> 5;
-            const int w_last = ((int)send[seedrow[min(cbase + 15, P - 1)]] - 1) >> 5;
+            if (ok_lo) { const int i0 = seedrow[cbase + g]; lo0 = i0 >> 5; hi0 = ((int)send[i0] - 1) >> 5; r0 = adj + adj_row(i0) - lo0; }
+            if (ok_hi) { const int i1 = seedrow[cbase + g + 8]; lo1 = i1 >> 5; hi1 = ((int)send[i1] - 1) >> 5; r1 = adj + adj_row(i1) - lo1; }
+            w_first = (int)seedrow[cbase] >> 5;
+            w_last = ((int)send[seedrow[min(cbase + 15, P - 1)]] - 1) >> 5;
+        }
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+            float acc[8][4];
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+            int cnt0 = 0, cnt1 = 0;
             for (int w = w_first; w <= w_last; ++w) {
                 const uint32_t m0w = (w >= lo0 && w <= hi0) ? r0[w] : 0u;
                 const uint32_t m1w = (w >= lo1 && w <= hi1) ? r1[w] : 0u;
@@ -321,11 +319,11 @@ __device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_
                 cnt1 += __popc(m1w);
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
-                    const uint32_t m0 = (m0w >> (16 * hh)) & 0xffffu, m1 = (m1w >> (16 * hh)) & 0xffffu;
-                    if (!__any_sync(kFull, (m0 | m1) != 0u)) continue;
-                    const uint32_t a0 = expand2((m0 >> (2 * tig)) & 3u), a2 = expand2((m0 >> (2 * tig + 8)) & 3u);
-                    const uint32_t a1 = expand2((m1 >> (2 * tig)) & 3u), a3 = expand2((m1 >> (2 * tig + 8)) & 3u);
-                    const uint32_t b_addr = b_lane + (w * 32 + hh * 16) * kPitch;
+                    const uint32_t m0 = (m0w >> (16 * hh + 2 * tig)), m1 = (m1w >> (16 * hh + 2 * tig));
+                    if (!__any_sync(kFull, ((m0 | m1) & 0x0303u) != 0u)) continue;
+                    const uint32_t a0 = expand2(m0 & 3u), a2 = expand2((m0 >> 8) & 3u);
+                    const uint32_t a1 = expand2(m1 & 3u), a3 = expand2((m1 >> 8) & 3u);
+                    const uint32_t b_addr = b_lane + (w * 32 + hh * 16) * kPitch + half * 128;
 #pragma unroll
                     for (int np = 0; np < 4; ++np) {
                         uint32_t b0, b1, b2, b3;
@@ -335,23 +333,20 @@ __device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_
                     }
                 }
             }
-        }
-        __syncthreads();   // every warp has read what it needs of rows [c0, ...)
-        if (active) {
-            const float inv0 = 1.0f / (float)max(cnt0, 1), inv1 = 1.0f / (float)max(cnt1, 1);
-            unsigned char* o_lo = area_ptr + (cbase + g) * kPitch + col_off + tig * 4;
-            unsigned char* o_hi = o_lo + 8 * kPitch;
-            const bool ok_lo = cbase + g < P, ok_hi = cbase + g + 8 < P;
+            merge_warps_sync();   // every merging warp has read what it needs of these columns
+            if (active) {
+                const float inv0 = 1.0f / (float)max(cnt0, 1), inv1 = 1.0f / (float)max(cnt1, 1);
+                unsigned char* o_lo = area_ptr + (cbase + g) * kPitch + half * 128 + tig * 4;
+                unsigned char* o_hi = o_lo + 8 * kPitch;
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(acc[nt][0] * inv0, acc[nt][1] * inv0);
-                __nv_bfloat162 hi = __floats2bfloat162_rn(acc[nt][2] * inv1, acc[nt][3] * inv1);
-                if (ok_lo) *reinterpret_cast<__nv_bfloat162*>(o_lo + nt * 16) = lo;
-                if (ok_hi) *reinterpret_cast<__nv_bfloat162*>(o_hi + nt * 16) = hi;
-            }
-            if (write_counts && tig == 0) {   // the row's 16-byte pad carries its member count
-                if (ok_lo) *reinterpret_cast<int*>(area_ptr + (cbase + g) * kPitch + kRowBytes) = cnt0;
-                if (ok_hi) *reinterpret_cast<int*>(area_ptr + (cbase + g + 8) * kPitch + kRowBytes) = cnt1;
+                for (int nt = 0; nt < 8; ++nt) {
+                    if (ok_lo) *reinterpret_cast<__nv_bfloat162*>(o_lo + nt * 16) = __floats2bfloat162_rn(acc[nt][0] * inv0, acc[nt][1] * inv0);
+                    if (ok_hi) *reinterpret_cast<__nv_bfloat162*>(o_hi + nt * 16) = __floats2bfloat162_rn(acc[nt][2] * inv1, acc[nt][3] * inv1);
+                }
+                if (write_counts && half == 0 && tig == 0) {
+                    if (ok_lo) *reinterpret_cast<int*>(area_ptr + (cbase + g) * kPitch + kRowBytes) = cnt0;
+                    if (ok_hi) *reinterpret_cast<int*>(area_ptr + (cbase + g + 8) * kPitch + kRowBytes) = cnt1;
+                }
             }
         }
     }
@@ -369,24 +364,15 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
     int* geo_buf = reinterpret_cast<int*>(smem + kMiscOff + 32);        // [2][8]
     int* misc = reinterpret_cast<int*>(smem + kMiscOff + 96);           // [0] output offset of the tile, [1] last block
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar_k = sbase + kBarOff, bar_v = sbase + kBarOff + 8;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int rwarp = kWarps - 1 - warp;   // work is dealt from the last warp down: warp 0 also scouts ahead
+    const int rwarp = kWarps - 1 - warp;   // per-tile work is dealt from the last warp down
     int dec_b = 0, dec_pref = 0;           // ticket decoding state (warp 0)
 
-    if (tid == 0) {
-        mbar_init(bar_k, 1);
-        mbar_init(bar_v, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
-    }
-    if (warp == 0) fetch_tile<kMode>(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
-    fence_async_proxy();
+    if (warp == 0) fetch_tile(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
     __syncthreads();
 
-    uint32_t phase_k = 0, phase_v = 0;
     int buf = 0;
-    bool failed = false;
 #ifdef SC_PHASE_TIMING
     long long t_prev = clock64();
 #endif
@@ -402,47 +388,33 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         const int nrb = (R + 31) >> 5;
         const int64_t goff = b * p.st.b + h * p.st.h + (int64_t)row0 * p.st.n;
 
-        // ---- 1. stage the rows ----
-        if (tid == 0) {
-            mbar_expect_tx(bar_k, (uint32_t)R * kRowBytes);
-            if (two_tensors) mbar_expect_tx(bar_v, (uint32_t)R * kRowBytes);
-        }
-        if (long_tile) {
-            if (tid < R) bulk_g2s(sbase + tid * kPitch, p.K + goff + (int64_t)tid * p.st.n, kRowBytes, bar_k);
-        } else if (tid < kShortRows) {
-            if (tid < R) bulk_g2s(sbase + tid * kPitch, p.K + goff + (int64_t)tid * p.st.n, kRowBytes, bar_k);
-        } else if (two_tensors) {
-            const int r = tid - kShortRows;
-            if (r < R) bulk_g2s(sbase + kVOff + r * kPitch, p.V + goff + (int64_t)r * p.st.n, kRowBytes, bar_v);
-        }
-        {   // rows [R, next multiple of 16) take part in the Eq. 3 product with zero weight: keep them finite
-            const int pad_chunks = (((R + 15) & ~15) - R) * 16;
-            for (int i = tid; i < pad_chunks; i += kThreads) {
-                unsigned char* dst = smem + (R + (i >> 4)) * kPitch + (i & 15) * 16;
-                *reinterpret_cast<uint4*>(dst) = make_uint4(0, 0, 0, 0);
-                if (two_tensors) *reinterpret_cast<uint4*>(dst + kVOff) = make_uint4(0, 0, 0, 0);
+        // ---- 1. stage the rows; prefetch ahead ----
+        stage_rows(sbase, p.K + goff, p.st.n, R, tid);
+        cp_async_commit();
+        if (two_tensors) stage_rows(sbase + kVOff, p.V + goff, p.st.n, R, tid);
+        cp_async_commit();
+        if (p.ahead_rows > 0 && tid == 64) {   // contiguous cache: tickets advance in memory order
+            const int64_t first = (int64_t)bh * p.n + row0 + p.ahead_rows;
+            const int64_t rows = min((int64_t)R, p.total_rows - first);
+            if (rows > 0) {
+                l2_prefetch(p.K + first * kD, (uint32_t)rows * kRowBytes);
+                if (kMode != kCountOnly) l2_prefetch(p.V + first * kD, (uint32_t)rows * kRowBytes);
             }
         }
-        CF_T(0);
-
-        // ---- scout: next ticket, its geometry, L2 prefetch (warp 0); segment bookkeeping (others) ----
-        if (warp == 0) {
-            fetch_tile<kMode>(p, lane, dec_b, dec_pref, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
+        // end of the segment each row is in (0 past the tile)
+        if (tid < kNW) seedmask[tid] = 0u;
+        if (nseg == 1) {
+            for (int r = tid; r < R; r += kThreads) send[r] = (uint16_t)R;
         } else {
-            if (tid - 32 < kNW) seedmask[tid - 32] = 0u;
-            for (int r = tid - 32; r < nrb * 32; r += kThreads - 32) {   // end of the segment each row is in
-                int lo = 0, hi = nseg;                                    // segs[lo] <= r < segs[hi]
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (segs[mid] <= r) lo = mid; else hi = mid;
-                }
-                send[r] = (r < R) ? (uint16_t)segs[lo + 1] : (uint16_t)0;
+            for (int s = tid; s < nseg; s += kThreads) {
+                const int a = segs[s], e = segs[s + 1];
+                for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
             }
         }
-        CF_T(1);
-        failed = !mbar_wait(bar_k, phase_k);
-        phase_k ^= 1u;
-        if (__syncthreads_or(failed)) { failed = true; break; }
+        for (int r = R + tid; r < nrb * 32; r += kThreads) send[r] = (uint16_t)0;
+        CF_T(0);
+        cp_async_wait<1>();   // this thread's K copies; the barrier publishes everyone's
+        __syncthreads();
         CF_T(2);
 
         // ---- 2. Gram blocks -> norms -> adjacency bits ----
@@ -450,14 +422,14 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
             float acc[2][4][4];
             const bool have = rwarp < nrb;
             if (have) {
-                gram_block(sbase, rwarp, rwarp, lane, acc);
+                gram_block<true>(sbase, rwarp, rwarp, lane, acc);
                 store_norms(acc, rwarp, lane, norm);
             }
             __syncthreads();
             CF_T(3);
             if (have) {
-                if (p.tau < 0.f) threshold_block<true>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
-                else threshold_block<false>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
+                if (p.tau < 0.f) threshold_block<true, true>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
+                else threshold_block<false, true>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
             }
             if (nrb > 1) {
                 for (int k = rwarp; k < 28; k += kWarps) {
@@ -465,9 +437,9 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                     if (cb >= nrb) continue;
                     const int reach = ((int)send[min(rb * 32 + 31, R - 1)] - 1) >> 5;   // last block a segment of rb spans
                     if (cb > reach) continue;
-                    gram_block(sbase, rb, cb, lane, acc);
-                    if (p.tau < 0.f) threshold_block<true>(acc, rb, cb, lane, p.tau, norm, send, adj);
-                    else threshold_block<false>(acc, rb, cb, lane, p.tau, norm, send, adj);
+                    gram_block<false>(sbase, rb, cb, lane, acc);
+                    if (p.tau < 0.f) threshold_block<true, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
+                    else threshold_block<false, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
                 }
             }
         }
@@ -516,8 +488,11 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
 #pragma unroll
         for (int w = 0; w < kNW; ++w) P += __popc(seedmask[w]);
         uint32_t* stt = p.tile_state + (size_t)bh * p.n_tile_cap;
+        int16_t* segs_next = segs_buf + (buf ^ 1) * kSegsStride;
+        int* geo_next = geo_buf + (buf ^ 1) * 8;
         if (kMode == kCountOnly) {
             if (tid == 0) stt[t] = (uint32_t)P;
+            if (warp == 0) fetch_tile(p, lane, dec_b, dec_pref, geo_next, segs_next);
         } else {
             if (kMode == kLookBack && tid == 0)
                 atomicExch(&stt[t], (t == 0 ? kFlagPrefix : kFlagAggregate) | (uint32_t)P);
@@ -529,23 +504,19 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                     seedrow[rank] = (uint16_t)tid;
                 }
             }
-            if (two_tensors) {
-                failed = !mbar_wait(bar_v, phase_v);
-                phase_v ^= 1u;
-            }
-            if (__syncthreads_or(failed)) { failed = true; break; }
+            cp_async_wait<0>();   // V
+            __syncthreads();
             CF_T(6);
 
-            // ---- 5. Eq. 3 (K, and V when it is staged) ----
-            if (long_tile)
-                merge_rounds(sbase, smem, (warp & 1) * 128, warp >> 1, 4, P, seedrow, send, adj, lane, (warp & 1) == 0);
-            else
-                merge_rounds(sbase + ((warp >> 1) & 1) * kVOff, smem + ((warp >> 1) & 1) * kVOff, (warp & 1) * 128,
-                             warp >> 2, 2, P, seedrow, send, adj, lane, (warp & 3) == 0);
-            CF_T(7);
-
-            // ---- output offset of the tile (warp 0) ----
-            if (warp == 0) {
+            // ---- 5. warps 4-7: Eq. 3; warp 0: next ticket; warp 1: output offset of the tile ----
+            if (warp >= kMergeWarp0) {
+                const int mw = warp - kMergeWarp0;
+                if (long_tile) merge_rounds(sbase, smem, mw, 4, P, seedrow, send, adj, lane, true);
+                else merge_rounds(sbase + (mw & 1) * kVOff, smem + (mw & 1) * kVOff, mw >> 1, 2, P, seedrow, send, adj, lane,
+                                  (mw & 1) == 0);
+            } else if (warp == 0) {
+                fetch_tile(p, lane, dec_b, dec_pref, geo_next, segs_next);
+            } else if (warp == 1) {
                 int base = 0;
                 if (kMode == kWriteWithCounts) {
                     for (int k = lane; k < t; k += 32) base += (int)stt[k];
@@ -607,14 +578,12 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
 
             // ---- a long segment: V takes the place of K and goes through the same product ----
             if (long_tile) {
-                fence_async_proxy();
                 __syncthreads();
-                if (tid == 0) mbar_expect_tx(bar_v, (uint32_t)R * kRowBytes);
-                if (tid < R) bulk_g2s(sbase + tid * kPitch, p.V + goff + (int64_t)tid * p.st.n, kRowBytes, bar_v);
-                failed = !mbar_wait(bar_v, phase_v);
-                phase_v ^= 1u;
-                if (__syncthreads_or(failed)) { failed = true; break; }
-                merge_rounds(sbase, smem, (warp & 1) * 128, warp >> 1, 4, P, seedrow, send, adj, lane, false);
+                stage_rows(sbase, p.V + goff, p.st.n, R, tid);
+                cp_async_commit();
+                cp_async_wait<0>();
+                __syncthreads();
+                if (warp >= kMergeWarp0) merge_rounds(sbase, smem, warp - kMergeWarp0, 4, P, seedrow, send, adj, lane, false);
                 __syncthreads();
                 for (int idx = tid; idx < P * 16; idx += kThreads) {
                     const int row = idx >> 4, c = idx & 15;
@@ -624,20 +593,12 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                 }
             }
         }
-
-        // the next tile's bulk copies overwrite what this one read and wrote through ordinary accesses
-        fence_async_proxy();
-        __syncthreads();
+        __syncthreads();   // the next tile's copies overwrite what this one read and wrote
         CF_T(9);
         buf ^= 1;
     }
 
     // ---- exit: the last block to finish leaves the workspace zeroed for the next call ----
-    if (failed) {
-        if (tid == 0) set_status(p.status, SC_ERR_TIMEOUT);
-        mbar_wait(bar_k, phase_k ^ 1u);   // bounded: let copies that may still be in flight land before leaving
-        mbar_wait(bar_v, phase_v ^ 1u);
-    }
     __syncthreads();
     if (tid == 0) {
         __threadfence();
@@ -696,6 +657,10 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
     // no more blocks than there can be tiles
     const int64_t max_tiles = (int64_t)a.B * a.Hkv * a.n_tile_cap;
     const int grid = (int)(max_tiles < grid_of[dev] ? max_tiles : grid_of[dev]);
+    // prefetch distance: the rows all resident blocks hold together
+    const bool contiguous = a.st.n == cf::kD && a.st.h == (int64_t)a.n * cf::kD && a.st.b == (int64_t)a.Hkv * a.n * cf::kD;
+    p.ahead_rows = contiguous ? grid * SC_TILE_ROWS : 0;
+    p.total_rows = (int64_t)a.B * a.Hkv * a.n;
     if (a.flags & SC_FLAG_TWO_PASS) {
         cf::Params pc = p;
         pc.assign = nullptr;
