@@ -49,7 +49,7 @@ constexpr int kSendOff = kNormOff + kMaxRows * 4; // uint16[256]: end of the seg
 constexpr int kSegsOff = kSendOff + kMaxRows * 2; // 2 x int16[132]: segment starts (this tile, next tile)
 constexpr int kSegsStride = 132;
 constexpr int kMiscOff = kSegsOff + 2 * kSegsStride * 2;   // uint32 seedmask[8]; int geo[2][8]; int misc[4]
-constexpr int kSmemBytes = kMiscOff + 32 + 64 + 16;
+constexpr int kSmemBytes = kMiscOff + 32 + 64 + 16 + 32;   // ... int reach[8]
 static_assert(kSmemBytes <= 76800, "three blocks per SM need <= 75 KB each");
 
 enum Mode { kCountOnly = 0, kWriteWithCounts = 1, kLookBack = 2 };
@@ -215,6 +215,129 @@ __device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int
 __constant__ uint8_t kOffDiag[28] = {0x01, 0x12, 0x23, 0x34, 0x45, 0x56, 0x67, 0x02, 0x13, 0x24, 0x35, 0x46, 0x57, 0x03,
                                      0x14, 0x25, 0x36, 0x47, 0x04, 0x15, 0x26, 0x37, 0x05, 0x16, 0x27, 0x06, 0x17, 0x07};
 
+// Eq. 2 + Algorithm 1 for one segment of 2..32 tokens, by one warp, in registers.
+// Rows [a, a + l) of the staged keys.  The upper triangle of the segment's own Gram matrix comes
+// from mma tiles laid over the segment's rows (16-row tiles down, 8-column tiles across, only
+// those that reach above the diagonal); lane 4g + t ends up owning row g + 8t with its adjacency
+// bits (later tokens only) in one word, and the greedy pass is a handful of word operations and
+// one shuffle per seed.  Results: seed bits into the tile's seedmask, each seed's member mask into
+// its (tile-relative) adjacency row for the Eq. 3 product, optionally the seed of every token.
+template <bool kNegTau>
+__device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int a, int l, float tau, float* nrm /*[32], this warp's*/,
+                                                  uint32_t* adj, uint32_t* seedmask, int32_t* as, int row0, int lane) {
+    const int g = lane >> 2, tig = lane & 3;
+    const int nnt = (l + 7) >> 3;          // 8-column tiles that hold tokens: 1..4
+    const bool two_mt = l > 16;
+    float acc[2][4][4];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = acc[mt][nt][2] = acc[mt][nt][3] = 0.f;
+    {
+        const int j = lane >> 3, r8 = lane & 7;
+        const uint32_t a_addr = kbase + (a + r8 + ((j & 1) << 3)) * kPitch + ((j >> 1) << 4);
+        const uint32_t b_addr = kbase + (a + r8 + ((j >> 1) << 3)) * kPitch + ((j & 1) << 4);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t a0[4], a1[4], b0[4], b1[4];
+            ldmatrix_x4(a_addr + ks * 32, a0[0], a0[1], a0[2], a0[3]);
+            ldmatrix_x4(b_addr + ks * 32, b0[0], b0[1], b0[2], b0[3]);
+            mma_bf16(acc[0][0], a0[0], a0[1], a0[2], a0[3], b0[0], b0[1]);
+            if (nnt > 1) mma_bf16(acc[0][1], a0[0], a0[1], a0[2], a0[3], b0[2], b0[3]);
+            if (two_mt) {
+                ldmatrix_x4(a_addr + 16 * kPitch + ks * 32, a1[0], a1[1], a1[2], a1[3]);
+                ldmatrix_x4(b_addr + 16 * kPitch + ks * 32, b1[0], b1[1], b1[2], b1[3]);
+                mma_bf16(acc[0][2], a0[0], a0[1], a0[2], a0[3], b1[0], b1[1]);
+                mma_bf16(acc[1][2], a1[0], a1[1], a1[2], a1[3], b1[0], b1[1]);
+                if (nnt > 3) {
+                    mma_bf16(acc[0][3], a0[0], a0[1], a0[2], a0[3], b1[2], b1[3]);
+                    mma_bf16(acc[1][3], a1[0], a1[1], a1[2], a1[3], b1[2], b1[3]);
+                }
+            }
+        }
+    }
+    // norms from the diagonal
+    if ((g >> 1) == tig) {
+        const int e = g & 1;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+                nrm[mt * 16 + hh * 8 + g] = sqrtf(e ? acc[mt][2 * mt + hh][hh * 2 + 1] : acc[mt][2 * mt + hh][hh * 2]);
+    }
+    __syncwarp();
+    float tn[4][2];
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+        const float2 nn = *reinterpret_cast<const float2*>(nrm + nt * 8 + 2 * tig);
+        tn[nt][0] = tau * nn.x;
+        tn[nt][1] = tau * nn.y;
+    }
+    uint32_t wrow[2][2];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            uint32_t w = 0;
+            if (mt == 0 || two_mt) {
+                const float ni = nrm[mt * 16 + hh * 8 + g];
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) {
+                    if (nt < 2 * mt + hh) continue;   // columns before the row's own
+                    if (nt < nnt) {
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const float thr = ni * tn[nt][e];
+                            bool hit = acc[mt][nt][hh * 2 + e] > thr;
+                            if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
+                            if (hit) w |= 1u << (nt * 8 + e);
+                        }
+                    }
+                }
+                w <<= 2 * tig;
+                w |= __shfl_xor_sync(kFull, w, 1);
+                w |= __shfl_xor_sync(kFull, w, 2);
+            }
+            wrow[mt][hh] = w;
+        }
+    __syncwarp();   // the norms are spent: the next segment of this warp may overwrite them
+    // lane 4g + t owns token g + 8t
+    const int own = g + 8 * tig;
+    const uint32_t lowmask = l >= 32 ? 0xffffffffu : ((1u << l) - 1u);
+    uint32_t mine = (tig & 2) ? ((tig & 1) ? wrow[1][1] : wrow[1][0]) : ((tig & 1) ? wrow[0][1] : wrow[0][0]);
+    mine &= (0xfffffffeu << own) & lowmask;   // later tokens of the segment only
+    // Algorithm 1
+    uint32_t U = lowmask, seeds = 0u, mymem = 0u;
+    int seed_of = 0;
+    while (U) {
+        const int i = __ffs(U) - 1;                      // lowest unassigned token: a seed
+        const int src = ((i & 7) << 2) | (i >> 3);
+        const uint32_t mem = (__shfl_sync(kFull, mine, src) & U) | (1u << i);
+        U &= ~mem;
+        if ((mem >> own) & 1u) seed_of = i;
+        if (lane == src) mymem = mem;
+        seeds |= 1u << i;
+    }
+    // hand the result to the tile
+    const int sh = a & 31, w0 = a >> 5;
+    if (lane == 0) {
+        atomicOr(&seedmask[w0], seeds << sh);
+        if (sh != 0 && (seeds >> (32 - sh)) != 0u) atomicOr(&seedmask[w0 + 1], seeds >> (32 - sh));
+    }
+    if (mymem != 0u) {
+        const int i = a + own;
+        const uint32_t lo = mymem << sh, hi = sh ? (mymem >> (32 - sh)) : 0u;
+        uint32_t* row = adj + adj_row(i);
+        if ((i >> 5) == w0) {
+            row[0] = lo;
+            if (((a + l - 1) >> 5) > w0) row[1] = hi;
+        } else {
+            row[0] = hi;
+        }
+    }
+    if (as != nullptr && own < l) as[a + own] = row0 + a + seed_of;
+}
+
 struct Params {
     const __nv_bfloat16* K; const __nv_bfloat16* V; sc_strides st;
     int B, Hkv, n;
@@ -362,7 +485,9 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
     int16_t* segs_buf = reinterpret_cast<int16_t*>(smem + kSegsOff);
     uint32_t* seedmask = reinterpret_cast<uint32_t*>(smem + kMiscOff);
     int* geo_buf = reinterpret_cast<int*>(smem + kMiscOff + 32);        // [2][8]
-    int* misc = reinterpret_cast<int*>(smem + kMiscOff + 96);           // [0] output offset of the tile, [1] last block
+    int* misc = reinterpret_cast<int*>(smem + kMiscOff + 96);           // [0] output offset of the tile, [1] last block,
+                                                                        // [2] 32-row blocks that a segment of > 32 tokens touches
+    int* reach = reinterpret_cast<int*>(smem + kMiscOff + 112);         // [8] last block such a segment spans from block k
     const uint32_t sbase = smem_u32(smem);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -370,6 +495,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
     int dec_b = 0, dec_pref = 0;           // ticket decoding state (warp 0)
 
     if (warp == 0) fetch_tile(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
+    if (tid < kNW) reach[tid] = 0;
+    if (tid == kNW) misc[2] = 0;
     __syncthreads();
 
     int buf = 0;
@@ -405,10 +532,13 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         if (tid < kNW) seedmask[tid] = 0u;
         if (nseg == 1) {
             for (int r = tid; r < R; r += kThreads) send[r] = (uint16_t)R;
+            if (R > 32 && tid < nrb) { atomicOr(&misc[2], 1 << tid); reach[tid] = nrb - 1; }
         } else {
             for (int s = tid; s < nseg; s += kThreads) {
                 const int a = segs[s], e = segs[s + 1];
                 for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
+                if (e - a > 32)
+                    for (int k = a >> 5; k <= (e - 1) >> 5; ++k) { atomicOr(&misc[2], 1 << k); atomicMax(&reach[k], (e - 1) >> 5); }
             }
         }
         for (int r = R + tid; r < nrb * 32; r += kThreads) send[r] = (uint16_t)0;
@@ -417,36 +547,32 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         __syncthreads();
         CF_T(2);
 
-        // ---- 2. Gram blocks -> norms -> adjacency bits ----
-        {
+        // ---- 2. segments of more than 32 tokens: Gram blocks -> norms -> adjacency bits in shared memory ----
+        const int longblocks = misc[2];
+        if (longblocks != 0) {
             float acc[2][4][4];
-            const bool have = rwarp < nrb;
+            const bool have = rwarp < nrb && ((longblocks >> rwarp) & 1);
             if (have) {
                 gram_block<true>(sbase, rwarp, rwarp, lane, acc);
                 store_norms(acc, rwarp, lane, norm);
             }
             __syncthreads();
-            CF_T(3);
             if (have) {
                 if (p.tau < 0.f) threshold_block<true, true>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
                 else threshold_block<false, true>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
             }
-            if (nrb > 1) {
-                for (int k = rwarp; k < 28; k += kWarps) {
-                    const int rb = kOffDiag[k] >> 4, cb = kOffDiag[k] & 15;
-                    if (cb >= nrb) continue;
-                    const int reach = ((int)send[min(rb * 32 + 31, R - 1)] - 1) >> 5;   // last block a segment of rb spans
-                    if (cb > reach) continue;
-                    gram_block<false>(sbase, rb, cb, lane, acc);
-                    if (p.tau < 0.f) threshold_block<true, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
-                    else threshold_block<false, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
-                }
+            for (int k = rwarp; k < 28; k += kWarps) {
+                const int rb = kOffDiag[k] >> 4, cb = kOffDiag[k] & 15;
+                if (cb >= nrb || !((longblocks >> rb) & 1) || cb > reach[rb]) continue;
+                gram_block<false>(sbase, rb, cb, lane, acc);
+                if (p.tau < 0.f) threshold_block<true, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
+                else threshold_block<false, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
             }
+            __syncthreads();
         }
-        __syncthreads();
         CF_T(4);
 
-        // ---- 3. Algorithm 1 per segment: one warp per segment, lane c owns word c ----
+        // ---- 3. Algorithm 1 per segment, one warp each: in registers up to 32 tokens, else on the bit rows ----
         int32_t* as = p.assign ? p.assign + (size_t)bh * p.n + row0 : nullptr;
         for (int s = rwarp; s < nseg; s += kWarps) {
             const int a = segs[s], e = segs[s + 1];
@@ -456,6 +582,11 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                     atomicOr(&seedmask[a >> 5], 1u << (a & 31));
                     if (as) as[a] = row0 + a;
                 }
+                continue;
+            }
+            if (e - a <= 32) {
+                if (p.tau < 0.f) gsc_short_segment<true>(sbase, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
+                else gsc_short_segment<false>(sbase, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
                 continue;
             }
             const int w1 = (e - 1) >> 5;
@@ -593,6 +724,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                 }
             }
         }
+        if (tid < kNW) reach[tid] = 0;
+        if (tid == kNW) misc[2] = 0;
         __syncthreads();   // the next tile's copies overwrite what this one read and wrote
         CF_T(9);
         buf ^= 1;
