@@ -49,7 +49,7 @@ constexpr int kSendOff = kNormOff + kMaxRows * 4; // uint16[256]: end of the seg
 constexpr int kSegsOff = kSendOff + kMaxRows * 2; // 2 x int16[132]: segment starts (this tile, next tile)
 constexpr int kSegsStride = 132;
 constexpr int kMiscOff = kSegsOff + 2 * kSegsStride * 2;   // uint32 seedmask[8]; int geo[2][8]; int misc[4]
-constexpr int kSmemBytes = kMiscOff + 32 + 64 + 16 + 32;   // ... int reach[8]
+constexpr int kSmemBytes = kMiscOff + 32 + 64 + 16 + 32 + 128;   // ... int reach[8]; uint8 multi[128]
 static_assert(kSmemBytes <= 76800, "three blocks per SM need <= 75 KB each");
 
 enum Mode { kCountOnly = 0, kWriteWithCounts = 1, kLookBack = 2 };
@@ -72,7 +72,6 @@ __device__ unsigned long long g_phase_cycles[16];
 
 constexpr uint32_t kFlagAggregate = 1u << 30, kFlagPrefix = 2u << 30, kValueMask = (1u << 30) - 1;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // the look-back gives up after 2 s
-constexpr int kMergeWarp0 = 4;                               // warps 4..7 run the Eq. 3 product
 constexpr int kCtlWords = 64;                                // ticket, done counter, padding
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -88,9 +87,6 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int sr
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void merge_warps_sync() {   // the four warps of the Eq. 3 product
-    asm volatile("bar.sync 1, 128;\n" ::: "memory");
-}
 __device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
 }
@@ -207,7 +203,9 @@ __device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int
             w <<= 2 * tig;
             w |= __shfl_xor_sync(kFull, w, 1);
             w |= __shfl_xor_sync(kFull, w, 2);
-            if (tig == 0) adj[adj_row(i) + (cb - rb)] = w & bits_between(i + 1, (int)send[i], cb);
+            // (a token with no later token in its segment keeps its word: a one-token segment's is already final)
+            const int e_i = (int)send[i];
+            if (tig == 0 && e_i > i + 1) adj[adj_row(i) + (cb - rb)] = w & bits_between(i + 1, e_i, cb);
         }
 }
 
@@ -403,38 +401,34 @@ __device__ __forceinline__ void stage_rows(uint32_t dst, const __nv_bfloat16* sr
     if (r < ((R + 15) & ~15)) cp_async16(dst + r * kPitch + c * 16, src, 0);
 }
 
-// Eq. 3 on the tensor cores for one staged tensor (K or V rows at `area`, pitch kPitch), run by the
-// four warps kMergeWarp0..+3.  Cluster c (in seed order) has its member mask in the adjacency row
-// of its seed seedrow[c].  A warp owns one tile of 16 clusters (mt_in_round of a round of
-// mts_per_round tiles) and does the 128 columns in two halves:
-//     acc[16 x 64] = mask[16 x rows] . rows[rows x 64].
+// Eq. 3 on the tensor cores for one staged tensor (K or V rows at `area`, pitch kPitch).
+// Cluster c (in seed order) has its member mask in the adjacency row of its seed seedrow[c].  A
+// warp owns one tile of 16 clusters (mt_in_round of a round of mts_per_round tiles) and one half
+// of the 128 columns:  acc[16 x 64] = mask[16 x rows] . rows[rows x 64].
 // The scaled, rounded cores overwrite rows [0, P) of the same area: cluster c only reads rows >=
-// its seed >= c, rounds go up in c, and inside a half every warp has finished reading before any
+// its seed >= c, rounds go up in c, and inside a round every warp has finished reading before any
 // of them writes.  The 16-byte pad of row c receives the cluster's member count.
-__device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_ptr, int mt_in_round, int mts_per_round,
-                                             int P, const uint16_t* seedrow, const uint16_t* send, const uint32_t* adj,
-                                             int lane, bool write_counts) {
+__device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_ptr, int half, int mt_in_round,
+                                             int mts_per_round, int P, const uint16_t* seedrow, const uint16_t* send,
+                                             const uint32_t* adj, int lane, bool write_counts) {
     const int g = lane >> 2, tig = lane & 3;
-    const uint32_t b_lane = area + ((lane & 7) + ((lane >> 3) & 1) * 8) * kPitch + (lane >> 4) * 16;
+    const uint32_t b_lane = area + ((lane & 7) + ((lane >> 3) & 1) * 8) * kPitch + (lane >> 4) * 16 + half * 128;
     for (int c0 = 0; c0 < P; c0 += 16 * mts_per_round) {
         const int cbase = c0 + 16 * mt_in_round;
         const bool active = cbase < P;
         const bool ok_lo = cbase + g < P, ok_hi = cbase + g + 8 < P;
-        int lo0 = 0, hi0 = -2, lo1 = 0, hi1 = -2, w_first = 0, w_last = -1;
-        const uint32_t* r0 = adj;
-        const uint32_t* r1 = adj;
+        float acc[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+        int cnt0 = 0, cnt1 = 0;
         if (active) {
+            int lo0 = 0, hi0 = -2, lo1 = 0, hi1 = -2;
+            const uint32_t* r0 = adj;
+            const uint32_t* r1 = adj;
             if (ok_lo) { const int i0 = seedrow[cbase + g]; lo0 = i0 >> 5; hi0 = ((int)send[i0] - 1) >> 5; r0 = adj + adj_row(i0) - lo0; }
             if (ok_hi) { const int i1 = seedrow[cbase + g + 8]; lo1 = i1 >> 5; hi1 = ((int)send[i1] - 1) >> 5; r1 = adj + adj_row(i1) - lo1; }
-            w_first = (int)seedrow[cbase] >> 5;
-            w_last = ((int)send[seedrow[min(cbase + 15, P - 1)]] - 1) >> 5;
-        }
-#pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-            float acc[8][4];
-#pragma unroll
-            for (int nt = 0; nt < 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-            int cnt0 = 0, cnt1 = 0;
+            const int w_first = (int)seedrow[cbase] >> 5;
+            const int w_last = ((int)send[seedrow[min(cbase + 15, P - 1)]] - 1) >> 5;
             for (int w = w_first; w <= w_last; ++w) {
                 const uint32_t m0w = (w >= lo0 && w <= hi0) ? r0[w] : 0u;
                 const uint32_t m1w = (w >= lo1 && w <= hi1) ? r1[w] : 0u;
@@ -446,7 +440,7 @@ __device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_
                     if (!__any_sync(kFull, ((m0 | m1) & 0x0303u) != 0u)) continue;
                     const uint32_t a0 = expand2(m0 & 3u), a2 = expand2((m0 >> 8) & 3u);
                     const uint32_t a1 = expand2(m1 & 3u), a3 = expand2((m1 >> 8) & 3u);
-                    const uint32_t b_addr = b_lane + (w * 32 + hh * 16) * kPitch + half * 128;
+                    const uint32_t b_addr = b_lane + (w * 32 + hh * 16) * kPitch;
 #pragma unroll
                     for (int np = 0; np < 4; ++np) {
                         uint32_t b0, b1, b2, b3;
@@ -456,20 +450,20 @@ __device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_
                     }
                 }
             }
-            merge_warps_sync();   // every merging warp has read what it needs of these columns
-            if (active) {
-                const float inv0 = 1.0f / (float)max(cnt0, 1), inv1 = 1.0f / (float)max(cnt1, 1);
-                unsigned char* o_lo = area_ptr + (cbase + g) * kPitch + half * 128 + tig * 4;
-                unsigned char* o_hi = o_lo + 8 * kPitch;
+        }
+        __syncthreads();   // every warp has read what it needs of rows [c0, ...)
+        if (active) {
+            const float inv0 = 1.0f / (float)max(cnt0, 1), inv1 = 1.0f / (float)max(cnt1, 1);
+            unsigned char* o_lo = area_ptr + (cbase + g) * kPitch + half * 128 + tig * 4;
+            unsigned char* o_hi = o_lo + 8 * kPitch;
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) {
-                    if (ok_lo) *reinterpret_cast<__nv_bfloat162*>(o_lo + nt * 16) = __floats2bfloat162_rn(acc[nt][0] * inv0, acc[nt][1] * inv0);
-                    if (ok_hi) *reinterpret_cast<__nv_bfloat162*>(o_hi + nt * 16) = __floats2bfloat162_rn(acc[nt][2] * inv1, acc[nt][3] * inv1);
-                }
-                if (write_counts && half == 0 && tig == 0) {
-                    if (ok_lo) *reinterpret_cast<int*>(area_ptr + (cbase + g) * kPitch + kRowBytes) = cnt0;
-                    if (ok_hi) *reinterpret_cast<int*>(area_ptr + (cbase + g + 8) * kPitch + kRowBytes) = cnt1;
-                }
+            for (int nt = 0; nt < 8; ++nt) {
+                if (ok_lo) *reinterpret_cast<__nv_bfloat162*>(o_lo + nt * 16) = __floats2bfloat162_rn(acc[nt][0] * inv0, acc[nt][1] * inv0);
+                if (ok_hi) *reinterpret_cast<__nv_bfloat162*>(o_hi + nt * 16) = __floats2bfloat162_rn(acc[nt][2] * inv1, acc[nt][3] * inv1);
+            }
+            if (write_counts && tig == 0) {
+                if (ok_lo) *reinterpret_cast<int*>(area_ptr + (cbase + g) * kPitch + kRowBytes) = cnt0;
+                if (ok_hi) *reinterpret_cast<int*>(area_ptr + (cbase + g + 8) * kPitch + kRowBytes) = cnt1;
             }
         }
     }
@@ -486,8 +480,10 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
     uint32_t* seedmask = reinterpret_cast<uint32_t*>(smem + kMiscOff);
     int* geo_buf = reinterpret_cast<int*>(smem + kMiscOff + 32);        // [2][8]
     int* misc = reinterpret_cast<int*>(smem + kMiscOff + 96);           // [0] output offset of the tile, [1] last block,
-                                                                        // [2] 32-row blocks that a segment of > 32 tokens touches
+                                                                        // [2] 32-row blocks that a segment of > 32 tokens touches,
+                                                                        // [3] number of segments of more than one token
     int* reach = reinterpret_cast<int*>(smem + kMiscOff + 112);         // [8] last block such a segment spans from block k
+    uint8_t* multi = smem + kMiscOff + 144;                             // [128] the segments of more than one token
     const uint32_t sbase = smem_u32(smem);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -496,7 +492,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
 
     if (warp == 0) fetch_tile(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
     if (tid < kNW) reach[tid] = 0;
-    if (tid == kNW) misc[2] = 0;
+    if (tid == kNW) misc[2] = misc[3] = 0;
+    if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
     __syncthreads();
 
     int buf = 0;
@@ -529,13 +526,24 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
             }
         }
         // end of the segment each row is in (0 past the tile)
-        if (tid < kNW) seedmask[tid] = 0u;
-        if (nseg == 1) {
+        // also: one-token segments (delimiters, lone tokens) are clusters of their own -- no key needed;
+        // the others are listed for the warps
+        int32_t* as = p.assign ? p.assign + (size_t)bh * p.n + row0 : nullptr;
+        if (nseg == 1 && R > 1) {
             for (int r = tid; r < R; r += kThreads) send[r] = (uint16_t)R;
             if (R > 32 && tid < nrb) { atomicOr(&misc[2], 1 << tid); reach[tid] = nrb - 1; }
+            if (tid == 0) { multi[0] = 0; misc[3] = 1; }
         } else {
             for (int s = tid; s < nseg; s += kThreads) {
                 const int a = segs[s], e = segs[s + 1];
+                if (e - a == 1) {
+                    send[a] = (uint16_t)e;
+                    adj[adj_row(a)] = 1u << (a & 31);
+                    atomicOr(&seedmask[a >> 5], 1u << (a & 31));
+                    if (as) as[a] = row0 + a;
+                    continue;
+                }
+                multi[atomicAdd(&misc[3], 1)] = (uint8_t)s;
                 for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
                 if (e - a > 32)
                     for (int k = a >> 5; k <= (e - 1) >> 5; ++k) { atomicOr(&misc[2], 1 << k); atomicMax(&reach[k], (e - 1) >> 5); }
@@ -572,44 +580,42 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         }
         CF_T(4);
 
-        // ---- 3. Algorithm 1 per segment, one warp each: in registers up to 32 tokens, else on the bit rows ----
-        int32_t* as = p.assign ? p.assign + (size_t)bh * p.n + row0 : nullptr;
-        for (int s = rwarp; s < nseg; s += kWarps) {
-            const int a = segs[s], e = segs[s + 1];
-            if (e - a == 1) {   // a delimiter or a one-token run: its own cluster
-                if (lane == 0) {
-                    adj[adj_row(a)] = 1u << (a & 31);
-                    atomicOr(&seedmask[a >> 5], 1u << (a & 31));
-                    if (as) as[a] = row0 + a;
+        // ---- 3. warp 0 draws the block's next ticket; warps 1-7: Algorithm 1 per segment, one warp each,
+        //         in registers up to 32 tokens, else on the bit rows ----
+        if (warp == 0) {
+            fetch_tile(p, lane, dec_b, dec_pref, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
+        } else {
+            const int nmulti = misc[3];
+            for (int k = warp - 1; k < nmulti; k += kWarps - 1) {
+                const int s = multi[k];
+                const int a = segs[s], e = segs[s + 1];
+                if (e - a <= 32) {
+                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
+                    else gsc_short_segment<false>(sbase, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
+                    continue;
                 }
-                continue;
-            }
-            if (e - a <= 32) {
-                if (p.tau < 0.f) gsc_short_segment<true>(sbase, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
-                else gsc_short_segment<false>(sbase, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
-                continue;
-            }
-            const int w1 = (e - 1) >> 5;
-            uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
-            uint32_t seeds = 0u;
-            for (;;) {
-                const uint32_t any = __ballot_sync(kFull, U != 0u);
-                if (any == 0u) break;
-                const int wf = __ffs(any) - 1;
-                const int i = wf * 32 + __ffs(__shfl_sync(kFull, U, wf)) - 1;   // lowest unassigned token: a seed
-                if (lane >= wf && lane <= w1) {
-                    uint32_t* slot = adj + adj_row(i) + (lane - wf);
-                    uint32_t mem = *slot & U;
-                    if (lane == wf) { mem |= 1u << (i & 31); seeds |= 1u << (i & 31); }
-                    *slot = mem;            // the row now lists the cluster's members
-                    U &= ~mem;
-                    if (as) {
-                        uint32_t mm = mem;
-                        while (mm) { const int j = lane * 32 + __ffs(mm) - 1; mm &= mm - 1; as[j] = row0 + i; }
+                const int w1 = (e - 1) >> 5;
+                uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
+                uint32_t seeds = 0u;
+                for (;;) {
+                    const uint32_t any = __ballot_sync(kFull, U != 0u);
+                    if (any == 0u) break;
+                    const int wf = __ffs(any) - 1;
+                    const int i = wf * 32 + __ffs(__shfl_sync(kFull, U, wf)) - 1;   // lowest unassigned token: a seed
+                    if (lane >= wf && lane <= w1) {
+                        uint32_t* slot = adj + adj_row(i) + (lane - wf);
+                        uint32_t mem = *slot & U;
+                        if (lane == wf) { mem |= 1u << (i & 31); seeds |= 1u << (i & 31); }
+                        *slot = mem;            // the row now lists the cluster's members
+                        U &= ~mem;
+                        if (as) {
+                            uint32_t mm = mem;
+                            while (mm) { const int j = lane * 32 + __ffs(mm) - 1; mm &= mm - 1; as[j] = row0 + i; }
+                        }
                     }
                 }
+                if (seeds) atomicOr(&seedmask[lane], seeds);
             }
-            if (seeds) atomicOr(&seedmask[lane], seeds);
         }
         __syncthreads();
         CF_T(5);
@@ -619,11 +625,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
 #pragma unroll
         for (int w = 0; w < kNW; ++w) P += __popc(seedmask[w]);
         uint32_t* stt = p.tile_state + (size_t)bh * p.n_tile_cap;
-        int16_t* segs_next = segs_buf + (buf ^ 1) * kSegsStride;
-        int* geo_next = geo_buf + (buf ^ 1) * 8;
         if (kMode == kCountOnly) {
             if (tid == 0) stt[t] = (uint32_t)P;
-            if (warp == 0) fetch_tile(p, lane, dec_b, dec_pref, geo_next, segs_next);
         } else {
             if (kMode == kLookBack && tid == 0)
                 atomicExch(&stt[t], (t == 0 ? kFlagPrefix : kFlagAggregate) | (uint32_t)P);
@@ -639,15 +642,14 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
             __syncthreads();
             CF_T(6);
 
-            // ---- 5. warps 4-7: Eq. 3; warp 0: next ticket; warp 1: output offset of the tile ----
-            if (warp >= kMergeWarp0) {
-                const int mw = warp - kMergeWarp0;
-                if (long_tile) merge_rounds(sbase, smem, mw, 4, P, seedrow, send, adj, lane, true);
-                else merge_rounds(sbase + (mw & 1) * kVOff, smem + (mw & 1) * kVOff, mw >> 1, 2, P, seedrow, send, adj, lane,
-                                  (mw & 1) == 0);
-            } else if (warp == 0) {
-                fetch_tile(p, lane, dec_b, dec_pref, geo_next, segs_next);
-            } else if (warp == 1) {
+            // ---- 5. Eq. 3 on all warps (tile of 16 clusters x tensor x column half each) ----
+            if (long_tile) merge_rounds(sbase, smem, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, (warp & 1) == 0);
+            else merge_rounds(sbase + (warp & 1) * kVOff, smem + (warp & 1) * kVOff, (warp >> 1) & 1, warp >> 2, 2, P, seedrow,
+                              send, adj, lane, (warp & 3) == 0);
+            CF_T(7);
+
+            // ---- output offset of the tile (warp 0) ----
+            if (warp == 0) {
                 int base = 0;
                 if (kMode == kWriteWithCounts) {
                     for (int k = lane; k < t; k += 32) base += (int)stt[k];
@@ -714,7 +716,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                 cp_async_commit();
                 cp_async_wait<0>();
                 __syncthreads();
-                if (warp >= kMergeWarp0) merge_rounds(sbase, smem, warp - kMergeWarp0, 4, P, seedrow, send, adj, lane, false);
+                merge_rounds(sbase, smem, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, false);
                 __syncthreads();
                 for (int idx = tid; idx < P * 16; idx += kThreads) {
                     const int row = idx >> 4, c = idx & 15;
@@ -725,7 +727,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
             }
         }
         if (tid < kNW) reach[tid] = 0;
-        if (tid == kNW) misc[2] = 0;
+        if (tid == kNW) misc[2] = misc[3] = 0;
+        if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
         __syncthreads();   // the next tile's copies overwrite what this one read and wrote
         CF_T(9);
         buf ^= 1;
