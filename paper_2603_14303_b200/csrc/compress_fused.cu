@@ -32,8 +32,8 @@ namespace sc {
 
 namespace cf {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
+constexpr int kWarps = 8;                         // compute warps
+constexpr int kThreads = (kWarps + 1) * 32;       // plus one service warp: next ticket, look-back
 constexpr int kD = 128;
 constexpr int kRowBytes = 256;                    // one K or V row in global memory
 constexpr int kPitch = 272;                       // its pitch in shared memory (16-byte pad)
@@ -66,12 +66,21 @@ __device__ unsigned long long g_phase_cycles[16];
             t_prev = now_;                                                      \
         }                                                                       \
     } while (0)
+// the same for a span measured by one lane of any warp
+#define CF_SPAN_BEGIN() const long long span_t0_ = clock64()
+#define CF_SPAN_END(i)                                                                             \
+    do {                                                                                           \
+        if ((threadIdx.x & 31) == 0) atomicAdd(&g_phase_cycles[i], (unsigned long long)(clock64() - span_t0_)); \
+    } while (0)
 #else
 #define CF_T(i)
+#define CF_SPAN_BEGIN()
+#define CF_SPAN_END(i)
 #endif
 
 constexpr uint32_t kFlagAggregate = 1u << 30, kFlagPrefix = 2u << 30, kValueMask = (1u << 30) - 1;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // the look-back gives up after 2 s
+constexpr int kPollGroups = 4;                               // the look-back reads 128 predecessors per poll
 constexpr int kCtlWords = 64;                                // ticket, done counter, padding
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -87,6 +96,9 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int sr
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void compute_warps_sync() {   // the eight compute warps, not the service warp
+    asm volatile("bar.sync 1, 256;\n" ::: "memory");
+}
 __device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
 }
@@ -451,7 +463,7 @@ __device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_
                 }
             }
         }
-        __syncthreads();   // every warp has read what it needs of rows [c0, ...)
+        compute_warps_sync();   // every compute warp has read what it needs of rows [c0, ...)
         if (active) {
             const float inv0 = 1.0f / (float)max(cnt0, 1), inv1 = 1.0f / (float)max(cnt1, 1);
             unsigned char* o_lo = area_ptr + (cbase + g) * kPitch + half * 128 + tig * 4;
@@ -487,10 +499,10 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
     const uint32_t sbase = smem_u32(smem);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int rwarp = kWarps - 1 - warp;   // per-tile work is dealt from the last warp down
-    int dec_b = 0, dec_pref = 0;           // ticket decoding state (warp 0)
+    const bool service = warp == kWarps;   // the ninth warp
+    int dec_b = 0, dec_pref = 0;           // ticket decoding state (service warp)
 
-    if (warp == 0) fetch_tile(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
+    if (service) fetch_tile(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
     if (tid < kNW) reach[tid] = 0;
     if (tid == kNW) misc[2] = misc[3] = 0;
     if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
@@ -517,6 +529,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         cp_async_commit();
         if (two_tensors) stage_rows(sbase + kVOff, p.V + goff, p.st.n, R, tid);
         cp_async_commit();
+        CF_T(1);
         if (p.ahead_rows > 0 && tid == 64) {   // contiguous cache: tickets advance in memory order
             const int64_t first = (int64_t)bh * p.n + row0 + p.ahead_rows;
             const int64_t rows = min((int64_t)R, p.total_rows - first);
@@ -559,17 +572,17 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         const int longblocks = misc[2];
         if (longblocks != 0) {
             float acc[2][4][4];
-            const bool have = rwarp < nrb && ((longblocks >> rwarp) & 1);
+            const bool have = warp < nrb && ((longblocks >> warp) & 1);   // nrb <= kWarps
             if (have) {
-                gram_block<true>(sbase, rwarp, rwarp, lane, acc);
-                store_norms(acc, rwarp, lane, norm);
+                gram_block<true>(sbase, warp, warp, lane, acc);
+                store_norms(acc, warp, lane, norm);
             }
             __syncthreads();
             if (have) {
-                if (p.tau < 0.f) threshold_block<true, true>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
-                else threshold_block<false, true>(acc, rwarp, rwarp, lane, p.tau, norm, send, adj);
+                if (p.tau < 0.f) threshold_block<true, true>(acc, warp, warp, lane, p.tau, norm, send, adj);
+                else threshold_block<false, true>(acc, warp, warp, lane, p.tau, norm, send, adj);
             }
-            for (int k = rwarp; k < 28; k += kWarps) {
+            for (int k = service ? 28 : warp; k < 28; k += kWarps) {
                 const int rb = kOffDiag[k] >> 4, cb = kOffDiag[k] & 15;
                 if (cb >= nrb || !((longblocks >> rb) & 1) || cb > reach[rb]) continue;
                 gram_block<false>(sbase, rb, cb, lane, acc);
@@ -580,13 +593,16 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         }
         CF_T(4);
 
-        // ---- 3. warp 0 draws the block's next ticket; warps 1-7: Algorithm 1 per segment, one warp each,
-        //         in registers up to 32 tokens, else on the bit rows ----
-        if (warp == 0) {
+        // ---- 3. the service warp draws the block's next ticket; compute warps: Algorithm 1 per segment,
+        //         one warp each, in registers up to 32 tokens, else on the bit rows ----
+        if (service) {
+            CF_SPAN_BEGIN();
             fetch_tile(p, lane, dec_b, dec_pref, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
+            CF_SPAN_END(10);
         } else {
+            CF_SPAN_BEGIN();
             const int nmulti = misc[3];
-            for (int k = warp - 1; k < nmulti; k += kWarps - 1) {
+            for (int k = warp; k < nmulti; k += kWarps) {
                 const int s = multi[k];
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a <= 32) {
@@ -616,6 +632,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                 }
                 if (seeds) atomicOr(&seedmask[lane], seeds);
             }
+            if (warp == 0) CF_SPAN_END(11);
+            if (warp == 7) CF_SPAN_END(12);
         }
         __syncthreads();
         CF_T(5);
@@ -642,37 +660,50 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
             __syncthreads();
             CF_T(6);
 
-            // ---- 5. Eq. 3 on all warps (tile of 16 clusters x tensor x column half each) ----
-            if (long_tile) merge_rounds(sbase, smem, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, (warp & 1) == 0);
-            else merge_rounds(sbase + (warp & 1) * kVOff, smem + (warp & 1) * kVOff, (warp >> 1) & 1, warp >> 2, 2, P, seedrow,
-                              send, adj, lane, (warp & 3) == 0);
-            CF_T(7);
-
-            // ---- output offset of the tile (warp 0) ----
-            if (warp == 0) {
+            // ---- 5. compute warps: Eq. 3 (tile of 16 clusters x tensor x column half each);
+            //         service warp: output offset of the tile ----
+            if (!service) {
+                if (long_tile) merge_rounds(sbase, smem, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, (warp & 1) == 0);
+                else merge_rounds(sbase + (warp & 1) * kVOff, smem + (warp & 1) * kVOff, (warp >> 1) & 1, warp >> 2, 2, P,
+                                  seedrow, send, adj, lane, (warp & 3) == 0);
+                CF_T(7);
+            } else {
+                CF_SPAN_BEGIN();
                 int base = 0;
                 if (kMode == kWriteWithCounts) {
                     for (int k = lane; k < t; k += 32) base += (int)stt[k];
                     base = warp_sum_i(base);
                 } else {
-                    // look back over the predecessors, 32 at a time, nearest first
+                    // look back over the predecessors, nearest first: one poll reads kPollGroups x 32 status
+                    // words (the loads overlap), then they are consumed 32 at a time
                     int upto = t;      // tiles [0, upto) still to be accounted for
-                    bool gave_up = false;
+                    bool gave_up = false, done = false;
                     unsigned long long t0 = 0;
-                    while (upto > 0) {
-                        const int k = upto - 1 - lane;
-                        const uint32_t v = (k >= 0) ? ld_volatile(&stt[k]) : kFlagPrefix;   // before tile 0: prefix 0
-                        const uint32_t ready = __ballot_sync(kFull, (v >> 30) != 0u);
-                        const uint32_t pref = __ballot_sync(kFull, (v >> 30) == 2u);
-                        // usable run: lanes 0..m-1 all ready, stopping at the first that holds a full prefix
-                        const int first_unready = (ready == kFull) ? 32 : __ffs(~ready) - 1;
-                        const int first_pref = pref ? __ffs(pref) - 1 : 32;
-                        const int take = min(first_unready, first_pref + 1);
-                        const int contrib = (lane < take) ? (int)(v & kValueMask) : 0;
-                        base += warp_sum_i(contrib);
-                        if (first_pref < first_unready) break;        // reached an inclusive prefix
-                        upto -= take;
-                        if (take == 0) {
+                    while (upto > 0 && !done) {
+                        uint32_t v[kPollGroups];
+#pragma unroll
+                        for (int j = 0; j < kPollGroups; ++j) {
+                            const int k = upto - 1 - lane - 32 * j;
+                            v[j] = (k >= 0) ? ld_volatile(&stt[k]) : kFlagPrefix;   // before tile 0: prefix 0
+                        }
+                        bool stalled = false, progressed = false;
+#pragma unroll
+                        for (int j = 0; j < kPollGroups; ++j) {
+                            if (done || stalled) continue;
+                            const uint32_t ready = __ballot_sync(kFull, (v[j] >> 30) != 0u);
+                            const uint32_t pref = __ballot_sync(kFull, (v[j] >> 30) == 2u);
+                            // usable run: lanes 0..m-1 all ready, stopping at the first that holds a full prefix
+                            const int first_unready = (ready == kFull) ? 32 : __ffs(~ready) - 1;
+                            const int first_pref = pref ? __ffs(pref) - 1 : 32;
+                            const int take = min(first_unready, first_pref + 1);
+                            const int contrib = (lane < take) ? (int)(v[j] & kValueMask) : 0;
+                            base += warp_sum_i(contrib);
+                            if (first_pref < first_unready) { done = true; continue; }   // reached an inclusive prefix
+                            upto -= take;
+                            progressed |= take > 0;
+                            stalled = take < 32;
+                        }
+                        if (!done && !progressed) {
                             if (t0 == 0) t0 = global_ns();
                             else if (global_ns() - t0 > kWaitLimitNs) { gave_up = true; break; }
                             __nanosleep(64);
@@ -688,6 +719,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                         if (base + P > p.cap) set_status(p.status, SC_ERR_CAPACITY);
                     }
                 }
+                CF_SPAN_END(13);
             }
             __syncthreads();
             CF_T(8);
@@ -716,7 +748,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                 cp_async_commit();
                 cp_async_wait<0>();
                 __syncthreads();
-                merge_rounds(sbase, smem, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, false);
+                if (!service) merge_rounds(sbase, smem, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, false);
                 __syncthreads();
                 for (int idx = tid; idx < P * 16; idx += kThreads) {
                     const int row = idx >> 4, c = idx & 15;
