@@ -110,9 +110,9 @@ sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dt
     a.core_k = core_k; a.core_v = core_v; a.count = count; a.cap = cap; a.core_len = core_len;
     a.assign = assign; a.ws = workspace; a.status = status;
     cudaError_t e;
-    if (!(a.flags & SC_FLAG_GENERIC) && compress_fused_supported(a)) {
-        e = launch_compress_fused(a, st);
-    } else {
+    e = cudaErrorNotSupported;
+    if (!(a.flags & SC_FLAG_GENERIC) && compress_fused_supported(a)) e = launch_compress_fused(a, st);
+    if (e == cudaErrorNotSupported) {   // forced, or a shape / layout the fused kernel does not take
         a.ws = (char*)workspace + fused_region_bytes(B, Hkv, n);   // never touches the fused kernel's words
         e = launch_compress_generic(a, st);
     }

@@ -4,28 +4,32 @@
 // counter.  A tile is a run of whole segments of at most SC_TILE_ROWS tokens of one (sequence, KV
 // head) -- K and V both staged in shared memory -- or one longer segment alone (K staged, then V
 // in a second pass over the same buffer).  Per tile:
-//   1. the rows are staged with 16-byte cp.async copies into rows of 272 bytes (the 16-byte pad
-//      makes ldmatrix conflict free without address swizzling).  Tickets walk the cache in memory
-//      order, so each block also asks L2 to prefetch the rows a fixed distance ahead of its tile
-//      (about what all resident blocks hold together): DRAM stays busy during the compute phases
-//      and the copies into shared memory mostly hit L2;
-//   2. Gram blocks K.K^T of 32x32 rows on the tensor cores (mma.m16n8k16; bf16 products are exact
-//      in fp32) for exactly the block pairs a segment spans; the diagonal gives the norms and
-//      Sim > tau (Eq. 2) is decided as G_ij > tau*|k_i|*|k_j|, packed into adjacency bit rows
-//      (later tokens of the same segment only, stored as an upper triangle of 32-bit words);
-//   3. Algorithm 1 per segment on those bit rows: the lowest unassigned token becomes a seed and
-//      takes every unassigned adjacent token -- a few word operations per seed, one warp per
-//      segment with one lane per 32-token word; the seed's row then holds its member mask;
+//   1. the rows are staged by TMA (cp.async.bulk.tensor, boxes of 16 rows x 64 columns, 128-byte
+//      swizzle so that ldmatrix is conflict free, completion on an mbarrier), issued by the block's
+//      ninth "service" warp.  Tickets walk the cache in memory order, so each block also asks L2
+//      to prefetch the rows a fixed distance ahead of its tile (about what all resident blocks
+//      hold together): DRAM stays busy during the compute phases and the boxes mostly hit L2;
+//   2. Eq. 2 + Algorithm 1, one warp per segment.  Up to 32 tokens (the usual case) everything
+//      stays in registers: mma.m16n8k16 tiles laid over the segment's own rows give the upper
+//      triangle of its Gram matrix (bf16 products are exact in fp32), the diagonal gives the norms,
+//      Sim > tau is decided as G_ij > tau*|k_i|*|k_j|, each lane ends up with one row's adjacency
+//      word, and the greedy pass costs one shuffle and a few word operations per seed;
+//   3. longer segments go through 32x32 Gram blocks for exactly the block pairs they span, with the
+//      adjacency bits in shared memory (an upper triangle of 32-bit words per row) and one lane
+//      per word in the greedy pass; either way a seed's row ends up holding its member mask;
 //   4. the tile's cluster count enters a prefix sum over the tiles of its (sequence, head): a
 //      decoupled look-back over per-tile status words (tickets are handed out in order, so every
 //      predecessor is held by a running block and the bounded wait cannot starve), or, in
 //      two-pass mode, a count pass followed by a write pass;
-//   5. Eq. 3 as a product on the tensor cores (warps 4-7): member masks expanded to a 0/1 bf16
-//      matrix times the staged K (V) rows, fp32 accumulation, one multiply by 1/|S|, one rounding
-//      to bf16; the cores are compacted in place in shared memory and leave with 16-byte
-//      coalesced stores.  Meanwhile warp 0 draws the block's next ticket and warp 1 looks back.
+//   5. Eq. 3 as a product on the tensor cores: member masks expanded to a 0/1 bf16 matrix times
+//      the staged K (V) rows, fp32 accumulation, one multiply by 1/|S|, one rounding to bf16; the
+//      cores are compacted in place in shared memory and leave with 16-byte coalesced stores.
+//      Meanwhile the service warp looks back; it draws the block's next ticket during step 2.
 // The last block to finish zeroes the status words and counters, so a workspace that was zero
 // before the call is zero again after it.
+#include <cuda.h>
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace sc {
@@ -36,20 +40,27 @@ constexpr int kWarps = 8;                         // compute warps
 constexpr int kThreads = (kWarps + 1) * 32;       // plus one service warp: next ticket, look-back
 constexpr int kD = 128;
 constexpr int kRowBytes = 256;                    // one K or V row in global memory
-constexpr int kPitch = 272;                       // its pitch in shared memory (16-byte pad)
+constexpr int kHalfRow = 128;                     // a staged row is two 128-byte halves (64 columns each), see tile_addr
+constexpr int kBoxRows = 16;                      // rows per TMA box
+constexpr int kBoxBytes = kBoxRows * kHalfRow;    // 2048
 constexpr int kMaxRows = SC_MAX_CHUNK_LEN;        // 256: a long tile
 constexpr int kShortRows = SC_TILE_ROWS;          // 128
 constexpr int kNW = 8;                            // 32-bit words per (full) adjacency row
-constexpr int kKvBytes = kMaxRows * kPitch;       // 69632: short = K | V halves, long = one tensor
-constexpr int kVOff = kShortRows * kPitch;        // 34816
-constexpr int kAdjOff = kKvBytes;
+constexpr int kKvBytes = kMaxRows * kRowBytes;    // 65536: short = K | V, long = one tensor
+constexpr int kVOff = kShortRows * kRowBytes;     // 32768
+constexpr int kHalfShort = kShortRows * kHalfRow; // 16384: distance between the column halves of a short tile
+constexpr int kHalfLong = kMaxRows * kHalfRow;    // 32768: ... of a long one
+constexpr int kCntOff = kKvBytes;                 // uint16[256]: members of each cluster
+constexpr int kAdjOff = kCntOff + kMaxRows * 2;
 constexpr int kAdjWords = 32 * (8 + 7 + 6 + 5 + 4 + 3 + 2 + 1);   // rows of block k keep words k..7
 constexpr int kNormOff = kAdjOff + kAdjWords * 4; // float[256]; later uint16 seed row per cluster
 constexpr int kSendOff = kNormOff + kMaxRows * 4; // uint16[256]: end of the segment a row is in
 constexpr int kSegsOff = kSendOff + kMaxRows * 2; // 2 x int16[132]: segment starts (this tile, next tile)
 constexpr int kSegsStride = 132;
 constexpr int kMiscOff = kSegsOff + 2 * kSegsStride * 2;   // uint32 seedmask[8]; int geo[2][8]; int misc[4]
-constexpr int kSmemBytes = kMiscOff + 32 + 64 + 16 + 32 + 128;   // ... int reach[8]; uint8 multi[128]
+constexpr int kBarOff = kMiscOff + 32 + 64 + 16 + 32 + 128;      // ... int reach[8]; uint8 multi[128]; two mbarriers
+constexpr int kSmemBytes = kBarOff + 16;
+static_assert(kBarOff % 8 == 0, "mbarrier alignment");
 static_assert(kSmemBytes <= 76800, "three blocks per SM need <= 75 KB each");
 
 enum Mode { kCountOnly = 0, kWriteWithCounts = 1, kLookBack = 2 };
@@ -79,7 +90,7 @@ __device__ unsigned long long g_phase_cycles[16];
 #endif
 
 constexpr uint32_t kFlagAggregate = 1u << 30, kFlagPrefix = 2u << 30, kValueMask = (1u << 30) - 1;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // the look-back gives up after 2 s
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every wait gives up after 2 s
 constexpr int kPollGroups = 4;                               // the look-back reads 128 predecessors per poll
 constexpr int kCtlWords = 64;                                // ticket, done counter, padding
 
@@ -89,13 +100,39 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
     return t;
 }
-// 16-byte asynchronous copy; src_bytes = 0 fills the destination with zeros instead.
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0u;
+}
+// Bounded wait for a phase of an mbarrier; false if it gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > kWaitLimitNs) return false;
+    }
+}
+// One TMA box: 16 rows x 64 columns of a [B, Hkv, n, 128] tensor, 128-byte swizzled, no multicast.
+__device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* map, int col, int row, int h, int b, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(row), "r"(h), "r"(b), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+// Byte offset, inside one column half of a staged tensor, of 16-byte chunk `chunk` (0..7) of row
+// `row`: rows are 128 bytes apart and the chunk index is XORed with the row's low three bits (the
+// TMA 128-byte swizzle), which makes ldmatrix over eight consecutive rows conflict free.
+__device__ __forceinline__ uint32_t tile_addr(int row, int chunk) { return row * kHalfRow + ((chunk ^ (row & 7)) << 4); }
 __device__ __forceinline__ void compute_warps_sync() {   // the eight compute warps, not the service warp
     asm volatile("bar.sync 1, 256;\n" ::: "memory");
 }
@@ -137,26 +174,28 @@ __device__ __forceinline__ uint32_t expand2(uint32_t two_bits) {
     return ((two_bits * 0x8001u) & 0x00010001u) * 0x3F80u;
 }
 
-// 32x32 block of K.K^T: rows of block rb against rows of block cb (rows staged at pitch kPitch).
+// 32x32 block of K.K^T: rows of block rb against rows of block cb (column halves `hs` bytes apart).
 template <bool kDiag>
-__device__ __forceinline__ void gram_block(uint32_t kbase, int rb, int cb, int lane, float (&acc)[2][4][4]) {
+__device__ __forceinline__ void gram_block(uint32_t kbase, int hs, int rb, int cb, int lane, float (&acc)[2][4][4]) {
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = acc[mt][nt][2] = acc[mt][nt][3] = 0.f;
     const int j = lane >> 3, r8 = lane & 7;
     // A: matrices (r0-7,c) (r8-15,c) (r0-7,c+1) (r8-15,c+1);  B: (r0-7,c) (r0-7,c+1) (r8-15,c) (r8-15,c+1)
-    const uint32_t a_addr = kbase + (rb * 32 + r8 + ((j & 1) << 3)) * kPitch + ((j >> 1) << 4);
-    const uint32_t b_addr = kbase + (cb * 32 + r8 + ((j >> 1) << 3)) * kPitch + ((j & 1) << 4);
+    // chunk 2*ks + c of a row sits in half ks >> 2 at chunk (2*(ks & 3) + c) ^ (row & 7): XOR of a constant
+    const uint32_t a_addr = kbase + tile_addr(rb * 32 + r8 + ((j & 1) << 3), j >> 1);
+    const uint32_t b_addr = kbase + tile_addr(cb * 32 + r8 + ((j >> 1) << 3), j & 1);
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
         uint32_t a[2][4], bq[2][4];
+        const uint32_t kx = (ks & 3) << 5, ko = (ks >> 2) * hs;
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
-            ldmatrix_x4(a_addr + mt * 16 * kPitch + ks * 32, a[mt][0], a[mt][1], a[mt][2], a[mt][3]);
+            ldmatrix_x4((a_addr ^ kx) + ko + mt * 16 * kHalfRow, a[mt][0], a[mt][1], a[mt][2], a[mt][3]);
 #pragma unroll
         for (int p = 0; p < 2; ++p)
-            ldmatrix_x4(b_addr + p * 16 * kPitch + ks * 32, bq[p][0], bq[p][1], bq[p][2], bq[p][3]);
+            ldmatrix_x4((b_addr ^ kx) + ko + p * 16 * kHalfRow, bq[p][0], bq[p][1], bq[p][2], bq[p][3]);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
@@ -233,7 +272,7 @@ __constant__ uint8_t kOffDiag[28] = {0x01, 0x12, 0x23, 0x34, 0x45, 0x56, 0x67, 0
 // one shuffle per seed.  Results: seed bits into the tile's seedmask, each seed's member mask into
 // its (tile-relative) adjacency row for the Eq. 3 product, optionally the seed of every token.
 template <bool kNegTau>
-__device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int a, int l, float tau, float* nrm /*[32], this warp's*/,
+__device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int hs, int a, int l, float tau, float* nrm /*[32], this warp's*/,
                                                   uint32_t* adj, uint32_t* seedmask, int32_t* as, int row0, int lane) {
     const int g = lane >> 2, tig = lane & 3;
     const int nnt = (l + 7) >> 3;          // 8-column tiles that hold tokens: 1..4
@@ -245,18 +284,20 @@ __device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int a, int l, 
         for (int nt = 0; nt < 4; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = acc[mt][nt][2] = acc[mt][nt][3] = 0.f;
     {
         const int j = lane >> 3, r8 = lane & 7;
-        const uint32_t a_addr = kbase + (a + r8 + ((j & 1) << 3)) * kPitch + ((j >> 1) << 4);
-        const uint32_t b_addr = kbase + (a + r8 + ((j >> 1) << 3)) * kPitch + ((j & 1) << 4);
+        const uint32_t a_base = kbase + tile_addr(a + r8 + ((j & 1) << 3), j >> 1);
+        const uint32_t b_base = kbase + tile_addr(a + r8 + ((j >> 1) << 3), j & 1);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             uint32_t a0[4], a1[4], b0[4], b1[4];
-            ldmatrix_x4(a_addr + ks * 32, a0[0], a0[1], a0[2], a0[3]);
-            ldmatrix_x4(b_addr + ks * 32, b0[0], b0[1], b0[2], b0[3]);
+            const uint32_t a_addr = (a_base ^ ((ks & 3) << 5)) + (ks >> 2) * hs;
+            const uint32_t b_addr = (b_base ^ ((ks & 3) << 5)) + (ks >> 2) * hs;
+            ldmatrix_x4(a_addr, a0[0], a0[1], a0[2], a0[3]);
+            ldmatrix_x4(b_addr, b0[0], b0[1], b0[2], b0[3]);
             mma_bf16(acc[0][0], a0[0], a0[1], a0[2], a0[3], b0[0], b0[1]);
             if (nnt > 1) mma_bf16(acc[0][1], a0[0], a0[1], a0[2], a0[3], b0[2], b0[3]);
             if (two_mt) {
-                ldmatrix_x4(a_addr + 16 * kPitch + ks * 32, a1[0], a1[1], a1[2], a1[3]);
-                ldmatrix_x4(b_addr + 16 * kPitch + ks * 32, b1[0], b1[1], b1[2], b1[3]);
+                ldmatrix_x4(a_addr + 16 * kHalfRow, a1[0], a1[1], a1[2], a1[3]);
+                ldmatrix_x4(b_addr + 16 * kHalfRow, b1[0], b1[1], b1[2], b1[3]);
                 mma_bf16(acc[0][2], a0[0], a0[1], a0[2], a0[3], b1[0], b1[1]);
                 mma_bf16(acc[1][2], a1[0], a1[1], a1[2], a1[3], b1[0], b1[1]);
                 if (nnt > 3) {
@@ -358,6 +399,7 @@ struct Params {
     int32_t* ctl;            // [0] ticket counter, [1] blocks finished
     uint32_t* tile_state;    // [B*Hkv][n_tile_cap]
     int32_t* status;
+    CUtensorMap map_k, map_v;   // [B, Hkv, n, 128] bf16, boxes of 16 rows x 64 columns, 128-byte swizzle
     int ahead_rows;          // L2 prefetch distance in rows; 0 = the cache is not one contiguous [B*Hkv*n, d] array
     int64_t total_rows;      // B*Hkv*n
 };
@@ -397,34 +439,34 @@ __device__ __forceinline__ void fetch_tile(const Params& p, int lane, int& dec_b
     }
 }
 
-// Stages rows [0, R) of one tensor (row r at src + r*stride elements) at `dst`, pitch kPitch, and
-// zero-fills up to the next multiple of 16 rows (those rows enter the Eq. 3 product with weight 0).
-__device__ __forceinline__ void stage_rows(uint32_t dst, const __nv_bfloat16* src, int64_t stride, int R, int tid) {
-    const int c = tid & 15, r0 = tid >> 4;
-    const char* s = reinterpret_cast<const char*>(src + (int64_t)r0 * stride) + c * 16;
-    uint32_t d = dst + r0 * kPitch + c * 16;
-    const int64_t s_step = stride * (2 * (kThreads / 16));
-    for (int r = r0; r < R; r += kThreads / 16) {
-        cp_async16(d, s, 16);
-        s += s_step;
-        d += (kThreads / 16) * kPitch;
+// Stages rows [row0, row0 + R) of head (b, h) of one tensor with TMA: one box of 16 rows x 64 columns
+// per lane (R <= 256 needs at most 32 boxes for both column halves), the halves `hs` bytes apart at
+// `dst`.  Rows past R inside the last box are the cache's next rows, or zeros past the end of the
+// sequence: finite either way, and they only ever enter the Eq. 3 product with weight 0.
+__device__ __forceinline__ void stage_rows(uint32_t dst, int hs, const CUtensorMap* map, int row0, int R, int h, int b,
+                                           uint32_t bar, int lane) {
+    const int nb = (R + kBoxRows - 1) / kBoxRows;
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)(2 * nb * kBoxBytes));
+    __syncwarp();
+    if (lane < 2 * nb) {
+        const int half = lane >= nb, i = lane - half * nb;
+        tma_box(dst + half * hs + i * kBoxBytes, map, half * 64, row0 + i * kBoxRows, h, b, bar);
     }
-    const int r = R + r0;   // at most 15 rows of padding
-    if (r < ((R + 15) & ~15)) cp_async16(dst + r * kPitch + c * 16, src, 0);
 }
 
-// Eq. 3 on the tensor cores for one staged tensor (K or V rows at `area`, pitch kPitch).
+// Eq. 3 on the tensor cores for one staged tensor (K or V rows at `area`, column halves hs bytes apart).
 // Cluster c (in seed order) has its member mask in the adjacency row of its seed seedrow[c].  A
 // warp owns one tile of 16 clusters (mt_in_round of a round of mts_per_round tiles) and one half
 // of the 128 columns:  acc[16 x 64] = mask[16 x rows] . rows[rows x 64].
 // The scaled, rounded cores overwrite rows [0, P) of the same area: cluster c only reads rows >=
 // its seed >= c, rounds go up in c, and inside a round every warp has finished reading before any
-// of them writes.  The 16-byte pad of row c receives the cluster's member count.
-__device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_ptr, int half, int mt_in_round,
+// of them writes.  cnts[c] receives the cluster's member count (from the warps told to write it).
+__device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_ptr, int hs, int half, int mt_in_round,
                                              int mts_per_round, int P, const uint16_t* seedrow, const uint16_t* send,
-                                             const uint32_t* adj, int lane, bool write_counts) {
+                                             const uint32_t* adj, int lane, uint16_t* cnts /*or null*/) {
     const int g = lane >> 2, tig = lane & 3;
-    const uint32_t b_lane = area + ((lane & 7) + ((lane >> 3) & 1) * 8) * kPitch + (lane >> 4) * 16 + half * 128;
+    // the warp's 64 columns are exactly one column half; chunk 2*np + c of it, rows k0 + (0..15), k0 % 16 == 0
+    const uint32_t b_lane = area + half * hs + tile_addr((lane & 7) + ((lane >> 3) & 1) * 8, lane >> 4);
     for (int c0 = 0; c0 < P; c0 += 16 * mts_per_round) {
         const int cbase = c0 + 16 * mt_in_round;
         const bool active = cbase < P;
@@ -452,11 +494,11 @@ __device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_
                     if (!__any_sync(kFull, ((m0 | m1) & 0x0303u) != 0u)) continue;
                     const uint32_t a0 = expand2(m0 & 3u), a2 = expand2((m0 >> 8) & 3u);
                     const uint32_t a1 = expand2(m1 & 3u), a3 = expand2((m1 >> 8) & 3u);
-                    const uint32_t b_addr = b_lane + (w * 32 + hh * 16) * kPitch;
+                    const uint32_t b_addr = b_lane + (w * 32 + hh * 16) * kHalfRow;
 #pragma unroll
                     for (int np = 0; np < 4; ++np) {
                         uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4_trans(b_addr + np * 32, b0, b1, b2, b3);
+                        ldmatrix_x4_trans(b_addr ^ (np << 5), b0, b1, b2, b3);
                         mma_bf16(acc[2 * np], a0, a1, a2, a3, b0, b1);
                         mma_bf16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
                     }
@@ -466,24 +508,27 @@ __device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_
         compute_warps_sync();   // every compute warp has read what it needs of rows [c0, ...)
         if (active) {
             const float inv0 = 1.0f / (float)max(cnt0, 1), inv1 = 1.0f / (float)max(cnt1, 1);
-            unsigned char* o_lo = area_ptr + (cbase + g) * kPitch + half * 128 + tig * 4;
-            unsigned char* o_hi = o_lo + 8 * kPitch;
+            // rows cbase + g and cbase + g + 8 both have (row & 7) == g: chunk nt lands at chunk nt ^ g
+            unsigned char* o_lo = area_ptr + half * hs + (cbase + g) * kHalfRow + tig * 4;
+            unsigned char* o_hi = o_lo + 8 * kHalfRow;
 #pragma unroll
             for (int nt = 0; nt < 8; ++nt) {
-                if (ok_lo) *reinterpret_cast<__nv_bfloat162*>(o_lo + nt * 16) = __floats2bfloat162_rn(acc[nt][0] * inv0, acc[nt][1] * inv0);
-                if (ok_hi) *reinterpret_cast<__nv_bfloat162*>(o_hi + nt * 16) = __floats2bfloat162_rn(acc[nt][2] * inv1, acc[nt][3] * inv1);
+                const int o = (nt ^ g) << 4;
+                if (ok_lo) *reinterpret_cast<__nv_bfloat162*>(o_lo + o) = __floats2bfloat162_rn(acc[nt][0] * inv0, acc[nt][1] * inv0);
+                if (ok_hi) *reinterpret_cast<__nv_bfloat162*>(o_hi + o) = __floats2bfloat162_rn(acc[nt][2] * inv1, acc[nt][3] * inv1);
             }
-            if (write_counts && tig == 0) {
-                if (ok_lo) *reinterpret_cast<int*>(area_ptr + (cbase + g) * kPitch + kRowBytes) = cnt0;
-                if (ok_hi) *reinterpret_cast<int*>(area_ptr + (cbase + g + 8) * kPitch + kRowBytes) = cnt1;
+            if (cnts != nullptr && tig == 0) {
+                if (ok_lo) cnts[cbase + g] = (uint16_t)cnt0;
+                if (ok_hi) cnts[cbase + g + 8] = (uint16_t)cnt1;
             }
         }
     }
 }
 
 template <int kMode>
-__global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Params p) {
-    extern __shared__ __align__(128) unsigned char smem[];
+__global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __grid_constant__ Params p) {
+    extern __shared__ __align__(1024) unsigned char smem[];   // the swizzle pattern repeats every 1024 bytes
+    uint16_t* cnts = reinterpret_cast<uint16_t*>(smem + kCntOff);
     uint32_t* adj = reinterpret_cast<uint32_t*>(smem + kAdjOff);
     float* norm = reinterpret_cast<float*>(smem + kNormOff);
     uint16_t* seedrow = reinterpret_cast<uint16_t*>(smem + kNormOff);   // reuses the norms once they are spent
@@ -497,10 +542,21 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
     int* reach = reinterpret_cast<int*>(smem + kMiscOff + 112);         // [8] last block such a segment spans from block k
     uint8_t* multi = smem + kMiscOff + 144;                             // [128] the segments of more than one token
     const uint32_t sbase = smem_u32(smem);
+    const uint32_t bar_k = sbase + kBarOff, bar_v = bar_k + 8;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool service = warp == kWarps;   // the ninth warp
     int dec_b = 0, dec_pref = 0;           // ticket decoding state (service warp)
+
+    if (tid == 0) {
+        mbar_init(bar_k, 1);
+        mbar_init(bar_v, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        if ((sbase & 1023u) != 0u) set_status(p.status, SC_ERR_CUDA);   // the swizzled addressing assumes this
+    }
+    fence_async_proxy();
+    uint32_t phase_k = 0, phase_v = 0;
+    bool failed = false;
 
     if (service) fetch_tile(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
     if (tid < kNW) reach[tid] = 0;
@@ -522,13 +578,13 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         const bool long_tile = R > kShortRows;
         const bool two_tensors = (kMode != kCountOnly) && !long_tile;   // V staged beside K
         const int nrb = (R + 31) >> 5;
-        const int64_t goff = b * p.st.b + h * p.st.h + (int64_t)row0 * p.st.n;
+        const int hs = long_tile ? kHalfLong : kHalfShort;
 
-        // ---- 1. stage the rows; prefetch ahead ----
-        stage_rows(sbase, p.K + goff, p.st.n, R, tid);
-        cp_async_commit();
-        if (two_tensors) stage_rows(sbase + kVOff, p.V + goff, p.st.n, R, tid);
-        cp_async_commit();
+        // ---- 1. stage the rows (service warp, TMA); prefetch ahead ----
+        if (service) {
+            stage_rows(sbase, hs, &p.map_k, row0, R, h, b, bar_k, lane);
+            if (two_tensors) stage_rows(sbase + kVOff, hs, &p.map_v, row0, R, h, b, bar_v, lane);
+        }
         CF_T(1);
         if (p.ahead_rows > 0 && tid == 64) {   // contiguous cache: tickets advance in memory order
             const int64_t first = (int64_t)bh * p.n + row0 + p.ahead_rows;
@@ -564,8 +620,9 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
         }
         for (int r = R + tid; r < nrb * 32; r += kThreads) send[r] = (uint16_t)0;
         CF_T(0);
-        cp_async_wait<1>();   // this thread's K copies; the barrier publishes everyone's
-        __syncthreads();
+        failed = !mbar_wait(bar_k, phase_k);   // K has landed
+        phase_k ^= 1u;
+        if (__syncthreads_or(failed)) { failed = true; break; }
         CF_T(2);
 
         // ---- 2. segments of more than 32 tokens: Gram blocks -> norms -> adjacency bits in shared memory ----
@@ -574,7 +631,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
             float acc[2][4][4];
             const bool have = warp < nrb && ((longblocks >> warp) & 1);   // nrb <= kWarps
             if (have) {
-                gram_block<true>(sbase, warp, warp, lane, acc);
+                gram_block<true>(sbase, hs, warp, warp, lane, acc);
                 store_norms(acc, warp, lane, norm);
             }
             __syncthreads();
@@ -585,7 +642,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
             for (int k = service ? 28 : warp; k < 28; k += kWarps) {
                 const int rb = kOffDiag[k] >> 4, cb = kOffDiag[k] & 15;
                 if (cb >= nrb || !((longblocks >> rb) & 1) || cb > reach[rb]) continue;
-                gram_block<false>(sbase, rb, cb, lane, acc);
+                gram_block<false>(sbase, hs, rb, cb, lane, acc);
                 if (p.tau < 0.f) threshold_block<true, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
                 else threshold_block<false, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
             }
@@ -606,8 +663,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                 const int s = multi[k];
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a <= 32) {
-                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
-                    else gsc_short_segment<false>(sbase, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
+                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
+                    else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
                     continue;
                 }
                 const int w1 = (e - 1) >> 5;
@@ -656,16 +713,20 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                     seedrow[rank] = (uint16_t)tid;
                 }
             }
-            cp_async_wait<0>();   // V
-            __syncthreads();
+            if (two_tensors) {
+                failed = !mbar_wait(bar_v, phase_v);   // V has landed
+                phase_v ^= 1u;
+            }
+            if (__syncthreads_or(failed)) { failed = true; break; }
             CF_T(6);
 
             // ---- 5. compute warps: Eq. 3 (tile of 16 clusters x tensor x column half each);
             //         service warp: output offset of the tile ----
             if (!service) {
-                if (long_tile) merge_rounds(sbase, smem, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, (warp & 1) == 0);
-                else merge_rounds(sbase + (warp & 1) * kVOff, smem + (warp & 1) * kVOff, (warp >> 1) & 1, warp >> 2, 2, P,
-                                  seedrow, send, adj, lane, (warp & 3) == 0);
+                if (long_tile) merge_rounds(sbase, smem, hs, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane,
+                                            (warp & 1) == 0 ? cnts : nullptr);
+                else merge_rounds(sbase + (warp & 1) * kVOff, smem + (warp & 1) * kVOff, hs, (warp >> 1) & 1, warp >> 2, 2, P,
+                                  seedrow, send, adj, lane, (warp & 3) == 0 ? cnts : nullptr);
                 CF_T(7);
             } else {
                 CF_SPAN_BEGIN();
@@ -731,42 +792,50 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
                 const int row = idx >> 4, c = idx & 15;
                 if (base + row < p.cap) {
                     const size_t o = (obase + base + row) * kD + c * 8;
-                    *reinterpret_cast<uint4*>(p.core_k + o) = *reinterpret_cast<const uint4*>(smem + row * kPitch + c * 16);
-                    if (!long_tile)
-                        *reinterpret_cast<uint4*>(p.core_v + o) =
-                            *reinterpret_cast<const uint4*>(smem + kVOff + row * kPitch + c * 16);
+                    const unsigned char* src = smem + (c >> 3) * hs + tile_addr(row, c & 7);
+                    *reinterpret_cast<uint4*>(p.core_k + o) = *reinterpret_cast<const uint4*>(src);
+                    if (!long_tile) *reinterpret_cast<uint4*>(p.core_v + o) = *reinterpret_cast<const uint4*>(src + kVOff);
                 }
             }
             for (int row = tid; row < P; row += kThreads)
                 if (base + row < p.cap)
-                    p.count[obase + base + row] = *reinterpret_cast<const int*>(smem + row * kPitch + kRowBytes);
+                    p.count[obase + base + row] = (int32_t)cnts[row];
 
             // ---- a long segment: V takes the place of K and goes through the same product ----
             if (long_tile) {
+                fence_async_proxy();   // the copies below overwrite what ordinary accesses read and wrote
                 __syncthreads();
-                stage_rows(sbase, p.V + goff, p.st.n, R, tid);
-                cp_async_commit();
-                cp_async_wait<0>();
-                __syncthreads();
-                if (!service) merge_rounds(sbase, smem, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, false);
+                if (service) stage_rows(sbase, hs, &p.map_v, row0, R, h, b, bar_v, lane);
+                failed = !mbar_wait(bar_v, phase_v);
+                phase_v ^= 1u;
+                if (__syncthreads_or(failed)) { failed = true; break; }
+                if (!service) merge_rounds(sbase, smem, hs, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, nullptr);
                 __syncthreads();
                 for (int idx = tid; idx < P * 16; idx += kThreads) {
                     const int row = idx >> 4, c = idx & 15;
                     if (base + row < p.cap)
                         *reinterpret_cast<uint4*>(p.core_v + (obase + base + row) * kD + c * 8) =
-                            *reinterpret_cast<const uint4*>(smem + row * kPitch + c * 16);
+                            *reinterpret_cast<const uint4*>(smem + (c >> 3) * hs + tile_addr(row, c & 7));
                 }
             }
         }
         if (tid < kNW) reach[tid] = 0;
         if (tid == kNW) misc[2] = misc[3] = 0;
         if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
-        __syncthreads();   // the next tile's copies overwrite what this one read and wrote
+        fence_async_proxy();   // the next tile's copies overwrite what ordinary accesses read and wrote
+        __syncthreads();
         CF_T(9);
         buf ^= 1;
     }
 
     // ---- exit: the last block to finish leaves the workspace zeroed for the next call ----
+    if (failed) {   // a wait gave up: report it, and give copies that may still be in flight one more bounded
+                    // wait (either parity: whichever phase is open) before the block's shared memory goes away
+        if (tid == 0) set_status(p.status, SC_ERR_TIMEOUT);
+        mbar_wait(bar_k, phase_k ^ 1u);
+        mbar_wait(bar_v, phase_v ^ 1u);
+        mbar_wait(bar_v, phase_v);
+    }
     __syncthreads();
     if (tid == 0) {
         __threadfence();
@@ -786,10 +855,47 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const Param
 
 }  // namespace cf
 
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link the driver).
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// [B, Hkv, n, 128] bf16 with element strides st, read in boxes of 16 rows x 64 columns.
+bool make_map(CUtensorMap* map, const void* base, const sc_strides& st, int B, int Hkv, int n) {
+    EncodeTiledFn enc = encode_tiled();
+    if (enc == nullptr) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)cf::kD, (cuuint64_t)n, (cuuint64_t)Hkv, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)st.n * 2, (cuuint64_t)(Hkv > 1 ? st.h : st.n * n) * 2,
+                                   (cuuint64_t)(B > 1 ? st.b : st.n * n * (int64_t)Hkv) * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)cf::kBoxRows, 1, 1};
+    const cuuint32_t elem[4] = {1, 1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, elem,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 bool compress_fused_supported(const CompressArgs& a) {
-    // ticket arithmetic is 32-bit
+    // ticket arithmetic is 32-bit; TMA strides are below 2^40 bytes
+    const int64_t lim = (int64_t)1 << 39;
     return a.dt == SC_BF16 && a.d == cf::kD && a.n_tile_cap >= 1 &&
-           (int64_t)a.B * a.Hkv * (int64_t)a.n_tile_cap < (int64_t)1 << 30;
+           (int64_t)a.B * a.Hkv * (int64_t)a.n_tile_cap < (int64_t)1 << 30 && a.st.n > 0 && a.st.n < lim &&
+           a.st.h >= 0 && a.st.h < lim && a.st.b >= 0 && a.st.b < lim && encode_tiled() != nullptr;
 }
 
 size_t compress_fused_ws_bytes(int32_t B, int32_t Hkv, int32_t n) {
@@ -822,6 +928,8 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
     p.ctl = (int32_t*)a.ws;
     p.tile_state = (uint32_t*)a.ws + cf::kCtlWords;
     p.status = a.status;
+    if (!make_map(&p.map_k, a.K, a.st, a.B, a.Hkv, a.n) || !make_map(&p.map_v, a.V, a.st, a.B, a.Hkv, a.n))
+        return cudaErrorNotSupported;   // a layout TMA cannot describe: the caller takes the generic kernels
     // no more blocks than there can be tiles
     const int64_t max_tiles = (int64_t)a.B * a.Hkv * a.n_tile_cap;
     const int grid = (int)(max_tiles < grid_of[dev] ? max_tiles : grid_of[dev]);
@@ -829,6 +937,9 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
     const bool contiguous = a.st.n == cf::kD && a.st.h == (int64_t)a.n * cf::kD && a.st.b == (int64_t)a.Hkv * a.n * cf::kD;
     p.ahead_rows = contiguous ? grid * SC_TILE_ROWS : 0;
     p.total_rows = (int64_t)a.B * a.Hkv * a.n;
+#ifdef SC_TUNE   // tuning harness only
+    if (const char* e = getenv("SC_CF_AHEAD")) p.ahead_rows = contiguous ? atoi(e) : 0;
+#endif
     if (a.flags & SC_FLAG_TWO_PASS) {
         cf::Params pc = p;
         pc.assign = nullptr;
