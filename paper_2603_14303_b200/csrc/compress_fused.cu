@@ -6,9 +6,7 @@
 // in a second pass over the same buffer).  Per tile:
 //   1. the rows are staged by TMA (cp.async.bulk.tensor, boxes of 16 rows x 64 columns, 128-byte
 //      swizzle so that ldmatrix is conflict free, completion on an mbarrier), issued by the block's
-//      ninth "service" warp.  Tickets walk the cache in memory order, so each block also asks L2
-//      to prefetch the rows a fixed distance ahead of its tile (about what all resident blocks
-//      hold together): DRAM stays busy during the compute phases and the boxes mostly hit L2;
+//      ninth "service" warp;
 //   2. Eq. 2 + Algorithm 1, one warp per segment.  Up to 32 tokens (the usual case) everything
 //      stays in registers: mma.m16n8k16 tiles laid over the segment's own rows give the upper
 //      triangle of its Gram matrix (bf16 products are exact in fp32), the diagonal gives the norms,
@@ -21,14 +19,15 @@
 //      decoupled look-back over per-tile status words (tickets are handed out in order, so every
 //      predecessor is held by a running block and the bounded wait cannot starve), or, in
 //      two-pass mode, a count pass followed by a write pass;
-//   5. Eq. 3 as a product on the tensor cores: member masks expanded to a 0/1 bf16 matrix times
-//      the staged K (V) rows, fp32 accumulation, one multiply by 1/|S|, one rounding to bf16; the
-//      cores are compacted in place in shared memory and leave with 16-byte coalesced stores.
-//      Meanwhile the service warp looks back; it draws the block's next ticket during step 2.
+//   5. Eq. 3, beside the service warp's look-back: every token belongs to exactly one cluster, so the
+//      warp that clustered a segment sums each cluster's member rows (fp32, token order; a lane owns
+//      eight columns of the K or of the V row), scales by 1/|S|, rounds once to bf16 and overwrites
+//      the seed's staged row; clusters of one token are left as they are.  The cores then leave in
+//      seed order with 16-byte coalesced stores.  The service warp draws the block's next ticket
+//      during step 2.
 // The last block to finish zeroes the status words and counters, so a workspace that was zero
 // before the call is zero again after it.
 #include <cuda.h>
-#include <cstdlib>
 
 #include "common.cuh"
 
@@ -136,9 +135,6 @@ __device__ __forceinline__ uint32_t tile_addr(int row, int chunk) { return row *
 __device__ __forceinline__ void compute_warps_sync() {   // the eight compute warps, not the service warp
     asm volatile("bar.sync 1, 256;\n" ::: "memory");
 }
-__device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;\n" ::"l"(src), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -168,10 +164,6 @@ __device__ __forceinline__ uint32_t ld_volatile(const uint32_t* p) {
 __device__ __forceinline__ int adj_row(int i) {
     const int k = i >> 5;
     return 256 * k - 16 * k * (k - 1) + (i & 31) * (kNW - k);
-}
-// Two mask bits -> two bf16 (0.0 or 1.0) packed as an mma operand register.
-__device__ __forceinline__ uint32_t expand2(uint32_t two_bits) {
-    return ((two_bits * 0x8001u) & 0x00010001u) * 0x3F80u;
 }
 
 // 32x32 block of K.K^T: rows of block rb against rows of block cb (column halves `hs` bytes apart).
@@ -264,16 +256,37 @@ __device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int
 __constant__ uint8_t kOffDiag[28] = {0x01, 0x12, 0x23, 0x34, 0x45, 0x56, 0x67, 0x02, 0x13, 0x24, 0x35, 0x46, 0x57, 0x03,
                                      0x14, 0x25, 0x36, 0x47, 0x04, 0x15, 0x26, 0x37, 0x05, 0x16, 0x27, 0x06, 0x17, 0x07};
 
+// Eq. 3 building blocks.  A lane owns eight consecutive columns (one 16-byte chunk) of the K row
+// (lanes 0-15) or of the V row (lanes 16-31); `lane_base` is its tensor and column half, c7 its
+// chunk inside the half.  Sums are fp32, in token order.
+__device__ __forceinline__ void row_add(const unsigned char* lane_base, int row, int c7, float (&s)[8]) {
+    const uint4 v = *reinterpret_cast<const uint4*>(lane_base + tile_addr(row, c7));
+    s[0] += __uint_as_float(v.x << 16); s[1] += __uint_as_float(v.x & 0xffff0000u);
+    s[2] += __uint_as_float(v.y << 16); s[3] += __uint_as_float(v.y & 0xffff0000u);
+    s[4] += __uint_as_float(v.z << 16); s[5] += __uint_as_float(v.z & 0xffff0000u);
+    s[6] += __uint_as_float(v.w << 16); s[7] += __uint_as_float(v.w & 0xffff0000u);
+}
+__device__ __forceinline__ void row_put_mean(unsigned char* lane_base, int row, int c7, const float (&s)[8], float inv) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(s[0] * inv, s[1] * inv), b = __floats2bfloat162_rn(s[2] * inv, s[3] * inv);
+    __nv_bfloat162 c = __floats2bfloat162_rn(s[4] * inv, s[5] * inv), d = __floats2bfloat162_rn(s[6] * inv, s[7] * inv);
+    uint4 v;
+    v.x = *reinterpret_cast<uint32_t*>(&a); v.y = *reinterpret_cast<uint32_t*>(&b);
+    v.z = *reinterpret_cast<uint32_t*>(&c); v.w = *reinterpret_cast<uint32_t*>(&d);
+    *reinterpret_cast<uint4*>(lane_base + tile_addr(row, c7)) = v;
+}
+
 // Eq. 2 + Algorithm 1 for one segment of 2..32 tokens, by one warp, in registers.
 // Rows [a, a + l) of the staged keys.  The upper triangle of the segment's own Gram matrix comes
 // from mma tiles laid over the segment's rows (16-row tiles down, 8-column tiles across, only
 // those that reach above the diagonal); lane 4g + t ends up owning row g + 8t with its adjacency
 // bits (later tokens only) in one word, and the greedy pass is a handful of word operations and
-// one shuffle per seed.  Results: seed bits into the tile's seedmask, each seed's member mask into
-// its (tile-relative) adjacency row for the Eq. 3 product, optionally the seed of every token.
+// one shuffle per seed.  Results: seed bits into the tile's seedmask and, for pool_short_segment,
+// in `seeds` (bit i = token a + i is a seed) with the seed's member mask in `mymem` of the lane
+// that owns the seed (0 elsewhere); optionally the seed of every token.
 template <bool kNegTau>
 __device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int hs, int a, int l, float tau, float* nrm /*[32], this warp's*/,
-                                                  uint32_t* adj, uint32_t* seedmask, int32_t* as, int row0, int lane) {
+                                                  uint32_t* seedmask, int32_t* as, int row0, int lane, uint32_t& seeds,
+                                                  uint32_t& mymem) {
     const int g = lane >> 2, tig = lane & 3;
     const int nnt = (l + 7) >> 3;          // 8-column tiles that hold tokens: 1..4
     const bool two_mt = l > 16;
@@ -358,8 +371,10 @@ __device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int hs, int a,
     uint32_t mine = (tig & 2) ? ((tig & 1) ? wrow[1][1] : wrow[1][0]) : ((tig & 1) ? wrow[0][1] : wrow[0][0]);
     mine &= (0xfffffffeu << own) & lowmask;   // later tokens of the segment only
     // Algorithm 1
-    uint32_t U = lowmask, seeds = 0u, mymem = 0u;
+    uint32_t U = lowmask;
     int seed_of = 0;
+    seeds = 0u;
+    mymem = 0u;
     while (U) {
         const int i = __ffs(U) - 1;                      // lowest unassigned token: a seed
         const int src = ((i & 7) << 2) | (i >> 3);
@@ -375,18 +390,30 @@ __device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int hs, int a,
         atomicOr(&seedmask[w0], seeds << sh);
         if (sh != 0 && (seeds >> (32 - sh)) != 0u) atomicOr(&seedmask[w0 + 1], seeds >> (32 - sh));
     }
-    if (mymem != 0u) {
-        const int i = a + own;
-        const uint32_t lo = mymem << sh, hi = sh ? (mymem >> (32 - sh)) : 0u;
-        uint32_t* row = adj + adj_row(i);
-        if ((i >> 5) == w0) {
-            row[0] = lo;
-            if (((a + l - 1) >> 5) > w0) row[1] = hi;
-        } else {
-            row[0] = hi;
-        }
-    }
     if (as != nullptr && own < l) as[a + own] = row0 + a + seed_of;
+}
+
+// Eq. 3 for the clusters of a segment of 2..32 tokens starting at row a, from what gsc_short_segment
+// left in `seeds` and `mymem`.  Every token belongs to exactly one cluster, so a cluster's mean can
+// overwrite its seed's staged row once its members are summed; a cluster of one is left as it is.
+// cnts[seed row] receives the member count.
+__device__ __forceinline__ void pool_short_segment(unsigned char* lane_base, uint16_t* cnts, int a, uint32_t seeds,
+                                                   uint32_t mymem, int lane) {
+    const int c7 = lane & 7;
+    while (seeds) {
+        const int i = __ffs(seeds) - 1;
+        seeds &= seeds - 1;
+        uint32_t mem = __shfl_sync(kFull, mymem, ((i & 7) << 2) | (i >> 3));
+        const int cnt = __popc(mem);
+        if (lane == 0) cnts[a + i] = (uint16_t)cnt;
+        if (cnt == 1) continue;
+        float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        while (mem) {
+            row_add(lane_base, a + __ffs(mem) - 1, c7, sum);
+            mem &= mem - 1;
+        }
+        row_put_mean(lane_base, a + i, c7, sum, 1.0f / (float)cnt);
+    }
 }
 
 struct Params {
@@ -400,8 +427,6 @@ struct Params {
     uint32_t* tile_state;    // [B*Hkv][n_tile_cap]
     int32_t* status;
     CUtensorMap map_k, map_v;   // [B, Hkv, n, 128] bf16, boxes of 16 rows x 64 columns, 128-byte swizzle
-    int ahead_rows;          // L2 prefetch distance in rows; 0 = the cache is not one contiguous [B*Hkv*n, d] array
-    int64_t total_rows;      // B*Hkv*n
 };
 
 
@@ -454,73 +479,35 @@ __device__ __forceinline__ void stage_rows(uint32_t dst, int hs, const CUtensorM
     }
 }
 
-// Eq. 3 on the tensor cores for one staged tensor (K or V rows at `area`, column halves hs bytes apart).
-// Cluster c (in seed order) has its member mask in the adjacency row of its seed seedrow[c].  A
-// warp owns one tile of 16 clusters (mt_in_round of a round of mts_per_round tiles) and one half
-// of the 128 columns:  acc[16 x 64] = mask[16 x rows] . rows[rows x 64].
-// The scaled, rounded cores overwrite rows [0, P) of the same area: cluster c only reads rows >=
-// its seed >= c, rounds go up in c, and inside a round every warp has finished reading before any
-// of them writes.  cnts[c] receives the cluster's member count (from the warps told to write it).
-__device__ __forceinline__ void merge_rounds(uint32_t area, unsigned char* area_ptr, int hs, int half, int mt_in_round,
-                                             int mts_per_round, int P, const uint16_t* seedrow, const uint16_t* send,
-                                             const uint32_t* adj, int lane, uint16_t* cnts /*or null*/) {
-    const int g = lane >> 2, tig = lane & 3;
-    // the warp's 64 columns are exactly one column half; chunk 2*np + c of it, rows k0 + (0..15), k0 % 16 == 0
-    const uint32_t b_lane = area + half * hs + tile_addr((lane & 7) + ((lane >> 3) & 1) * 8, lane >> 4);
-    for (int c0 = 0; c0 < P; c0 += 16 * mts_per_round) {
-        const int cbase = c0 + 16 * mt_in_round;
-        const bool active = cbase < P;
-        const bool ok_lo = cbase + g < P, ok_hi = cbase + g + 8 < P;
-        float acc[8][4];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-        int cnt0 = 0, cnt1 = 0;
-        if (active) {
-            int lo0 = 0, hi0 = -2, lo1 = 0, hi1 = -2;
-            const uint32_t* r0 = adj;
-            const uint32_t* r1 = adj;
-            if (ok_lo) { const int i0 = seedrow[cbase + g]; lo0 = i0 >> 5; hi0 = ((int)send[i0] - 1) >> 5; r0 = adj + adj_row(i0) - lo0; }
-            if (ok_hi) { const int i1 = seedrow[cbase + g + 8]; lo1 = i1 >> 5; hi1 = ((int)send[i1] - 1) >> 5; r1 = adj + adj_row(i1) - lo1; }
-            const int w_first = (int)seedrow[cbase] >> 5;
-            const int w_last = ((int)send[seedrow[min(cbase + 15, P - 1)]] - 1) >> 5;
-            for (int w = w_first; w <= w_last; ++w) {
-                const uint32_t m0w = (w >= lo0 && w <= hi0) ? r0[w] : 0u;
-                const uint32_t m1w = (w >= lo1 && w <= hi1) ? r1[w] : 0u;
-                cnt0 += __popc(m0w);
-                cnt1 += __popc(m1w);
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const uint32_t m0 = (m0w >> (16 * hh + 2 * tig)), m1 = (m1w >> (16 * hh + 2 * tig));
-                    if (!__any_sync(kFull, ((m0 | m1) & 0x0303u) != 0u)) continue;
-                    const uint32_t a0 = expand2(m0 & 3u), a2 = expand2((m0 >> 8) & 3u);
-                    const uint32_t a1 = expand2(m1 & 3u), a3 = expand2((m1 >> 8) & 3u);
-                    const uint32_t b_addr = b_lane + (w * 32 + hh * 16) * kHalfRow;
-#pragma unroll
-                    for (int np = 0; np < 4; ++np) {
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4_trans(b_addr ^ (np << 5), b0, b1, b2, b3);
-                        mma_bf16(acc[2 * np], a0, a1, a2, a3, b0, b1);
-                        mma_bf16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+// Eq. 3 for the clusters of one segment of more than 32 tokens [a, e), whose seeds are marked in
+// seedmask and whose member masks sit in the seeds' adjacency rows.  The compute warps take the
+// clusters in turn; as everywhere, a mean overwrites its seed's staged row.  `lanes` is 32 when K
+// and V are both staged, 16 when only one tensor is (a tile longer than SC_TILE_ROWS).
+__device__ __forceinline__ void merge_long_segment(unsigned char* lane_base, int a, int e, const uint32_t* seedmask,
+                                                   const uint32_t* adj, uint16_t* cnts /*or null*/, int warp, int lane,
+                                                   int lanes) {
+    const int c7 = lane & 7, w_end = (e - 1) >> 5;
+    int turn = 0;
+    for (int w = a >> 5; w <= w_end; ++w) {
+        uint32_t sb = seedmask[w] & bits_between(a, e, w);
+        while (sb) {
+            const int i = w * 32 + __ffs(sb) - 1;
+            sb &= sb - 1;
+            if ((turn++ & (kWarps - 1)) != warp) continue;
+            const uint32_t* row = adj + adj_row(i) - (i >> 5);
+            float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            int cnt = 0;
+            for (int ww = i >> 5; ww <= w_end; ++ww) {
+                uint32_t mem = row[ww];
+                cnt += __popc(mem);
+                if (lane < lanes)
+                    while (mem) {
+                        row_add(lane_base, ww * 32 + __ffs(mem) - 1, c7, sum);
+                        mem &= mem - 1;
                     }
-                }
             }
-        }
-        compute_warps_sync();   // every compute warp has read what it needs of rows [c0, ...)
-        if (active) {
-            const float inv0 = 1.0f / (float)max(cnt0, 1), inv1 = 1.0f / (float)max(cnt1, 1);
-            // rows cbase + g and cbase + g + 8 both have (row & 7) == g: chunk nt lands at chunk nt ^ g
-            unsigned char* o_lo = area_ptr + half * hs + (cbase + g) * kHalfRow + tig * 4;
-            unsigned char* o_hi = o_lo + 8 * kHalfRow;
-#pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                const int o = (nt ^ g) << 4;
-                if (ok_lo) *reinterpret_cast<__nv_bfloat162*>(o_lo + o) = __floats2bfloat162_rn(acc[nt][0] * inv0, acc[nt][1] * inv0);
-                if (ok_hi) *reinterpret_cast<__nv_bfloat162*>(o_hi + o) = __floats2bfloat162_rn(acc[nt][2] * inv1, acc[nt][3] * inv1);
-            }
-            if (cnts != nullptr && tig == 0) {
-                if (ok_lo) cnts[cbase + g] = (uint16_t)cnt0;
-                if (ok_hi) cnts[cbase + g + 8] = (uint16_t)cnt1;
-            }
+            if (cnts != nullptr && lane == 0) cnts[i] = (uint16_t)cnt;
+            if (cnt > 1 && lane < lanes) row_put_mean(lane_base, i, c7, sum, 1.0f / (float)cnt);
         }
     }
 }
@@ -586,14 +573,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
             if (two_tensors) stage_rows(sbase + kVOff, hs, &p.map_v, row0, R, h, b, bar_v, lane);
         }
         CF_T(1);
-        if (p.ahead_rows > 0 && tid == 64) {   // contiguous cache: tickets advance in memory order
-            const int64_t first = (int64_t)bh * p.n + row0 + p.ahead_rows;
-            const int64_t rows = min((int64_t)R, p.total_rows - first);
-            if (rows > 0) {
-                l2_prefetch(p.K + first * kD, (uint32_t)rows * kRowBytes);
-                if (kMode != kCountOnly) l2_prefetch(p.V + first * kD, (uint32_t)rows * kRowBytes);
-            }
-        }
         // end of the segment each row is in (0 past the tile)
         // also: one-token segments (delimiters, lone tokens) are clusters of their own -- no key needed;
         // the others are listed for the warps
@@ -607,21 +586,26 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a == 1) {
                     send[a] = (uint16_t)e;
-                    adj[adj_row(a)] = 1u << (a & 31);
+                    cnts[a] = (uint16_t)1;
                     atomicOr(&seedmask[a >> 5], 1u << (a & 31));
                     if (as) as[a] = row0 + a;
                     continue;
                 }
                 multi[atomicAdd(&misc[3], 1)] = (uint8_t)s;
-                for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
-                if (e - a > 32)
+                if (e - a > 32) {   // only the long-segment path reads send[] (of every row of the blocks it touches)
+                    for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
                     for (int k = a >> 5; k <= (e - 1) >> 5; ++k) { atomicOr(&misc[2], 1 << k); atomicMax(&reach[k], (e - 1) >> 5); }
+                }
             }
         }
         for (int r = R + tid; r < nrb * 32; r += kThreads) send[r] = (uint16_t)0;
         CF_T(0);
         failed = !mbar_wait(bar_k, phase_k);   // K has landed
         phase_k ^= 1u;
+        if (two_tensors && !failed) {
+            failed = !mbar_wait(bar_v, phase_v);   // and V
+            phase_v ^= 1u;
+        }
         if (__syncthreads_or(failed)) { failed = true; break; }
         CF_T(2);
 
@@ -652,6 +636,9 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
 
         // ---- 3. the service warp draws the block's next ticket; compute warps: Algorithm 1 per segment,
         //         one warp each, in registers up to 32 tokens, else on the bit rows ----
+        unsigned char* lane_base = smem + (lane >> 4) * kVOff + ((lane >> 3) & 1) * hs;   // see row_add
+        int keep_a[2] = {0, 0};
+        uint32_t keep_seeds[2] = {0u, 0u}, keep_mem[2] = {0u, 0u};
         if (service) {
             CF_SPAN_BEGIN();
             fetch_tile(p, lane, dec_b, dec_pref, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
@@ -663,8 +650,14 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 const int s = multi[k];
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a <= 32) {
-                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
-                    else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 32, adj, seedmask, as, row0, lane);
+                    uint32_t seeds, mymem;
+                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 32, seedmask, as, row0, lane, seeds, mymem);
+                    else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 32, seedmask, as, row0, lane, seeds, mymem);
+                    if (kMode == kCountOnly) continue;
+                    // Eq. 3 waits for the next phase (beside the look-back); a warp's third segment and up is pooled now
+                    if (k == warp) { keep_a[0] = a; keep_seeds[0] = seeds; keep_mem[0] = mymem; }
+                    else if (k == warp + kWarps) { keep_a[1] = a; keep_seeds[1] = seeds; keep_mem[1] = mymem; }
+                    else pool_short_segment(lane_base, cnts, a, seeds, mymem, lane);
                     continue;
                 }
                 const int w1 = (e - 1) >> 5;
@@ -695,7 +688,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         __syncthreads();
         CF_T(5);
 
-        // ---- 4. cluster count of the tile; publish it; seed row of every cluster ----
+        // ---- 4. cluster count of the tile, published at once.  Service warp: output offset of the tile
+        //         (look-back).  Compute warps: the seed row of every cluster, and Eq. 3 ----
         int P = 0;
 #pragma unroll
         for (int w = 0; w < kNW; ++w) P += __popc(seedmask[w]);
@@ -703,33 +697,30 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         if (kMode == kCountOnly) {
             if (tid == 0) stt[t] = (uint32_t)P;
         } else {
-            if (kMode == kLookBack && tid == 0)
-                atomicExch(&stt[t], (t == 0 ? kFlagPrefix : kFlagAggregate) | (uint32_t)P);
-            if (tid < R) {
-                const uint32_t wbits = seedmask[tid >> 5];
-                if ((wbits >> (tid & 31)) & 1u) {
-                    int rank = __popc(wbits & ((1u << (tid & 31)) - 1u));
-                    for (int w = 0; w < (tid >> 5); ++w) rank += __popc(seedmask[w]);
-                    seedrow[rank] = (uint16_t)tid;
-                }
-            }
-            if (two_tensors) {
-                failed = !mbar_wait(bar_v, phase_v);   // V has landed
-                phase_v ^= 1u;
-            }
-            if (__syncthreads_or(failed)) { failed = true; break; }
-            CF_T(6);
-
-            // ---- 5. compute warps: Eq. 3 (tile of 16 clusters x tensor x column half each);
-            //         service warp: output offset of the tile ----
             if (!service) {
-                if (long_tile) merge_rounds(sbase, smem, hs, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane,
-                                            (warp & 1) == 0 ? cnts : nullptr);
-                else merge_rounds(sbase + (warp & 1) * kVOff, smem + (warp & 1) * kVOff, hs, (warp >> 1) & 1, warp >> 2, 2, P,
-                                  seedrow, send, adj, lane, (warp & 3) == 0 ? cnts : nullptr);
+                if (tid < R) {
+                    const uint32_t wbits = seedmask[tid >> 5];
+                    if ((wbits >> (tid & 31)) & 1u) {
+                        int rank = __popc(wbits & ((1u << (tid & 31)) - 1u));
+                        for (int w = 0; w < (tid >> 5); ++w) rank += __popc(seedmask[w]);
+                        seedrow[rank] = (uint16_t)tid;
+                    }
+                }
+#pragma unroll
+                for (int q = 0; q < 2; ++q) pool_short_segment(lane_base, cnts, keep_a[q], keep_seeds[q], keep_mem[q], lane);
+                if (longblocks != 0) {
+                    const int nmulti = misc[3];
+                    for (int k = 0; k < nmulti; ++k) {
+                        const int s = multi[k];
+                        const int a = segs[s], e = segs[s + 1];
+                        if (e - a > 32) merge_long_segment(lane_base, a, e, seedmask, adj, cnts, warp, lane, long_tile ? 16 : 32);
+                    }
+                }
                 CF_T(7);
             } else {
                 CF_SPAN_BEGIN();
+                if (kMode == kLookBack && lane == 0)
+                    atomicExch(&stt[t], (t == 0 ? kFlagPrefix : kFlagAggregate) | (uint32_t)P);
                 int base = 0;
                 if (kMode == kWriteWithCounts) {
                     for (int k = lane; k < t; k += 32) base += (int)stt[k];
@@ -785,23 +776,23 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
             __syncthreads();
             CF_T(8);
 
-            // ---- compact, coalesced stores of the cores ----
+            // ---- compact, coalesced stores of the cores: cluster `row` of the tile sits in its seed's staged row ----
             const int base = misc[0];
             const size_t obase = (size_t)bh * p.cap;
             for (int idx = tid; idx < P * 16; idx += kThreads) {
                 const int row = idx >> 4, c = idx & 15;
                 if (base + row < p.cap) {
                     const size_t o = (obase + base + row) * kD + c * 8;
-                    const unsigned char* src = smem + (c >> 3) * hs + tile_addr(row, c & 7);
+                    const unsigned char* src = smem + (c >> 3) * hs + tile_addr(seedrow[row], c & 7);
                     *reinterpret_cast<uint4*>(p.core_k + o) = *reinterpret_cast<const uint4*>(src);
                     if (!long_tile) *reinterpret_cast<uint4*>(p.core_v + o) = *reinterpret_cast<const uint4*>(src + kVOff);
                 }
             }
             for (int row = tid; row < P; row += kThreads)
                 if (base + row < p.cap)
-                    p.count[obase + base + row] = (int32_t)cnts[row];
+                    p.count[obase + base + row] = (int32_t)cnts[seedrow[row]];
 
-            // ---- a long segment: V takes the place of K and goes through the same product ----
+            // ---- a tile longer than SC_TILE_ROWS: V takes the place of K and is pooled with the same masks ----
             if (long_tile) {
                 fence_async_proxy();   // the copies below overwrite what ordinary accesses read and wrote
                 __syncthreads();
@@ -809,13 +800,13 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 failed = !mbar_wait(bar_v, phase_v);
                 phase_v ^= 1u;
                 if (__syncthreads_or(failed)) { failed = true; break; }
-                if (!service) merge_rounds(sbase, smem, hs, warp & 1, warp >> 1, 4, P, seedrow, send, adj, lane, nullptr);
+                if (!service) merge_long_segment(lane_base, 0, R, seedmask, adj, nullptr, warp, lane, 16);
                 __syncthreads();
                 for (int idx = tid; idx < P * 16; idx += kThreads) {
                     const int row = idx >> 4, c = idx & 15;
                     if (base + row < p.cap)
                         *reinterpret_cast<uint4*>(p.core_v + (obase + base + row) * kD + c * 8) =
-                            *reinterpret_cast<const uint4*>(smem + (c >> 3) * hs + tile_addr(row, c & 7));
+                            *reinterpret_cast<const uint4*>(smem + (c >> 3) * hs + tile_addr(seedrow[row], c & 7));
                 }
             }
         }
@@ -933,13 +924,6 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
     // no more blocks than there can be tiles
     const int64_t max_tiles = (int64_t)a.B * a.Hkv * a.n_tile_cap;
     const int grid = (int)(max_tiles < grid_of[dev] ? max_tiles : grid_of[dev]);
-    // prefetch distance: the rows all resident blocks hold together
-    const bool contiguous = a.st.n == cf::kD && a.st.h == (int64_t)a.n * cf::kD && a.st.b == (int64_t)a.Hkv * a.n * cf::kD;
-    p.ahead_rows = contiguous ? grid * SC_TILE_ROWS : 0;
-    p.total_rows = (int64_t)a.B * a.Hkv * a.n;
-#ifdef SC_TUNE   // tuning harness only
-    if (const char* e = getenv("SC_CF_AHEAD")) p.ahead_rows = contiguous ? atoi(e) : 0;
-#endif
     if (a.flags & SC_FLAG_TWO_PASS) {
         cf::Params pc = p;
         pc.assign = nullptr;
