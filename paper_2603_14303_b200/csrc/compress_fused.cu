@@ -52,8 +52,8 @@ constexpr int kHalfLong = kMaxRows * kHalfRow;    // 32768: ... of a long one
 constexpr int kCntOff = kKvBytes;                 // uint16[256]: members of each cluster
 constexpr int kAdjOff = kCntOff + kMaxRows * 2;
 constexpr int kAdjWords = 32 * (8 + 7 + 6 + 5 + 4 + 3 + 2 + 1);   // rows of block k keep words k..7
-constexpr int kNormOff = kAdjOff + kAdjWords * 4; // float[256]; later uint16 seed row per cluster
-constexpr int kSendOff = kNormOff + kMaxRows * 4; // uint16[256]: end of the segment a row is in
+constexpr int kNormOff = kAdjOff + kAdjWords * 4; // float[512]: norms (64 per warp, or one per row); later uint16 seed row per cluster
+constexpr int kSendOff = kNormOff + kWarps * 64 * 4; // uint16[256]: end of the segment a row is in
 constexpr int kSegsOff = kSendOff + kMaxRows * 2; // 2 x int16[132]: segment starts (this tile, next tile)
 constexpr int kSegsStride = 132;
 constexpr int kMiscOff = kSegsOff + 2 * kSegsStride * 2;   // uint32 seedmask[8]; int geo[2][8]; int misc[4]
@@ -479,13 +479,91 @@ __device__ __forceinline__ void stage_rows(uint32_t dst, int hs, const CUtensorM
     }
 }
 
+// Eq. 2 for one segment of 33..64 tokens [a, a + l), by one warp on its own (no block-level step):
+// the upper triangle of the segment's Gram matrix in 16-row bands, last band first so that the
+// norms a band needs (its own rows', from its diagonal, and those of all later rows) are known
+// when it is thresholded.  Every row's adjacency bits (later tokens of the segment) go to its
+// words of the tile's bit rows, where the greedy pass for longer segments reads them.
+template <bool kNegTau>
+__device__ __forceinline__ void gram_mid_segment(uint32_t kbase, int hs, int a, int l, float tau, float* nrm /*[64], this warp's*/,
+                                                 uint32_t* adj, int lane) {
+    const int g = lane >> 2, tig = lane & 3;
+    const int nnt = (l + 7) >> 3, nmt = (l + 15) >> 4;   // 5..8 column tiles, 3..4 row bands
+    const int j = lane >> 3, r8 = lane & 7;
+    const int sh = a & 31, wb = a >> 5, w_end = (a + l - 1) >> 5;
+#pragma unroll
+    for (int mt = 3; mt >= 0; --mt) {
+        if (mt >= nmt) continue;
+        float acc[8][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+        const uint32_t a_base = kbase + tile_addr(a + mt * 16 + r8 + ((j & 1) << 3), j >> 1);
+        const uint32_t b_base = kbase + tile_addr(a + r8 + ((j >> 1) << 3), j & 1);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t kx = (ks & 3) << 5, ko = (ks >> 2) * hs;
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4((a_base ^ kx) + ko, a0, a1, a2, a3);
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                if (np < mt || 2 * np >= nnt) continue;   // left of the band's diagonal, or past the segment
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4((b_base ^ kx) + ko + np * 16 * kHalfRow, b0, b1, b2, b3);
+                mma_bf16(acc[2 * np], a0, a1, a2, a3, b0, b1);
+                if (2 * np + 1 < nnt) mma_bf16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
+            }
+        }
+        if ((g >> 1) == tig) {   // the band's own norms, from its diagonal
+            const int e = g & 1;
+            nrm[mt * 16 + g] = sqrtf(e ? acc[2 * mt][1] : acc[2 * mt][0]);
+            nrm[mt * 16 + 8 + g] = sqrtf(e ? acc[2 * mt + 1][3] : acc[2 * mt + 1][2]);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int i = mt * 16 + hh * 8 + g;        // token of the segment
+            const float ni = nrm[i];
+            uint32_t lo = 0u, hi = 0u;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                if (nt < 2 * mt + hh || nt >= nnt) continue;
+                const float2 nn = *reinterpret_cast<const float2*>(nrm + nt * 8 + 2 * tig);
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const float thr = ni * (tau * (e ? nn.y : nn.x));
+                    bool hit = acc[nt][hh * 2 + e] > thr;
+                    if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
+                    if (hit) { if (nt < 4) lo |= 1u << (nt * 8 + e); else hi |= 1u << ((nt - 4) * 8 + e); }
+                }
+            }
+            lo <<= 2 * tig; hi <<= 2 * tig;
+            lo |= __shfl_xor_sync(kFull, lo, 1); hi |= __shfl_xor_sync(kFull, hi, 1);
+            lo |= __shfl_xor_sync(kFull, lo, 2); hi |= __shfl_xor_sync(kFull, hi, 2);
+            if (tig == 0 && i < l) {
+                // later tokens of the segment only: bits (i, l)
+                const unsigned long long keep = (i >= 63 ? 0ull : (~0ull << (i + 1))) & (l >= 64 ? ~0ull : ((1ull << l) - 1ull));
+                const unsigned long long m = (((unsigned long long)hi << 32) | lo) & keep;
+                // to tile positions: shift by a; row a + i keeps words (a + i) >> 5 .. w_end
+                const uint32_t t0 = (uint32_t)(m << sh), t1 = (uint32_t)((m << sh) >> 32),
+                               t2 = sh ? (uint32_t)((m >> 32) >> (32 - sh)) : 0u;
+                const int wi = (a + i) >> 5;
+                uint32_t* row = adj + adj_row(a + i) - wi;
+                if (wb >= wi) row[wb] = t0;
+                if (wb + 1 >= wi && wb + 1 <= w_end) row[wb + 1] = t1;
+                if (wb + 2 >= wi && wb + 2 <= w_end) row[wb + 2] = t2;
+            }
+        }
+        __syncwarp();
+    }
+}
+
 // Eq. 3 for the clusters of one segment of more than 32 tokens [a, e), whose seeds are marked in
 // seedmask and whose member masks sit in the seeds' adjacency rows.  The compute warps take the
-// clusters in turn; as everywhere, a mean overwrites its seed's staged row.  `lanes` is 32 when K
+// clusters in turn (or one warp takes them all); as everywhere, a mean overwrites its seed's staged row.  `lanes` is 32 when K
 // and V are both staged, 16 when only one tensor is (a tile longer than SC_TILE_ROWS).
 __device__ __forceinline__ void merge_long_segment(unsigned char* lane_base, int a, int e, const uint32_t* seedmask,
-                                                   const uint32_t* adj, uint16_t* cnts /*or null*/, int warp, int lane,
-                                                   int lanes) {
+                                                   const uint32_t* adj, uint16_t* cnts /*or null*/, int warp /*-1: every cluster*/,
+                                                   int lane, int lanes) {
     const int c7 = lane & 7, w_end = (e - 1) >> 5;
     int turn = 0;
     for (int w = a >> 5; w <= w_end; ++w) {
@@ -493,7 +571,7 @@ __device__ __forceinline__ void merge_long_segment(unsigned char* lane_base, int
         while (sb) {
             const int i = w * 32 + __ffs(sb) - 1;
             sb &= sb - 1;
-            if ((turn++ & (kWarps - 1)) != warp) continue;
+            if (warp >= 0 && (turn++ & (kWarps - 1)) != warp) continue;
             const uint32_t* row = adj + adj_row(i) - (i >> 5);
             float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
             int cnt = 0;
@@ -579,7 +657,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         int32_t* as = p.assign ? p.assign + (size_t)bh * p.n + row0 : nullptr;
         if (nseg == 1 && R > 1) {
             for (int r = tid; r < R; r += kThreads) send[r] = (uint16_t)R;
-            if (R > 32 && tid < nrb) { atomicOr(&misc[2], 1 << tid); reach[tid] = nrb - 1; }
+            if (R > 64 && tid < nrb) { atomicOr(&misc[2], 1 << tid); reach[tid] = nrb - 1; }
             if (tid == 0) { multi[0] = 0; misc[3] = 1; }
         } else {
             for (int s = tid; s < nseg; s += kThreads) {
@@ -592,7 +670,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                     continue;
                 }
                 multi[atomicAdd(&misc[3], 1)] = (uint8_t)s;
-                if (e - a > 32) {   // only the long-segment path reads send[] (of every row of the blocks it touches)
+                if (e - a > 64) {   // only the block-level path reads send[] (of every row of the blocks it touches)
                     for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
                     for (int k = a >> 5; k <= (e - 1) >> 5; ++k) { atomicOr(&misc[2], 1 << k); atomicMax(&reach[k], (e - 1) >> 5); }
                 }
@@ -609,7 +687,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         if (__syncthreads_or(failed)) { failed = true; break; }
         CF_T(2);
 
-        // ---- 2. segments of more than 32 tokens: Gram blocks -> norms -> adjacency bits in shared memory ----
+        // ---- 2. segments of more than 64 tokens: Gram blocks -> norms -> adjacency bits in shared memory ----
         const int longblocks = misc[2];
         if (longblocks != 0) {
             float acc[2][4][4];
@@ -651,14 +729,18 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a <= 32) {
                     uint32_t seeds, mymem;
-                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 32, seedmask, as, row0, lane, seeds, mymem);
-                    else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 32, seedmask, as, row0, lane, seeds, mymem);
+                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, as, row0, lane, seeds, mymem);
+                    else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, as, row0, lane, seeds, mymem);
                     if (kMode == kCountOnly) continue;
                     // Eq. 3 waits for the next phase (beside the look-back); a warp's third segment and up is pooled now
                     if (k == warp) { keep_a[0] = a; keep_seeds[0] = seeds; keep_mem[0] = mymem; }
                     else if (k == warp + kWarps) { keep_a[1] = a; keep_seeds[1] = seeds; keep_mem[1] = mymem; }
                     else pool_short_segment(lane_base, cnts, a, seeds, mymem, lane);
                     continue;
+                }
+                if (e - a <= 64) {   // the warp builds the segment's bit rows itself
+                    if (p.tau < 0.f) gram_mid_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 64, adj, lane);
+                    else gram_mid_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 64, adj, lane);
                 }
                 const int w1 = (e - 1) >> 5;
                 uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
@@ -708,12 +790,13 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 }
 #pragma unroll
                 for (int q = 0; q < 2; ++q) pool_short_segment(lane_base, cnts, keep_a[q], keep_seeds[q], keep_mem[q], lane);
-                if (longblocks != 0) {
+                {   // segments of more than 32 tokens: 33..64 by the warp that clustered them, longer ones shared
                     const int nmulti = misc[3];
                     for (int k = 0; k < nmulti; ++k) {
                         const int s = multi[k];
                         const int a = segs[s], e = segs[s + 1];
-                        if (e - a > 32) merge_long_segment(lane_base, a, e, seedmask, adj, cnts, warp, lane, long_tile ? 16 : 32);
+                        if (e - a > 64) merge_long_segment(lane_base, a, e, seedmask, adj, cnts, warp, lane, long_tile ? 16 : 32);
+                        else if (e - a > 32 && (k & (kWarps - 1)) == warp) merge_long_segment(lane_base, a, e, seedmask, adj, cnts, -1, lane, 32);
                     }
                 }
                 CF_T(7);
