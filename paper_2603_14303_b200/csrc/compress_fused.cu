@@ -430,28 +430,30 @@ struct Params {
 };
 
 
-// Warp 0 draws the next ticket, turns it into a tile (sequence, head, tile index, rows) and copies
-// the tile's segment starts into shared memory.  Tickets walk the tiles of head 0 of sequence 0 in
-// order, then head 1, ...; a block's tickets only grow, so the sequence it last decoded (dec_b,
-// with dec_pref tickets before it) is where the search resumes.  geo[gT] = -1 when no work is left.
-__device__ __forceinline__ void fetch_tile(const Params& p, int lane, int& dec_b, int& dec_pref, int* geo,
-                                           int16_t* segs) {
-    int w = 0;
-    if (lane == 0) w = atomicAdd(&p.ctl[0], 1);
-    w = __shfl_sync(kFull, w, 0);
-    int nt = 0;
-    while (dec_b < p.B) {
-        nt = min(p.seq_tile_cnt[dec_b], p.n_tile_cap);
-        const int span = p.Hkv * nt;
-        if (w < dec_pref + span) break;
-        dec_pref += span;
-        ++dec_b;
+// The service warp draws the next ticket, turns it into a tile (sequence, head, tile index, rows) and
+// copies the tile's segment starts into shared memory.  Tickets go round the (sequence, head) pairs:
+// ticket w is tile w / (B*Hkv) of pair w % (B*Hkv), so consecutive tiles of one head are B*Hkv
+// tickets apart and a tile's predecessor has usually published its cluster count (and often its
+// prefix) by the time the tile looks back.  A pair with fewer tiles skips its surplus tickets.
+// geo[gT] = -1 when no work is left (max_nt = most tiles any sequence has).
+__device__ __forceinline__ void fetch_tile(const Params& p, int lane, int max_nt, int* geo, int16_t* segs) {
+    const int pairs = p.B * p.Hkv;
+    int b, h, t, nt;
+    for (;;) {
+        int w = 0;
+        if (lane == 0) w = atomicAdd(&p.ctl[0], 1);
+        w = __shfl_sync(kFull, w, 0);
+        t = w / pairs;
+        if (t >= max_nt) {
+            if (lane == 0) geo[gT] = -1;
+            return;
+        }
+        const int bh = w - t * pairs;
+        b = bh / p.Hkv;
+        h = bh - b * p.Hkv;
+        nt = min(p.seq_tile_cnt[b], p.n_tile_cap);
+        if (t < nt) break;
     }
-    if (dec_b >= p.B) {
-        if (lane == 0) geo[gT] = -1;
-        return;
-    }
-    const int r = w - dec_pref, h = r / nt, t = r - h * nt, b = dec_b;
     const int32_t* ts = p.tile_seg + (size_t)b * (p.n_tile_cap + 1);
     const int s_begin = ts[t], s_end = ts[t + 1];
     const int nseg = max(min(s_end - s_begin, kShortRows), 1);
@@ -611,7 +613,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool service = warp == kWarps;   // the ninth warp
-    int dec_b = 0, dec_pref = 0;           // ticket decoding state (service warp)
+    int max_nt = 0;                        // most tiles any sequence has (service warp)
 
     if (tid == 0) {
         mbar_init(bar_k, 1);
@@ -623,7 +625,11 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     uint32_t phase_k = 0, phase_v = 0;
     bool failed = false;
 
-    if (service) fetch_tile(p, lane, dec_b, dec_pref, geo_buf, segs_buf);
+    if (service) {
+        for (int b = lane; b < p.B; b += 32) max_nt = max(max_nt, min(p.seq_tile_cnt[b], p.n_tile_cap));
+        max_nt = warp_max_i(max_nt);
+        fetch_tile(p, lane, max_nt, geo_buf, segs_buf);
+    }
     if (tid < kNW) reach[tid] = 0;
     if (tid == kNW) misc[2] = misc[3] = 0;
     if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
@@ -719,7 +725,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         uint32_t keep_seeds[2] = {0u, 0u}, keep_mem[2] = {0u, 0u};
         if (service) {
             CF_SPAN_BEGIN();
-            fetch_tile(p, lane, dec_b, dec_pref, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
+            fetch_tile(p, lane, max_nt, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
             CF_SPAN_END(10);
         } else {
             CF_SPAN_BEGIN();
