@@ -49,8 +49,8 @@ constexpr int kKvBytes = kMaxRows * kRowBytes;    // 65536: short = K | V, long 
 constexpr int kVOff = kShortRows * kRowBytes;     // 32768
 constexpr int kHalfShort = kShortRows * kHalfRow; // 16384: distance between the column halves of a short tile
 constexpr int kHalfLong = kMaxRows * kHalfRow;    // 32768: ... of a long one
-constexpr int kCntOff = kKvBytes;                 // uint16[256]: members of each cluster
-constexpr int kAdjOff = kCntOff + kMaxRows * 2;
+constexpr int kCntOff = kKvBytes;                 // uint32[256] per seed row: what pool_clusters needs, then the member count
+constexpr int kAdjOff = kCntOff + kMaxRows * 4;
 constexpr int kAdjWords = 32 * (8 + 7 + 6 + 5 + 4 + 3 + 2 + 1);   // rows of block k keep words k..7
 constexpr int kNormOff = kAdjOff + kAdjWords * 4; // float[512]: norms (64 per warp, or one per row); later uint16 seed row per cluster
 constexpr int kSendOff = kNormOff + kWarps * 64 * 4; // uint16[256]: end of the segment a row is in
@@ -88,6 +88,9 @@ __device__ unsigned long long g_phase_cycles[16];
 #define CF_SPAN_END(i)
 #endif
 
+// cnts[seed row] while the cluster waits to be pooled: kPending | first row of its segment | (one past its last
+// row) << 9, the latter 0 for a segment of up to 32 tokens, whose member mask is one segment-relative word
+constexpr uint32_t kPending = 1u << 31;
 constexpr uint32_t kFlagAggregate = 1u << 30, kFlagPrefix = 2u << 30, kValueMask = (1u << 30) - 1;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every wait gives up after 2 s
 constexpr int kPollGroups = 4;                               // the look-back reads 128 predecessors per poll
@@ -259,12 +262,28 @@ __constant__ uint8_t kOffDiag[28] = {0x01, 0x12, 0x23, 0x34, 0x45, 0x56, 0x67, 0
 // Eq. 3 building blocks.  A lane owns eight consecutive columns (one 16-byte chunk) of the K row
 // (lanes 0-15) or of the V row (lanes 16-31); `lane_base` is its tensor and column half, c7 its
 // chunk inside the half.  Sums are fp32, in token order.
-__device__ __forceinline__ void row_add(const unsigned char* lane_base, int row, int c7, float (&s)[8]) {
-    const uint4 v = *reinterpret_cast<const uint4*>(lane_base + tile_addr(row, c7));
+__device__ __forceinline__ void add_chunk(const uint4& v, float (&s)[8]) {
     s[0] += __uint_as_float(v.x << 16); s[1] += __uint_as_float(v.x & 0xffff0000u);
     s[2] += __uint_as_float(v.y << 16); s[3] += __uint_as_float(v.y & 0xffff0000u);
     s[4] += __uint_as_float(v.z << 16); s[5] += __uint_as_float(v.z & 0xffff0000u);
     s[6] += __uint_as_float(v.w << 16); s[7] += __uint_as_float(v.w & 0xffff0000u);
+}
+// Adds the rows first + j for every set bit j of mem, in order; two loads are kept in flight (the
+// filler of an odd count is a row of zeros, which leaves the sums as they are).
+__device__ __forceinline__ void rows_add(const unsigned char* lane_base, int first, uint32_t mem, int c7, float (&s)[8]) {
+    while (mem) {
+        const int j0 = __ffs(mem) - 1;
+        mem &= mem - 1;
+        const uint4 v0 = *reinterpret_cast<const uint4*>(lane_base + tile_addr(first + j0, c7));
+        uint4 v1 = make_uint4(0u, 0u, 0u, 0u);
+        if (mem) {
+            const int j1 = __ffs(mem) - 1;
+            mem &= mem - 1;
+            v1 = *reinterpret_cast<const uint4*>(lane_base + tile_addr(first + j1, c7));
+        }
+        add_chunk(v0, s);
+        add_chunk(v1, s);
+    }
 }
 __device__ __forceinline__ void row_put_mean(unsigned char* lane_base, int row, int c7, const float (&s)[8], float inv) {
     __nv_bfloat162 a = __floats2bfloat162_rn(s[0] * inv, s[1] * inv), b = __floats2bfloat162_rn(s[2] * inv, s[3] * inv);
@@ -280,13 +299,13 @@ __device__ __forceinline__ void row_put_mean(unsigned char* lane_base, int row, 
 // from mma tiles laid over the segment's rows (16-row tiles down, 8-column tiles across, only
 // those that reach above the diagonal); lane 4g + t ends up owning row g + 8t with its adjacency
 // bits (later tokens only) in one word, and the greedy pass is a handful of word operations and
-// one shuffle per seed.  Results: seed bits into the tile's seedmask and, for pool_short_segment,
-// in `seeds` (bit i = token a + i is a seed) with the seed's member mask in `mymem` of the lane
-// that owns the seed (0 elsewhere); optionally the seed of every token.
+// one shuffle per seed.  Results: seed bits into the tile's seedmask; for pool_clusters each seed's
+// member mask (bit j = token a + j) in the first word of its adjacency row and a note in cnts;
+// optionally the seed of every token.
 template <bool kNegTau>
 __device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int hs, int a, int l, float tau, float* nrm /*[32], this warp's*/,
-                                                  uint32_t* seedmask, int32_t* as, int row0, int lane, uint32_t& seeds,
-                                                  uint32_t& mymem) {
+                                                  uint32_t* seedmask, uint32_t* adj, uint32_t* cnts, int32_t* as, int row0,
+                                                  int lane) {
     const int g = lane >> 2, tig = lane & 3;
     const int nnt = (l + 7) >> 3;          // 8-column tiles that hold tokens: 1..4
     const bool two_mt = l > 16;
@@ -371,10 +390,8 @@ __device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int hs, int a,
     uint32_t mine = (tig & 2) ? ((tig & 1) ? wrow[1][1] : wrow[1][0]) : ((tig & 1) ? wrow[0][1] : wrow[0][0]);
     mine &= (0xfffffffeu << own) & lowmask;   // later tokens of the segment only
     // Algorithm 1
-    uint32_t U = lowmask;
+    uint32_t U = lowmask, seeds = 0u, mymem = 0u;
     int seed_of = 0;
-    seeds = 0u;
-    mymem = 0u;
     while (U) {
         const int i = __ffs(U) - 1;                      // lowest unassigned token: a seed
         const int src = ((i & 7) << 2) | (i >> 3);
@@ -390,29 +407,49 @@ __device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int hs, int a,
         atomicOr(&seedmask[w0], seeds << sh);
         if (sh != 0 && (seeds >> (32 - sh)) != 0u) atomicOr(&seedmask[w0 + 1], seeds >> (32 - sh));
     }
+    if (mymem != 0u) {
+        adj[adj_row(a + own)] = mymem;
+        cnts[a + own] = kPending | (uint32_t)a;
+    }
     if (as != nullptr && own < l) as[a + own] = row0 + a + seed_of;
 }
 
-// Eq. 3 for the clusters of a segment of 2..32 tokens starting at row a, from what gsc_short_segment
-// left in `seeds` and `mymem`.  Every token belongs to exactly one cluster, so a cluster's mean can
-// overwrite its seed's staged row once its members are summed; a cluster of one is left as it is.
-// cnts[seed row] receives the member count.
-__device__ __forceinline__ void pool_short_segment(unsigned char* lane_base, uint16_t* cnts, int a, uint32_t seeds,
-                                                   uint32_t mymem, int lane) {
+// Eq. 3 for the tile's clusters, dealt to the compute warps in seed order.  Every token belongs to
+// exactly one cluster, so a cluster's mean can overwrite its seed's staged row once its members are
+// summed (fp32, token order); a cluster of one is left as it is.  cnts[seed row] ends up holding the
+// member count.  `lanes` is 32 when K and V are both staged, 16 when only K is.
+__device__ __forceinline__ void pool_clusters(unsigned char* lane_base, const uint32_t* seedmask, int nrb, const uint32_t* adj,
+                                              uint32_t* cnts, int warp, int lane, int lanes) {
     const int c7 = lane & 7;
-    while (seeds) {
-        const int i = __ffs(seeds) - 1;
-        seeds &= seeds - 1;
-        uint32_t mem = __shfl_sync(kFull, mymem, ((i & 7) << 2) | (i >> 3));
-        const int cnt = __popc(mem);
-        if (lane == 0) cnts[a + i] = (uint16_t)cnt;
-        if (cnt == 1) continue;
-        float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        while (mem) {
-            row_add(lane_base, a + __ffs(mem) - 1, c7, sum);
-            mem &= mem - 1;
+    int turn = 0;
+    for (int w = 0; w < nrb; ++w) {
+        uint32_t sb = seedmask[w];
+        while (sb) {
+            const int i = w * 32 + __ffs(sb) - 1;
+            sb &= sb - 1;
+            if ((turn++ & (kWarps - 1)) != warp) continue;
+            const uint32_t info = cnts[i];
+            if (!(info & kPending)) continue;   // a one-token segment: settled when the tile was staged
+            const int a = info & 511, e = (info >> 9) & 511;
+            float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            int cnt;
+            if (e == 0) {   // up to 32 tokens: one word, relative to the segment
+                uint32_t mem = adj[adj_row(i)];
+                cnt = __popc(mem);
+                if (cnt > 1 && lane < lanes) rows_add(lane_base, a, mem, c7, sum);
+            } else {        // longer: the row's words, at tile positions
+                const uint32_t* row = adj + adj_row(i) - (i >> 5);
+                cnt = 0;
+                for (int ww = i >> 5; ww <= (e - 1) >> 5; ++ww) {
+                    const uint32_t mem = row[ww];
+                    cnt += __popc(mem);
+                    if (lane < lanes) rows_add(lane_base, ww * 32, mem, c7, sum);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) cnts[i] = (uint32_t)cnt;
+            if (cnt > 1 && lane < lanes) row_put_mean(lane_base, i, c7, sum, 1.0f / (float)cnt);
         }
-        row_put_mean(lane_base, a + i, c7, sum, 1.0f / (float)cnt);
     }
 }
 
@@ -559,13 +596,10 @@ __device__ __forceinline__ void gram_mid_segment(uint32_t kbase, int hs, int a, 
     }
 }
 
-// Eq. 3 for the clusters of one segment of more than 32 tokens [a, e), whose seeds are marked in
-// seedmask and whose member masks sit in the seeds' adjacency rows.  The compute warps take the
-// clusters in turn (or one warp takes them all); as everywhere, a mean overwrites its seed's staged row.  `lanes` is 32 when K
-// and V are both staged, 16 when only one tensor is (a tile longer than SC_TILE_ROWS).
+// The same for the second tensor of a tile longer than SC_TILE_ROWS (V staged where K was): one
+// segment [a, e), seeds in seedmask, member masks in the seeds' adjacency rows, counts already known.
 __device__ __forceinline__ void merge_long_segment(unsigned char* lane_base, int a, int e, const uint32_t* seedmask,
-                                                   const uint32_t* adj, uint16_t* cnts /*or null*/, int warp /*-1: every cluster*/,
-                                                   int lane, int lanes) {
+                                                   const uint32_t* adj, int warp, int lane, int lanes) {
     const int c7 = lane & 7, w_end = (e - 1) >> 5;
     int turn = 0;
     for (int w = a >> 5; w <= w_end; ++w) {
@@ -573,20 +607,15 @@ __device__ __forceinline__ void merge_long_segment(unsigned char* lane_base, int
         while (sb) {
             const int i = w * 32 + __ffs(sb) - 1;
             sb &= sb - 1;
-            if (warp >= 0 && (turn++ & (kWarps - 1)) != warp) continue;
+            if ((turn++ & (kWarps - 1)) != warp) continue;
             const uint32_t* row = adj + adj_row(i) - (i >> 5);
             float sum[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
             int cnt = 0;
             for (int ww = i >> 5; ww <= w_end; ++ww) {
-                uint32_t mem = row[ww];
+                const uint32_t mem = row[ww];
                 cnt += __popc(mem);
-                if (lane < lanes)
-                    while (mem) {
-                        row_add(lane_base, ww * 32 + __ffs(mem) - 1, c7, sum);
-                        mem &= mem - 1;
-                    }
+                if (lane < lanes) rows_add(lane_base, ww * 32, mem, c7, sum);
             }
-            if (cnts != nullptr && lane == 0) cnts[i] = (uint16_t)cnt;
             if (cnt > 1 && lane < lanes) row_put_mean(lane_base, i, c7, sum, 1.0f / (float)cnt);
         }
     }
@@ -595,7 +624,7 @@ __device__ __forceinline__ void merge_long_segment(unsigned char* lane_base, int
 template <int kMode>
 __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __grid_constant__ Params p) {
     extern __shared__ __align__(1024) unsigned char smem[];   // the swizzle pattern repeats every 1024 bytes
-    uint16_t* cnts = reinterpret_cast<uint16_t*>(smem + kCntOff);
+    uint32_t* cnts = reinterpret_cast<uint32_t*>(smem + kCntOff);
     uint32_t* adj = reinterpret_cast<uint32_t*>(smem + kAdjOff);
     float* norm = reinterpret_cast<float*>(smem + kNormOff);
     uint16_t* seedrow = reinterpret_cast<uint16_t*>(smem + kNormOff);   // reuses the norms once they are spent
@@ -670,7 +699,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a == 1) {
                     send[a] = (uint16_t)e;
-                    cnts[a] = (uint16_t)1;
+                    cnts[a] = 1u;
                     atomicOr(&seedmask[a >> 5], 1u << (a & 31));
                     if (as) as[a] = row0 + a;
                     continue;
@@ -721,8 +750,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         // ---- 3. the service warp draws the block's next ticket; compute warps: Algorithm 1 per segment,
         //         one warp each, in registers up to 32 tokens, else on the bit rows ----
         unsigned char* lane_base = smem + (lane >> 4) * kVOff + ((lane >> 3) & 1) * hs;   // see row_add
-        int keep_a[2] = {0, 0};
-        uint32_t keep_seeds[2] = {0u, 0u}, keep_mem[2] = {0u, 0u};
         if (service) {
             CF_SPAN_BEGIN();
             fetch_tile(p, lane, max_nt, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
@@ -734,14 +761,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 const int s = multi[k];
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a <= 32) {
-                    uint32_t seeds, mymem;
-                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, as, row0, lane, seeds, mymem);
-                    else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, as, row0, lane, seeds, mymem);
-                    if (kMode == kCountOnly) continue;
-                    // Eq. 3 waits for the next phase (beside the look-back); a warp's third segment and up is pooled now
-                    if (k == warp) { keep_a[0] = a; keep_seeds[0] = seeds; keep_mem[0] = mymem; }
-                    else if (k == warp + kWarps) { keep_a[1] = a; keep_seeds[1] = seeds; keep_mem[1] = mymem; }
-                    else pool_short_segment(lane_base, cnts, a, seeds, mymem, lane);
+                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
+                    else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
                     continue;
                 }
                 if (e - a <= 64) {   // the warp builds the segment's bit rows itself
@@ -759,7 +780,11 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                     if (lane >= wf && lane <= w1) {
                         uint32_t* slot = adj + adj_row(i) + (lane - wf);
                         uint32_t mem = *slot & U;
-                        if (lane == wf) { mem |= 1u << (i & 31); seeds |= 1u << (i & 31); }
+                        if (lane == wf) {
+                            mem |= 1u << (i & 31);
+                            seeds |= 1u << (i & 31);
+                            cnts[i] = kPending | (uint32_t)a | ((uint32_t)e << 9);
+                        }
                         *slot = mem;            // the row now lists the cluster's members
                         U &= ~mem;
                         if (as) {
@@ -794,17 +819,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                         seedrow[rank] = (uint16_t)tid;
                     }
                 }
-#pragma unroll
-                for (int q = 0; q < 2; ++q) pool_short_segment(lane_base, cnts, keep_a[q], keep_seeds[q], keep_mem[q], lane);
-                {   // segments of more than 32 tokens: 33..64 by the warp that clustered them, longer ones shared
-                    const int nmulti = misc[3];
-                    for (int k = 0; k < nmulti; ++k) {
-                        const int s = multi[k];
-                        const int a = segs[s], e = segs[s + 1];
-                        if (e - a > 64) merge_long_segment(lane_base, a, e, seedmask, adj, cnts, warp, lane, long_tile ? 16 : 32);
-                        else if (e - a > 32 && (k & (kWarps - 1)) == warp) merge_long_segment(lane_base, a, e, seedmask, adj, cnts, -1, lane, 32);
-                    }
-                }
+                pool_clusters(lane_base, seedmask, nrb, adj, cnts, warp, lane, long_tile ? 16 : 32);
                 CF_T(7);
             } else {
                 CF_SPAN_BEGIN();
@@ -889,7 +904,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 failed = !mbar_wait(bar_v, phase_v);
                 phase_v ^= 1u;
                 if (__syncthreads_or(failed)) { failed = true; break; }
-                if (!service) merge_long_segment(lane_base, 0, R, seedmask, adj, nullptr, warp, lane, 16);
+                if (!service) merge_long_segment(lane_base, 0, R, seedmask, adj, warp, lane, 16);
                 __syncthreads();
                 for (int idx = tid; idx < P * 16; idx += kThreads) {
                     const int row = idx >> 4, c = idx & 15;
