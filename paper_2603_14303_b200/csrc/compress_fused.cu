@@ -414,20 +414,16 @@ __device__ __forceinline__ void gsc_short_segment(uint32_t kbase, int hs, int a,
     if (as != nullptr && own < l) as[a + own] = row0 + a + seed_of;
 }
 
-// Eq. 3 for the tile's clusters, dealt to the compute warps in seed order.  Every token belongs to
+// Eq. 3 for the tile's P clusters (seedrow[c] = seed row of cluster c), dealt to the compute warps in turn.  Every token belongs to
 // exactly one cluster, so a cluster's mean can overwrite its seed's staged row once its members are
 // summed (fp32, token order); a cluster of one is left as it is.  cnts[seed row] ends up holding the
 // member count.  `lanes` is 32 when K and V are both staged, 16 when only K is.
-__device__ __forceinline__ void pool_clusters(unsigned char* lane_base, const uint32_t* seedmask, int nrb, const uint32_t* adj,
+__device__ __forceinline__ void pool_clusters(unsigned char* lane_base, const uint16_t* seedrow, int P, const uint32_t* adj,
                                               uint32_t* cnts, int warp, int lane, int lanes) {
     const int c7 = lane & 7;
-    int turn = 0;
-    for (int w = 0; w < nrb; ++w) {
-        uint32_t sb = seedmask[w];
-        while (sb) {
-            const int i = w * 32 + __ffs(sb) - 1;
-            sb &= sb - 1;
-            if ((turn++ & (kWarps - 1)) != warp) continue;
+    {
+        for (int c = warp; c < P; c += kWarps) {
+            const int i = seedrow[c];
             const uint32_t info = cnts[i];
             if (!(info & kPending)) continue;   // a one-token segment: settled when the tile was staged
             const int a = info & 511, e = (info >> 9) & 511;
@@ -819,7 +815,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                         seedrow[rank] = (uint16_t)tid;
                     }
                 }
-                pool_clusters(lane_base, seedmask, nrb, adj, cnts, warp, lane, long_tile ? 16 : 32);
+                compute_warps_sync();   // the table of seed rows is complete
+                pool_clusters(lane_base, seedrow, P, adj, cnts, warp, lane, long_tile ? 16 : 32);
                 CF_T(7);
             } else {
                 CF_SPAN_BEGIN();
