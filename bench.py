@@ -110,15 +110,17 @@ class Pipeline:
                                                torch.empty((w.B, w.Hkv, self.cap, w.d), dtype=dt, device=device),
                                                torch.zeros((w.B, w.Hkv, self.cap), **i32),
                                                torch.zeros((w.B, w.Hkv), **i32)) for _ in range(w.L)]
-        self.cws = binding.compress_workspace(w.B, w.Hkv, w.n, device)
-        # one workspace per layer: consecutive layer launches overlap and must not share scratch
+        # one workspace per layer (both stages): consecutive layer launches overlap and must not share scratch
+        self.cws = [binding.compress_workspace(w.B, w.Hkv, w.n, device) for _ in range(w.L)]
         self.dws = [binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, self.cap, device) for _ in range(w.L)]
         self.q = torch.stack([torch.stack([synth.queries(w, s, l, device) for l in range(w.L)])
                               for s in range(w.decode_steps)])            # [steps, L, B, Hq, d]
         self.out = torch.empty_like(self.q)
         self.plan = None
         self.decode_flags = 0
+        self.compress_flags = 0
         self.status = torch.zeros((w.L, 1), **i32)
+        self.cstatus = torch.zeros((w.L, 1), **i32)
         self.launches_compress = self.launches_decode = 0
         self.g_compress = self.g_decode = None
 
@@ -133,7 +135,11 @@ class Pipeline:
             b.sc_chunk(self.ids_dev, w.delims, w.max_chunk_len, p.seg_off, p.seq_seg_off, p.n_seg, p.tile_seg,
                        p.seq_tile_cnt, self._chunk_ws, p.status)
         for l in range(w.L):
-            b.compress(self.K[l], self.V[l], self.plan, w.tau, cap=self.cap, workspace=self.cws, out=self.layers[l])
+            # layer 0 follows sc_chunk and needs its plan; the other layers share nothing they write with
+            # their predecessor (own K/V, cores, workspace, status) and may overlap its tail
+            ly = self.layers[l]
+            b.sc_compress(self.K[l], self.V[l], self.plan, w.tau, ly.core_k, ly.core_v, ly.count, ly.core_len, None,
+                          self.cws[l], self.cstatus[l], self.compress_flags if l > 0 else 0)
 
     def run_decode(self):
         b, w = self.b, self.w
@@ -149,6 +155,8 @@ class Pipeline:
         self.run_decode()
         torch.cuda.synchronize(self.dev)
         self.b.check_status(self.plan.status, "warm-up pass")
+        if int(self.cstatus.abs().max().item()) != 0:
+            raise RuntimeError("sc_compress reported a device-side error in the warm-up pass")
         self.g_compress, self.g_decode = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
         c0 = self.b.launch_counter()
         with torch.cuda.graph(self.g_compress):
@@ -192,6 +200,7 @@ def run_ours(args):
     pipe = Pipeline(w, dev)
     # the per-layer decode calls of a step are independent (own q, out, workspace): let them overlap
     pipe.decode_flags = 0 if args.no_overlap else binding.SC_FLAG_OVERLAP_PREV
+    pipe.compress_flags = pipe.decode_flags
     pipe.capture()
     cbytes, dbytes, per_layer, kept = pipe.algorithmic_bytes()
 
@@ -221,8 +230,8 @@ def run_ours(args):
     t_wall = time.perf_counter() - t_wall
     clocks = sampler.stop() if rank == 0 else None
     binding.check_status(pipe.plan.status, "timed region")
-    if int(pipe.status.abs().max().item()) != 0:
-        raise RuntimeError("sc_decode_attn reported a device-side error")
+    if int(pipe.status.abs().max().item()) != 0 or int(pipe.cstatus.abs().max().item()) != 0:
+        raise RuntimeError("sc_compress / sc_decode_attn reported a device-side error")
     ms_c = [e[0].elapsed_time(e[1]) for e in ev]
     ms_d = [e[1].elapsed_time(e[2]) for e in ev]
     total_ms = ev[0][0].elapsed_time(ev[-1][2])

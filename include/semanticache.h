@@ -54,7 +54,8 @@ typedef enum { SC_BF16 = 0, SC_F32 = 1 } sc_dtype;
 #define SC_FLAG_GENERIC 1u     /* force the generic (CUDA-core, any dtype) kernels */
 #define SC_FLAG_TWO_PASS 2u    /* fused compress: count pass + write pass instead of the
                                   single pass whose tiles look back for their output offset */
-#define SC_FLAG_OVERLAP_PREV 4u /* sc_decode_attn: launch with programmatic stream serialization and
+#define SC_FLAG_OVERLAP_PREV 4u /* sc_decode_attn, sc_compress (fused bf16 path, single pass): launch with
+                                  programmatic stream serialization and
                                   do not wait for the kernel enqueued just before on this stream.
                                   The caller promises that that kernel and this call share no
                                   buffer that either of them writes (q, out, workspace, status and

@@ -640,6 +640,9 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     const bool service = warp == kWarps;   // the ninth warp
     int max_nt = 0;                        // most tiles any sequence has (service warp)
 
+    // Let the next kernel of the stream start beside this one if it was launched with programmatic stream
+    // serialization (a no-op otherwise); this kernel itself never waits for its predecessor.
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     if (tid == 0) {
         mbar_init(bar_k, 1);
         mbar_init(bar_v, 1);
@@ -1032,8 +1035,21 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
         cf::compress_fused_kernel<cf::kWriteWithCounts><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
         note_launches(2);
     } else {
-        cf::compress_fused_kernel<cf::kLookBack><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
+        // With SC_FLAG_OVERLAP_PREV the kernel may start while the one enqueued before it on the stream is
+        // still draining (the caller has promised they share nothing either writes): the tail of one
+        // layer's persistent blocks then overlaps the start of the next layer's.
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(cf::kThreads);
+        cfg.dynamicSmemBytes = cf::kSmemBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = (a.flags & SC_FLAG_OVERLAP_PREV) ? 1 : 0;
         note_launches(1);
+        return cudaLaunchKernelEx(&cfg, cf::compress_fused_kernel<cf::kLookBack>, p);
     }
     return cudaGetLastError();
 }

@@ -267,6 +267,38 @@ def test_compress_workspace_is_left_clean_and_can_be_shared_by_consecutive_calls
             assert int(ws.view(torch.int32)[:n_words].abs().max()) == 0, "status words and counters are zero again"
 
 
+def test_compress_overlapped_independent_layer_launches_match_ordinary_ones():
+    """SC_FLAG_OVERLAP_PREV on sc_compress: layers with their own K/V, cores, workspace and status, launched
+    back to back so that one layer's tail overlaps the next layer's start."""
+    w = synth.config(1, n=8192, L=4)
+    ids, run_id, run_lens = synth.token_ids(w)
+    plan = binding.chunk(ids.to(DEV), w.delims)
+    KV = [tuple(x.to(DEV) for x in synth.layer_kv(w, l, run_id, run_lens)) for l in range(w.L)]
+    refs = [oracle_compress(ids, KV[l][0].cpu(), KV[l][1].cpu(), w.delims, w.tau) for l in range(w.L)]
+    ws = [binding.compress_workspace(w.B, w.Hkv, w.n, DEV) for _ in range(w.L)]
+    st = torch.zeros((w.L, 1), dtype=torch.int32, device=DEV)
+    outs = [None] * w.L
+    torch.cuda.synchronize()
+    for rep in range(3):
+        for l in range(w.L):
+            if outs[l] is None:
+                outs[l] = binding.compress(KV[l][0], KV[l][1], plan, w.tau, workspace=ws[l])   # allocates once
+                continue
+            o = outs[l]
+            o.core_k.zero_(); o.core_len.zero_()
+        torch.cuda.synchronize()
+        for l in range(w.L):
+            o = outs[l]
+            binding.sc_compress(KV[l][0], KV[l][1], plan, w.tau, o.core_k, o.core_v, o.count, o.core_len, None, ws[l], st[l],
+                                binding.SC_FLAG_OVERLAP_PREV if l > 0 else 0)
+        torch.cuda.synchronize()
+        assert int(st.abs().max()) == 0
+        for l in range(w.L):
+            compare_compressed(outs[l], refs[l], torch.bfloat16, check_assign=False)
+            n_words = 64 + w.B * w.Hkv * plan.n_tile_cap
+            assert int(ws[l].view(torch.int32)[:n_words].abs().max()) == 0
+
+
 # ---------------------------------------------------------------------------- sc_decode_attn
 
 
