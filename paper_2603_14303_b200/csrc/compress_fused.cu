@@ -4,7 +4,7 @@
 // counter.  A tile is a run of whole segments of at most SC_TILE_ROWS tokens of one (sequence, KV
 // head) -- K and V both staged in shared memory -- or one longer segment alone (K staged, then V
 // in a second pass over the same buffer).  Per tile:
-//   1. the rows are staged by TMA (cp.async.bulk.tensor, boxes of 16 rows x 64 columns, 128-byte
+//   1. the rows are staged by TMA (cp.async.bulk.tensor, boxes of 32 rows x 64 columns, 128-byte
 //      swizzle so that ldmatrix is conflict free, completion on an mbarrier), issued by the block's
 //      ninth "service" warp;
 //   2. Eq. 2 + Algorithm 1, one warp per segment.  Up to 32 tokens (the usual case) everything
@@ -40,8 +40,8 @@ constexpr int kThreads = (kWarps + 1) * 32;       // plus one service warp: next
 constexpr int kD = 128;
 constexpr int kRowBytes = 256;                    // one K or V row in global memory
 constexpr int kHalfRow = 128;                     // a staged row is two 128-byte halves (64 columns each), see tile_addr
-constexpr int kBoxRows = 16;                      // rows per TMA box
-constexpr int kBoxBytes = kBoxRows * kHalfRow;    // 2048
+constexpr int kBoxRows = 32;                      // rows per TMA box
+constexpr int kBoxBytes = kBoxRows * kHalfRow;    // 4096
 constexpr int kMaxRows = SC_MAX_CHUNK_LEN;        // 256: a long tile
 constexpr int kShortRows = SC_TILE_ROWS;          // 128
 constexpr int kNW = 8;                            // 32-bit words per (full) adjacency row
@@ -125,7 +125,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (global_ns() - t0 > kWaitLimitNs) return false;
     }
 }
-// One TMA box: 16 rows x 64 columns of a [B, Hkv, n, 128] tensor, 128-byte swizzled, no multicast.
+// One TMA box: 32 rows x 64 columns of a [B, Hkv, n, 128] tensor, 128-byte swizzled, no multicast.
 __device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* map, int col, int row, int h, int b, uint32_t bar) {
     asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
                  ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(col), "r"(row), "r"(h), "r"(b), "r"(bar) : "memory");
@@ -459,7 +459,7 @@ struct Params {
     int32_t* ctl;            // [0] ticket counter, [1] blocks finished
     uint32_t* tile_state;    // [B*Hkv][n_tile_cap]
     int32_t* status;
-    CUtensorMap map_k, map_v;   // [B, Hkv, n, 128] bf16, boxes of 16 rows x 64 columns, 128-byte swizzle
+    CUtensorMap map_k, map_v;   // [B, Hkv, n, 128] bf16, boxes of 32 rows x 64 columns, 128-byte swizzle
 };
 
 
@@ -499,8 +499,8 @@ __device__ __forceinline__ void fetch_tile(const Params& p, int lane, int max_nt
     }
 }
 
-// Stages rows [row0, row0 + R) of head (b, h) of one tensor with TMA: one box of 16 rows x 64 columns
-// per lane (R <= 256 needs at most 32 boxes for both column halves), the halves `hs` bytes apart at
+// Stages rows [row0, row0 + R) of head (b, h) of one tensor with TMA: one box of 32 rows x 64 columns
+// per lane (R <= 256 needs at most 16 boxes for both column halves), the halves `hs` bytes apart at
 // `dst`.  Rows past R inside the last box are the cache's next rows, or zeros past the end of the
 // sequence: finite either way, and they only ever enter the Eq. 3 product with weight 0.
 __device__ __forceinline__ void stage_rows(uint32_t dst, int hs, const CUtensorMap* map, int row0, int R, int h, int b,
@@ -969,7 +969,7 @@ EncodeTiledFn encode_tiled() {
     return fn;
 }
 
-// [B, Hkv, n, 128] bf16 with element strides st, read in boxes of 16 rows x 64 columns.
+// [B, Hkv, n, 128] bf16 with element strides st, read in boxes of 32 rows x 64 columns.
 bool make_map(CUtensorMap* map, const void* base, const sc_strides& st, int B, int Hkv, int n) {
     EncodeTiledFn enc = encode_tiled();
     if (enc == nullptr) return false;
