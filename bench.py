@@ -34,6 +34,11 @@ from paper_2603_14303_b200 import synth  # noqa: E402
 METRIC = "compressed_kv_decode_tokens_per_s"
 UNIT = "tokens/s"
 
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/, by workload:
+# sc_decode_attn (decode_mma_kernel_cfg1_8layers.md) and sc_compress (compress_fused_kernel_cfg1_8layers.md).
+# Only valid while those kernels are the ones that were captured; other workloads report null.
+NCU_TRAFFIC = {"cfg1-llama3-8b-32k": {"decode": 34.31e6, "compress": 153.3e6}}
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -271,7 +276,14 @@ def run_ours(args):
         "roofline": {"kernel": "sc_decode_attn (one layer per launch)", "bound": "hbm", "achieved": achieved,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8tbs": achieved / 8000.0, "bytes_per_launch": layer_bytes,
-                     "us_per_launch": dec_launch_us, "traffic": args.traffic},
+                     "us_per_launch": dec_launch_us,
+                     "traffic": args.traffic if args.traffic is not None else
+                     NCU_TRAFFIC.get(w.name, {}).get("decode")},
+        "roofline_compress": {"kernel": "sc_compress (one layer per launch)", "bound": "hbm", "achieved": comp_gbs,
+                              "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": comp_gbs / peak,
+                              "frac_of_nominal_8tbs": comp_gbs / 8000.0, "bytes_per_launch": cbytes / w.L,
+                              "us_per_launch": comp_ms * 1e3 / w.L,
+                              "traffic": NCU_TRAFFIC.get(w.name, {}).get("compress")},
         "gpu_launches": args.steps * (pipe.launches_compress + pipe.launches_decode),
         "gpu_launches_per_step": {"chunk+compress": pipe.launches_compress, "decode": pipe.launches_decode},
         "clocks": clocks, "e2e": e2e, "wall_s": t_wall,
