@@ -251,6 +251,15 @@ def test_compress_near_ties_are_decided_consistently():
     compare_compressed(got, dict(core_k=ck, core_v=cv, count=cnt, core_len=clen, assign=assign), torch.bfloat16)
 
 
+@pytest.mark.parametrize("n", [1, 5, 31, 33, 130])
+def test_compress_tiny_contexts(n):
+    """Contexts shorter than a TMA box / a tile, two sequences and heads."""
+    w = synth.config(0, B=2, n=n, Hkv=2, Hq=8, gap=("poisson", 6.0), centroids=("uniform", 3), seed=n)
+    ref, got, plan, _ = _compress_both(w)
+    binding.check_status(plan.status)
+    compare_compressed(got, ref, torch.bfloat16)
+
+
 def test_compress_workspace_is_left_clean_and_can_be_shared_by_consecutive_calls():
     w = synth.config(0, n=6000, L=3, gap=("poisson", 40.0))
     ids, run_id, run_lens = synth.token_ids(w)
