@@ -771,11 +771,10 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 const int w1 = (e - 1) >> 5;
                 uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
                 uint32_t seeds = 0u;
-                for (;;) {
-                    const uint32_t any = __ballot_sync(kFull, U != 0u);
-                    if (any == 0u) break;
-                    const int wf = __ffs(any) - 1;
-                    const int i = wf * 32 + __ffs(__shfl_sync(kFull, U, wf)) - 1;   // lowest unassigned token: a seed
+                for (int wf = a >> 5; wf <= w1;) {   // wf: first word that may still hold unassigned tokens
+                    const uint32_t u = __shfl_sync(kFull, U, wf);
+                    if (u == 0u) { ++wf; continue; }
+                    const int i = wf * 32 + __ffs(u) - 1;   // lowest unassigned token: a seed
                     if (lane >= wf && lane <= w1) {
                         uint32_t* slot = adj + adj_row(i) + (lane - wf);
                         uint32_t mem = *slot & U;
