@@ -12,19 +12,22 @@
 //      triangle of its Gram matrix (bf16 products are exact in fp32), the diagonal gives the norms,
 //      Sim > tau is decided as G_ij > tau*|k_i|*|k_j|, each lane ends up with one row's adjacency
 //      word, and the greedy pass costs one shuffle and a few word operations per seed;
-//   3. longer segments go through 32x32 Gram blocks for exactly the block pairs they span, with the
-//      adjacency bits in shared memory (an upper triangle of 32-bit words per row) and one lane
-//      per word in the greedy pass; either way a seed's row ends up holding its member mask;
+//   3. a segment of 33..64 tokens is still one warp's own business: it builds the bit rows of the
+//      segment in 16-row bands in shared memory and runs the greedy pass on them; beyond 64 tokens
+//      the Gram matrix is cut into 32x32 blocks (exactly the block pairs the segment spans) that all
+//      warps share, and one warp runs the greedy pass with one lane per 32-token word.  The
+//      adjacency bits live in an upper triangle of 32-bit words per row; a seed's row ends up
+//      holding its member mask;
 //   4. the tile's cluster count enters a prefix sum over the tiles of its (sequence, head): a
 //      decoupled look-back over per-tile status words (tickets are handed out in order, so every
 //      predecessor is held by a running block and the bounded wait cannot starve), or, in
 //      two-pass mode, a count pass followed by a write pass;
-//   5. Eq. 3, beside the service warp's look-back: every token belongs to exactly one cluster, so the
-//      warp that clustered a segment sums each cluster's member rows (fp32, token order; a lane owns
-//      eight columns of the K or of the V row), scales by 1/|S|, rounds once to bf16 and overwrites
-//      the seed's staged row; clusters of one token are left as they are.  The cores then leave in
-//      seed order with 16-byte coalesced stores.  The service warp draws the block's next ticket
-//      during step 2.
+//   5. Eq. 3, beside the service warp's look-back: every token belongs to exactly one cluster, so a
+//      cluster's mean can overwrite its seed's staged row.  The clusters are dealt to the compute
+//      warps in seed order; a lane owns eight columns of the K or of the V row, sums the member
+//      rows in fp32 in token order, scales by 1/|S| and rounds once to bf16; clusters of one token
+//      are left as they are.  The cores then leave in seed order with 16-byte coalesced stores.
+//      The service warp draws the block's next ticket during step 2.
 // The last block to finish zeroes the status words and counters, so a workspace that was zero
 // before the call is zero again after it.
 #include <cuda.h>
