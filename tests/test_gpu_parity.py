@@ -308,6 +308,27 @@ def test_compress_overlapped_independent_layer_launches_match_ordinary_ones():
             assert int(ws[l].view(torch.int32)[:n_words].abs().max()) == 0
 
 
+def test_compress_bounded_wait_reports_timeout_and_leaves_the_context_usable():
+    """The look-back's wait is bounded: if a predecessor never reports (here: the ticket counter starts one
+    round in, so the first tile of every head is never processed), the waiting tiles give up after the
+    limit, the status word says SC_ERR_TIMEOUT, the kernel ends, and the next call works."""
+    w = synth.config(0, n=4096)
+    ids, run_id, run_lens = synth.token_ids(w)
+    K, V = synth.layer_kv(w, 0, run_id, run_lens)
+    plan = binding.chunk(ids.to(DEV), w.delims)
+    ws = binding.compress_workspace(w.B, w.Hkv, w.n, DEV)
+    ws.view(torch.int32)[0] = w.B * w.Hkv          # first ticket handed out = tile 1 of head 0
+    out = binding.compress(K.to(DEV), V.to(DEV), plan, w.tau, workspace=ws)    # allocates the outputs
+    torch.cuda.synchronize()
+    assert int(plan.status.item()) == binding.SC_ERR_TIMEOUT
+    # as the header says: zero the workspace after a timeout, then carry on
+    ws.zero_(); plan.status.zero_()
+    ref = oracle_compress(ids, K, V, w.delims, w.tau)
+    got = binding.compress(K.to(DEV), V.to(DEV), plan, w.tau, workspace=ws, out=out)
+    binding.check_status(plan.status)
+    compare_compressed(got, ref, torch.bfloat16, check_assign=False)
+
+
 # ---------------------------------------------------------------------------- sc_decode_attn
 
 
