@@ -201,7 +201,7 @@ def test_compress_capacity_overflow_is_reported_not_written(flags):
     compare_compressed(view, ref_cap, torch.bfloat16)
 
 
-@pytest.mark.parametrize("cfg,kw", [(1, {}), (3, dict(tau=0.9, sigma=0.15)), (4, dict(B=1, gap=("poisson", 128.0))),
+@pytest.mark.parametrize("cfg,kw", [(1, {}), (2, {}), (3, dict(tau=0.9, sigma=0.15)), (4, dict(B=1, gap=("poisson", 128.0))),
                                     (4, dict(B=2, n=32768, gap=("poisson", 8.0), centroids=("ratio", 2.0)))])
 def test_compress_full_size_layer_of_the_benchmark_shapes(cfg, kw):
     """One whole layer at the benchmark's sizes (every block walks many tiles; cfg4 with mean chunk
@@ -383,6 +383,26 @@ def test_decode_is_deterministic_and_scale_is_honoured(flags):
     c = binding.decode_attn(q, got, workspace=ws, flags=flags, scale=0.05)
     want = oracle.attn(synth.to_numpy_bits(q), ref["core_k"], ref["core_v"], ref["count"], ref["core_len"], scale=0.05)
     assert_close_vectors(to_f64(c), want, 1e-2, "custom scale")
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4])
+def test_decode_full_size_layer_in_the_benchmark_launch_shape(cfg):
+    """One layer of each benchmark workload at full size, cores compressed on the GPU into buffers of the
+    benchmark's capacity (n / 2, which sets the number of splits), three decode steps against the oracle."""
+    w = synth.config(cfg, L=1)
+    ids, run_id, run_lens = synth.token_ids(w)
+    K, V = synth.layer_kv(w, 0, run_id, run_lens)
+    ref = oracle_compress(ids, K, V, w.delims, w.tau, w.max_chunk_len, w.n // 2)
+    plan = binding.chunk(ids.to(DEV), w.delims, w.max_chunk_len)
+    got = binding.compress(K.to(DEV), V.to(DEV), plan, w.tau, cap=w.n // 2)
+    binding.check_status(plan.status)
+    assert np.array_equal(got.core_len.cpu().numpy(), ref["core_len"])
+    ws = binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, w.n // 2, DEV)
+    for step in range(3):
+        q = synth.queries(w, step, 0)
+        want = oracle.attn(synth.to_numpy_bits(q), ref["core_k"], ref["core_v"], ref["count"], ref["core_len"])
+        out = binding.decode_attn(q.to(DEV), got, workspace=ws)
+        assert_close_vectors(to_f64(out), want, 1e-2, f"cfg{cfg} step {step}")
 
 
 def test_no_merge_compress_then_decode_equals_exact_attention():
