@@ -187,6 +187,41 @@ SC_API sc_status sc_decode_attn(const void* q, sc_dtype dt, int32_t B, int32_t H
                          void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
 
 /*
+ * One generated token joins a layer's compressed cache (incremental form of Sec. 2.2-2.4).
+ *
+ * The paper compresses the prompt's cache once and is silent about the tokens generated after
+ * it.  This library's reading: the chunking rule of Eq. 1 keeps running over the generated
+ * stream, starting afresh behind the prompt.  Rows [0, core_len) of a head are finished cores;
+ * behind them sit tail_len tokens of the chunk that is still open, stored as they are with
+ * count 1.  A call adds one token per sequence:
+ *   - a token that is not a delimiter is stored behind the tail; when the tail thereby reaches
+ *     max_chunk_len tokens the chunk is finished;
+ *   - a delimiter finishes the open chunk (if any) and then becomes a core of its own with
+ *     count 1 and its K/V bits unchanged.
+ * A finished chunk is clustered (Algorithm 1 on Eq. 2) and mean-pooled (Eq. 3) where it lies,
+ * its cores replacing its first rows, with the same arithmetic as sc_compress (fp32 sums in
+ * token order, one rounding); core_len grows by the number of clusters and tail_len returns
+ * to 0.  The cache therefore ends up as if the generated tokens had been a second prompt.
+ *
+ *   k_new, v_new  [B, Hkv, d] contiguous, dtype dt: this layer's K/V of the new tokens
+ *   token_ids     [B] int32 (device): the new token of each sequence
+ *   delim_ids     HOST, n_delim <= SC_MAX_DELIMS ids;  max_chunk_len in [1, SC_MAX_CHUNK_LEN]
+ *   tau           threshold of Algorithm 1 (Sim > tau joins)
+ *   core_k/v, count, cap   the layer's cache as written by sc_compress, updated in place
+ *   core_len      in/out [B, Hkv]: finished cores of each head
+ *   tail_len      in/out [B, Hkv]: tokens of the open chunk (zero it once after sc_compress)
+ *   attn_len      out [B, Hkv]: core_len + tail_len, the length to give sc_decode_attn
+ *   status        SC_ERR_CAPACITY if a head has no free row (core_len + tail_len == cap): that
+ *                 head is left as it is.  SC_ERR_INVALID_ARG for lengths that cannot be a state
+ *                 of this call (negative, or tail_len >= max_chunk_len).
+ * Any d > 0.  One kernel launch; no workspace.
+ */
+SC_API sc_status sc_append(const void* k_new, const void* v_new, sc_dtype dt, int32_t B, int32_t Hkv, int32_t d,
+                    const int32_t* token_ids, const int32_t* delim_ids /*HOST*/, int32_t n_delim,
+                    int32_t max_chunk_len, float tau, void* core_k, void* core_v, int32_t* count, int32_t cap,
+                    int32_t* core_len, int32_t* tail_len, int32_t* attn_len, int32_t* status, void* stream);
+
+/*
  * sc_decode_attn for callers that cannot allocate device memory.  (A convenience of this
  * library; the paper has no counterpart.)
  *

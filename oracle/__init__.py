@@ -166,3 +166,53 @@ def compress(token_ids, delim_ids, K, V, tau, max_chunk_len=256, cap=None):
     core_k, core_v, count, core_len = merge(K, V, assign, cap, seg_off, seq_seg_off)
     return dict(seg_off=seg_off, seq_seg_off=seq_seg_off, assign=assign, margin=margin,
                 core_k=core_k, core_v=core_v, count=count, core_len=core_len)
+
+
+def append(state: dict, token_ids_new, k_new: np.ndarray, v_new: np.ndarray, delim_ids, tau: float,
+           max_chunk_len: int = 256) -> None:
+    """One generated token per sequence joins one layer's cache, in place (the incremental reading).
+
+    The paper compresses the prompt once and does not say what happens to generated tokens.  The
+    reading taken: Eq. 1 keeps running over the generated stream, starting afresh behind the prompt.
+    ``state`` holds ``core_k``/``core_v`` [B, Hkv, cap, d], ``count`` [B, Hkv, cap], ``core_len`` and
+    ``tail_len`` [B, Hkv], and ``margin`` (the smallest |Sim - tau| met so far).  Rows
+    [core_len, core_len + tail_len) are the tokens of the chunk that is still open, as they came.
+    A token that is not a delimiter is stored behind them; a chunk is finished by reaching
+    ``max_chunk_len`` tokens or by a delimiter, which then becomes a core of its own.  A finished
+    chunk goes through ``gsc`` and ``merge`` as one segment and its cores replace its first rows.
+    """
+    ck, cv, cnt, clen, tlen = (state[k] for k in ("core_k", "core_v", "count", "core_len", "tail_len"))
+    B, Hkv, cap, d = ck.shape
+    delims = set(int(x) for x in delim_ids)
+
+    def finish(b, h):
+        cl, tl = int(clen[b, h]), int(tlen[b, h])
+        if tl >= 2:
+            Kt = np.ascontiguousarray(ck[b:b + 1, h:h + 1, cl:cl + tl])
+            Vt = np.ascontiguousarray(cv[b:b + 1, h:h + 1, cl:cl + tl])
+            seg_off, seq_seg_off = np.array([0, tl], dtype=np.int32), np.array([0, 1], dtype=np.int32)
+            assign, margin = gsc(Kt, seg_off, seq_seg_off, tau)
+            pk, pv, pc, pl = merge(Kt, Vt, assign, tl, seg_off, seq_seg_off)
+            p = int(pl[0, 0])
+            ck[b, h, cl:cl + p], cv[b, h, cl:cl + p], cnt[b, h, cl:cl + p] = pk[0, 0, :p], pv[0, 0, :p], pc[0, 0, :p]
+            state["margin"] = min(state.get("margin", np.inf), margin)
+            tl = p
+        clen[b, h], tlen[b, h] = cl + tl, 0
+
+    for b in range(B):
+        is_delim = int(token_ids_new[b]) in delims
+        for h in range(Hkv):
+            if int(clen[b, h]) + int(tlen[b, h]) >= cap:
+                raise OverflowError(f"no free row in sequence {b}, head {h}")
+            if is_delim:
+                if tlen[b, h] > 0:
+                    finish(b, h)
+                row = int(clen[b, h])
+                ck[b, h, row], cv[b, h, row], cnt[b, h, row] = k_new[b, h], v_new[b, h], 1
+                clen[b, h] = row + 1
+            else:
+                row = int(clen[b, h]) + int(tlen[b, h])
+                ck[b, h, row], cv[b, h, row], cnt[b, h, row] = k_new[b, h], v_new[b, h], 1
+                tlen[b, h] += 1
+                if tlen[b, h] == max_chunk_len:
+                    finish(b, h)

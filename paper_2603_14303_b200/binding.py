@@ -24,7 +24,7 @@ _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CA
 
 EXPORTS = ["sc_version", "sc_launch_counter", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
            "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn",
-           "sc_decode_attn_static"]
+           "sc_decode_attn_static", "sc_append"]
 SC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -75,6 +75,9 @@ def lib() -> ctypes.CDLL:
         L.sc_decode_attn_static.restype = _i32
         L.sc_decode_attn_static.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp,
                                             ctypes.c_float, ctypes.c_uint32, _vp, _vp, _vp]
+        L.sc_append.restype = _i32
+        L.sc_append.argtypes = [_vp, _vp, _i32, _i32, _i32, _i32, _vp, ctypes.POINTER(_i32), _i32, _i32, ctypes.c_float,
+                                _vp, _vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
         _lib = L
     return _lib
 
@@ -180,6 +183,21 @@ def sc_decode_attn_static(q, core_k, core_v, count, core_len, out, scale=0.0, st
                                        cap, _ptr(core_len), float(scale), int(flags), _ptr(out), _ptr(status),
                                        _stream(q))
     _check("sc_decode_attn_static", code)
+
+
+def sc_append(k_new, v_new, token_ids, delim_ids, max_chunk_len, tau, core_k, core_v, count, core_len, tail_len,
+              attn_len, status=None):
+    """Raw sc_append: one generated token per sequence joins one layer's cache (see the header)."""
+    _need_cuda(k_new, v_new, token_ids, core_k, core_v, count, core_len, tail_len, attn_len, status)
+    B, Hkv, d = k_new.shape
+    cap = core_k.shape[2]
+    assert k_new.is_contiguous() and v_new.is_contiguous() and core_k.is_contiguous() and core_v.is_contiguous()
+    assert core_k.shape == (B, Hkv, cap, d) and token_ids.dtype == torch.int32 and token_ids.numel() == B
+    delims = (_i32 * max(len(delim_ids), 1))(*[int(x) for x in delim_ids])
+    code = lib().sc_append(_ptr(k_new), _ptr(v_new), _dt(k_new), B, Hkv, d, _ptr(token_ids), delims, len(delim_ids),
+                           int(max_chunk_len), float(tau), _ptr(core_k), _ptr(core_v), _ptr(count), cap,
+                           _ptr(core_len), _ptr(tail_len), _ptr(attn_len), _ptr(status), _stream(k_new))
+    _check("sc_append", code)
 
 
 # ------------------------------------------------------------------------- convenience wrappers

@@ -103,4 +103,12 @@ struct DecodeArgs {
 cudaError_t launch_decode_generic(const DecodeArgs& a, cudaStream_t st);
 size_t decode_generic_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap);
 
+struct AppendArgs {
+    const void* k_new; const void* v_new; sc_dtype dt; int32_t B, Hkv, d;
+    const int32_t* token_ids; int32_t delim[SC_MAX_DELIMS]; int32_t n_delim; int32_t max_chunk_len; float tau;
+    void* core_k; void* core_v; int32_t* count; int32_t cap;
+    int32_t* core_len; int32_t* tail_len; int32_t* attn_len; int32_t* status;
+};
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
+
 }  // namespace sc
