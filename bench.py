@@ -24,6 +24,8 @@ import sys
 import threading
 import time
 
+import numpy as np
+
 import torch
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -290,9 +292,60 @@ def run_ours(args):
         "gpu_launches_per_step": {"chunk+compress": pipe.launches_compress, "decode": pipe.launches_decode},
         "clocks": clocks, "e2e": e2e, "wall_s": t_wall,
     }
+    if args.gpus == 1:
+        line["append"] = measure_append(pipe)
     if not args.no_cpu_baseline and args.gpus == 1:
         line["cpu_baseline"] = cpu_baseline(w, budget_s=args.cpu_budget)
     print(json.dumps(line))
+
+
+def measure_append(pipe, m: int = 256, layers: int = 4):
+    """sc_append behind the compressed prompt (outside the timed step; it changes the caches, so it runs
+    last): m generated tokens into the first few layers.  Device time per call comes from one CUDA graph
+    holding all m x layers calls (replayed once to warm up, once timed: the stream is appended twice more);
+    calls launched one by one from Python are bound by the host and only show what finishing a chunk adds."""
+    b, w, dev = pipe.b, pipe.w, pipe.dev
+    layers = min(layers, w.L)
+    i32 = dict(dtype=torch.int32, device=dev)
+    status = torch.zeros(1, **i32)
+    plain, closing, calls = [], [], []
+    for layer in range(layers):
+        ids, K, V = synth.generated_stream(w, m, layer)
+        ids, K, V = ids.to(dev), K.to(dev), V.to(dev)
+        lay = pipe.layers[layer]
+        tail, alen = torch.zeros((w.B, w.Hkv), **i32), torch.zeros((w.B, w.Hkv), **i32)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(m)]
+        before = []
+        for t in range(m):
+            args_t = (K[:, :, t].contiguous(), V[:, :, t].contiguous(), ids[:, t].contiguous(), w.delims, w.max_chunk_len,
+                      w.tau, lay.core_k, lay.core_v, lay.count, lay.core_len, tail, alen, status)
+            calls.append(args_t)
+            before.append(tail.clone())
+            ev[t][0].record()
+            b.sc_append(*args_t)
+            ev[t][1].record()
+        torch.cuda.synchronize()
+        before.append(tail.clone())
+        for t in range(8, m):   # the first calls warm up
+            shrank = bool((before[t + 1] < before[t]).any())   # some sequence's open chunk was finished by this call
+            (closing if shrank else plain).append(ev[t][0].elapsed_time(ev[t][1]) * 1e3)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for args_t in calls:
+            b.sc_append(*args_t)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    b.check_status(status, "sc_append")
+    med = lambda a: float(np.median(a)) if a else None
+    return {"what": "sc_append: one call per layer and generated token",
+            "tokens": m, "layers": layers, "us_per_call_device": e0.elapsed_time(e1) * 1e3 / len(calls),
+            "calls_finishing_a_chunk_fraction": len(closing) / max(len(closing) + len(plain), 1),
+            "host_bound_us_per_call_storing": med(plain), "host_bound_us_per_call_finishing_a_chunk": med(closing)}
 
 
 def run_e2e(pipe, args, barrier):

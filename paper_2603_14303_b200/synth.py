@@ -180,6 +180,27 @@ def queries(w: Workload, step: int, layer: int, device="cpu") -> torch.Tensor:
     return torch.randn((w.B, w.Hq, w.d), generator=g, device=dev).to(_torch_dtype(w))
 
 
+def generated_stream(w: Workload, m: int, layer: int = 0, mean_gap: float = 20.0, n_centroids: int = 5):
+    """A seeded stand-in for m generated tokens per sequence: ids [B, m] int32 with a delimiter after
+    Poisson(mean_gap) ordinary tokens, and this layer's K, V [B, Hkv, m, d] in the workload's dtype
+    (keys: one of n_centroids unit directions per head plus noise of RMS norm w.sigma; values N(0, 1))."""
+    rng = np.random.default_rng((w.seed * 1000003 + layer * 9176 + 77) & 0x7FFFFFFF)
+    ids = rng.integers(1000, w.vocab, size=(w.B, m)).astype(np.int32)
+    ids[np.isin(ids, np.array(w.delims))] = 999
+    for b in range(w.B):
+        t = int(rng.poisson(mean_gap))
+        while t < m:
+            ids[b, t] = w.delims[int(rng.integers(len(w.delims)))]
+            t += 1 + int(rng.poisson(mean_gap))
+    cent = rng.normal(size=(w.Hkv, n_centroids, w.d))
+    cent /= np.linalg.norm(cent, axis=-1, keepdims=True)
+    pick = rng.integers(0, n_centroids, size=(w.B, w.Hkv, m))
+    K = cent[np.arange(w.Hkv)[None, :, None], pick] + w.sigma / math.sqrt(w.d) * rng.normal(size=(w.B, w.Hkv, m, w.d))
+    V = rng.normal(size=(w.B, w.Hkv, m, w.d))
+    dt = _torch_dtype(w)
+    return torch.from_numpy(ids), torch.from_numpy(K).to(dt), torch.from_numpy(V).to(dt)
+
+
 def to_numpy_bits(t: torch.Tensor) -> np.ndarray:
     """CPU numpy view for the test oracle: bf16 -> uint16 raw bits, others unchanged."""
     t = t.detach().cpu()
