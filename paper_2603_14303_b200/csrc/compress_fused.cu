@@ -12,8 +12,8 @@
 //      triangle of its Gram matrix (bf16 products are exact in fp32), the diagonal gives the norms,
 //      Sim > tau is decided as G_ij > tau*|k_i|*|k_j|, each lane ends up with one row's adjacency
 //      word, and the greedy pass costs one shuffle and a few word operations per seed;
-//   3. a segment of 33..64 tokens is still one warp's own business: it builds the bit rows of the
-//      segment in 16-row bands in shared memory and runs the greedy pass on them; beyond 64 tokens
+//   3. a segment of 33..kWarpSegMax (48) tokens is still one warp's own business: it builds the bit rows of the
+//      segment in 16-row bands in shared memory and runs the greedy pass on them; beyond that
 //      the Gram matrix is cut into 32x32 blocks (exactly the block pairs the segment spans) that all
 //      warps share, and one warp runs the greedy pass with one lane per 32-token word.  The
 //      adjacency bits live in an upper triangle of 32-bit words per row; a seed's row ends up
@@ -47,6 +47,11 @@ constexpr int kBoxRows = 32;                      // rows per TMA box
 constexpr int kBoxBytes = kBoxRows * kHalfRow;    // 4096
 constexpr int kMaxRows = SC_MAX_CHUNK_LEN;        // 256: a long tile
 constexpr int kShortRows = SC_TILE_ROWS;          // 128
+// Longest segment one warp clusters on its own; longer ones share their Gram blocks among all warps.  The
+// warp-private code handles up to 64 tokens, but a tile that waits for one warp to finish a long segment
+// also holds up the tiles that look back to it: 48 measured best on every workload (32 and 40 were slower
+// for Poisson(30) chunks, 56 and 64 for lognormal ones).
+constexpr int kWarpSegMax = 48;
 constexpr int kNW = 8;                            // 32-bit words per (full) adjacency row
 constexpr int kKvBytes = kMaxRows * kRowBytes;    // 65536: short = K | V, long = one tensor
 constexpr int kVOff = kShortRows * kRowBytes;     // 32768
@@ -505,7 +510,7 @@ __device__ __forceinline__ void fetch_tile(const Params& p, int lane, int max_nt
 // Stages rows [row0, row0 + R) of head (b, h) of one tensor with TMA: one box of 32 rows x 64 columns
 // per lane (R <= 256 needs at most 16 boxes for both column halves), the halves `hs` bytes apart at
 // `dst`.  Rows past R inside the last box are the cache's next rows, or zeros past the end of the
-// sequence: finite either way, and they only ever enter the Eq. 3 product with weight 0.
+// sequence; no one reads them.
 __device__ __forceinline__ void stage_rows(uint32_t dst, int hs, const CUtensorMap* map, int row0, int R, int h, int b,
                                            uint32_t bar, int lane) {
     const int nb = (R + kBoxRows - 1) / kBoxRows;
@@ -517,7 +522,7 @@ __device__ __forceinline__ void stage_rows(uint32_t dst, int hs, const CUtensorM
     }
 }
 
-// Eq. 2 for one segment of 33..64 tokens [a, a + l), by one warp on its own (no block-level step):
+// Eq. 2 for one segment of 33..64 tokens [a, a + l) (the kernel sends it up to kWarpSegMax), by one warp on its own (no block-level step):
 // the upper triangle of the segment's Gram matrix in 16-row bands, last band first so that the
 // norms a band needs (its own rows', from its diagonal, and those of all later rows) are known
 // when it is thresholded.  Every row's adjacency bits (later tokens of the segment) go to its
@@ -694,7 +699,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         int32_t* as = p.assign ? p.assign + (size_t)bh * p.n + row0 : nullptr;
         if (nseg == 1 && R > 1) {
             for (int r = tid; r < R; r += kThreads) send[r] = (uint16_t)R;
-            if (R > 64 && tid < nrb) { atomicOr(&misc[2], 1 << tid); reach[tid] = nrb - 1; }
+            if (R > kWarpSegMax && tid < nrb) { atomicOr(&misc[2], 1 << tid); reach[tid] = nrb - 1; }
             if (tid == 0) { multi[0] = 0; misc[3] = 1; }
         } else {
             for (int s = tid; s < nseg; s += kThreads) {
@@ -707,7 +712,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                     continue;
                 }
                 multi[atomicAdd(&misc[3], 1)] = (uint8_t)s;
-                if (e - a > 64) {   // only the block-level path reads send[] (of every row of the blocks it touches)
+                if (e - a > kWarpSegMax) {   // only the block-level path reads send[] (of every row of the blocks it touches)
                     for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
                     for (int k = a >> 5; k <= (e - 1) >> 5; ++k) { atomicOr(&misc[2], 1 << k); atomicMax(&reach[k], (e - 1) >> 5); }
                 }
@@ -724,7 +729,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         if (__syncthreads_or(failed)) { failed = true; break; }
         CF_T(2);
 
-        // ---- 2. segments of more than 64 tokens: Gram blocks -> norms -> adjacency bits in shared memory ----
+        // ---- 2. segments of more than kWarpSegMax tokens: Gram blocks -> norms -> adjacency bits in shared memory ----
         const int longblocks = misc[2];
         if (longblocks != 0) {
             float acc[2][4][4];
@@ -767,7 +772,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                     else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
                     continue;
                 }
-                if (e - a <= 64) {   // the warp builds the segment's bit rows itself
+                if (e - a <= kWarpSegMax) {   // the warp builds the segment's bit rows itself
                     if (p.tau < 0.f) gram_mid_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 64, adj, lane);
                     else gram_mid_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 64, adj, lane);
                 }

@@ -105,7 +105,7 @@ def test_compress_cfg0_matches_oracle(dtype, flags):
 
 
 @pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC, binding.SC_FLAG_TWO_PASS])
-@pytest.mark.parametrize("length", [1, 2, 31, 32, 33, 63, 64, 65, 127, 128, 129, 200, 255, 256])
+@pytest.mark.parametrize("length", [1, 2, 31, 32, 33, 47, 48, 49, 63, 64, 65, 127, 128, 129, 200, 255, 256])
 def test_compress_fixed_chunk_lengths(length, flags):
     w = synth.config(0, n=3000, Hkv=2, Hq=8, gap=("fixed", length), centroids=("uniform", 5), seed=length)
     ref, got, plan, _ = _compress_both(w, flags=flags)
