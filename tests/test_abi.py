@@ -47,6 +47,12 @@ def test_host_side_validation_needs_no_gpu(lib):
                            None, None, None, 16, 1, None, None, 0, None, None) == binding.SC_ERR_UNSUPPORTED
     assert lib.sc_decode_attn(None, 0, 1, 30, 8, 128, None, None, None, 0, None, 0.0, 0, None, None, 0, None,
                               None) == binding.SC_ERR_INVALID_ARG  # Hq % Hkv != 0
+    ap = lambda dt, B, max_len, k: lib.sc_append(k, k, dt, B, 8, 128, None, None, 0, max_len, 0.7, None, None, None, 64,
+                                                 None, None, None, None, None)
+    assert ap(0, 1, 300, None) == binding.SC_ERR_INVALID_ARG       # max_chunk_len beyond SC_MAX_CHUNK_LEN
+    assert ap(5, 1, 256, None) == binding.SC_ERR_UNSUPPORTED      # unknown dtype
+    assert ap(0, 1, 256, None) == binding.SC_ERR_INVALID_ARG       # null tensors
+    assert ap(0, 0, 256, None) == binding.SC_OK                    # nothing to do
 
 
 def test_missing_library_fails_loudly(monkeypatch):

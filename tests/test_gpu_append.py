@@ -150,3 +150,14 @@ def test_append_full_cache_is_reported_and_left_alone():
     assert torch.equal(both.ck, before[0]) and torch.equal(both.cnt, before[1])
     assert torch.equal(both.clen, before[2]) and torch.equal(both.tlen, before[3])
     assert (both.alen.cpu().numpy() == 4).all()
+
+
+def test_append_refuses_lengths_that_cannot_be_its_own_state():
+    B, Hkv, d, cap = 1, 2, 128, 16
+    ids, K, V = _stream(2, B, Hkv, 1, d, 0.0, torch.bfloat16)
+    both = Both(B, Hkv, cap, d, torch.bfloat16)
+    both.tlen.fill_(5)            # an open chunk of 5 tokens cannot exist with max_chunk_len = 4
+    binding.sc_append(K[:, :, 0].contiguous().to(DEV), V[:, :, 0].contiguous().to(DEV), ids[:, 0].contiguous().to(DEV), DELIM, 4,
+                      0.7, both.ck, both.cv, both.cnt, both.clen, both.tlen, both.alen, both.status)
+    assert int(both.status.item()) == binding.SC_ERR_INVALID_ARG
+    assert int(both.clen.abs().max()) == 0 and (both.tlen == 5).all() and int(both.cnt.abs().max()) == 0
