@@ -756,7 +756,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
 
         // ---- 3. the service warp draws the block's next ticket; compute warps: Algorithm 1 per segment,
         //         one warp each, in registers up to 32 tokens, else on the bit rows ----
-        unsigned char* lane_base = smem + (lane >> 4) * kVOff + ((lane >> 3) & 1) * hs;   // see row_add
+        unsigned char* lane_base = smem + (lane >> 4) * kVOff + ((lane >> 3) & 1) * hs;   // see rows_add
         if (service) {
             CF_SPAN_BEGIN();
             fetch_tile(p, lane, max_nt, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
