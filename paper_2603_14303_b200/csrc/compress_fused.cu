@@ -101,7 +101,7 @@ __device__ unsigned long long g_phase_cycles[16];
 constexpr uint32_t kPending = 1u << 31;
 constexpr uint32_t kFlagAggregate = 1u << 30, kFlagPrefix = 2u << 30, kValueMask = (1u << 30) - 1;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // every wait gives up after 2 s
-constexpr int kPollGroups = 4;                               // the look-back reads 128 predecessors per poll
+constexpr int kPollGroups = 2;                               // the look-back reads 64 predecessors per poll (4 and 8 measured slower, 1 slower on short chunks)
 constexpr int kCtlWords = 64;                                // ticket, done counter, padding
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
