@@ -39,7 +39,7 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/, by workload:
 # sc_decode_attn (decode_mma_kernel_cfg1_8layers.md) and sc_compress (compress_fused_kernel_cfg1_8layers.md).
 # Only valid while those kernels are the ones that were captured; other workloads report null.
-NCU_TRAFFIC = {"cfg1-llama3-8b-32k": {"decode": 34.31e6, "compress": 155.0e6}}
+NCU_TRAFFIC = {"cfg1-llama3-8b-32k": {"decode": 34.31e6, "compress": 153.7e6}}
 
 
 def measured_peaks():
