@@ -2,13 +2,18 @@
 """Benchmark of the SemantiCache hot path on B200.
 
 One *step* = one pass of the whole path over one synthetic batch: sc_chunk once, sc_compress for
-every layer, then ``decode_steps`` decode steps of sc_decode_attn over every layer's cores.
+every layer, then ``decode_steps`` decode steps of sc_decode_attn over every layer's cores; inside
+a decode step the layers form a dependent chain (layer l+1's query is layer l's output), as in a
+model's decode loop.
 Reported ``value`` = decoded tokens per second over the whole step (compress included); the
 decode-only rate, the compress time per 32K context and the achieved HBM bandwidth of both
 stages are added as extra keys.  Everything is launched through the C-ABI library; the launch
 sequence is captured into CUDA graphs so Python is not on the timed path.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl ours|reference]
+
+After the headline run (N = 1) short passes cover the other four workloads, the noise sweep and the
+chunk-length x reduction grid with exact attention over the raw cache beside it (``configs``).
 
 ``--impl reference`` times the CPU oracle (plain C, fp64) on a bounded sample of the same
 workload on the host cores.
@@ -36,10 +41,16 @@ from paper_2603_14303_b200 import synth  # noqa: E402
 METRIC = "compressed_kv_decode_tokens_per_s"
 UNIT = "tokens/s"
 
-# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/, by workload:
-# sc_decode_attn (decode_mma_kernel_cfg1_8layers.md) and sc_compress (compress_fused_kernel_cfg1_8layers.md).
-# Only valid while those kernels are the ones that were captured; other workloads report null.
-NCU_TRAFFIC = {"cfg1-llama3-8b-32k": {"decode": 34.31e6, "compress": 153.7e6}}
+
+def recorded_traffic(workload: str, stage: str):
+    """DRAM bytes (read + write) per launch from an ncu capture, or None.
+
+    The record (written by ``python -m paper_2603_14303_b200.ncu_traffic`` from an ncu CSV) names the
+    workload and carries a hash of the kernel's source file as it was when the counters were taken; a
+    kernel that has changed since gives None rather than a stale figure.  Not a measurement of this run."""
+    from paper_2603_14303_b200 import ncu_traffic
+    return ncu_traffic.lookup(workload, stage)
+
 
 
 def measured_peaks():
@@ -51,10 +62,11 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while timed regions run."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, index: int):
         self.index, self.proc, self.lines = index, None, []
@@ -71,16 +83,16 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
-    def stop(self):
+    def summary(self, t0: float = 0.0, t1: float = float("inf")):
+        """Median SM clock and the throttle reasons seen between host times t0 and t1."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        self.thread.join(timeout=2)
         sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for ts, ln in list(self.lines):
+            if ts < t0 or ts > t1 + 0.1:
+                continue
             p = [x.strip() for x in ln.split(",")]
             if len(p) < 7:
                 continue
@@ -88,20 +100,35 @@ class ClockSampler:
                 sm.append(float(p[0])); smax.append(float(p[1]))
             except ValueError:
                 continue
-            for nm, v in zip(names, p[3:7]):
+            for nm, v in zip(self.NAMES, p[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(nm)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
 
+    def stop(self, t0: float = 0.0, t1: float = float("inf")):
+        if self.proc is not None:
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+        return self.summary(t0, t1)
+
 
 # ------------------------------------------------------------------------------------- ours
+
+# How the L per-layer sc_decode_attn calls of one decode step are launched:
+#   chain        layer l+1's query is layer l's output, as in a model's decode loop; launched with
+#                SC_FLAG_OVERLAP_CHAIN (the cores are prefetched while the previous layer still runs, the
+#                query is read once it is complete)
+#   serial       the same dependent chain in plain stream order
+#   independent  every layer has its own seeded query and SC_FLAG_OVERLAP_PREV: an attention-only loop
+#                whose launches do not depend on one another
+DECODE_MODES = ("chain", "serial", "independent")
 
 
 class Pipeline:
     """Device-resident state of one rank: inputs, plan, cores, and the captured launch graphs."""
 
-    def __init__(self, w: synth.Workload, device, cap_frac: float = 0.5):
+    def __init__(self, w: synth.Workload, device, cap_frac: float = 0.5, raw_comparator: bool = False):
         from paper_2603_14303_b200 import binding
         self.b, self.w, self.dev = binding, w, device
         self.ids, self.run_id, self.run_lens = synth.token_ids(w)
@@ -117,19 +144,24 @@ class Pipeline:
                                                torch.empty((w.B, w.Hkv, self.cap, w.d), dtype=dt, device=device),
                                                torch.zeros((w.B, w.Hkv, self.cap), **i32),
                                                torch.zeros((w.B, w.Hkv), **i32)) for _ in range(w.L)]
-        # one workspace per layer (both stages): consecutive layer launches overlap and must not share scratch
         self.cws = [binding.compress_workspace(w.B, w.Hkv, w.n, device) for _ in range(w.L)]
         self.dws = [binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, self.cap, device) for _ in range(w.L)]
+        # q[s, 0] feeds layer 0 of decode step s in every mode; q[s, l > 0] only the independent mode
         self.q = torch.stack([torch.stack([synth.queries(w, s, l, device) for l in range(w.L)])
                               for s in range(w.decode_steps)])            # [steps, L, B, Hq, d]
         self.out = torch.empty_like(self.q)
         self.plan = None
-        self.decode_flags = 0
-        self.compress_flags = 0
         self.status = torch.zeros((w.L, 1), **i32)
         self.cstatus = torch.zeros((w.L, 1), **i32)
-        self.launches_compress = self.launches_decode = 0
-        self.g_compress = self.g_decode = None
+        self.launches_compress = 0
+        self.g_compress = None
+        self.g_decode, self.launches_decode = {}, {}
+        # exact attention over the raw cache with the same kernel (count = NULL, every head n rows long)
+        self.raw = None
+        if raw_comparator:
+            self.raw_len = torch.full((w.B, w.Hkv), w.n, **i32)
+            self.raw_ws = [binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, w.n, device) for _ in range(w.L)]
+            self.raw = True
 
     # the launch sequences (also what the graphs capture)
     def run_compress(self):
@@ -142,40 +174,71 @@ class Pipeline:
             b.sc_chunk(self.ids_dev, w.delims, w.max_chunk_len, p.seg_off, p.seq_seg_off, p.n_seg, p.tile_seg,
                        p.seq_tile_cnt, self._chunk_ws, p.status)
         for l in range(w.L):
-            # layer 0 follows sc_chunk and needs its plan; the other layers share nothing they write with
-            # their predecessor (own K/V, cores, workspace, status) and may overlap its tail
             ly = self.layers[l]
             b.sc_compress(self.K[l], self.V[l], self.plan, w.tau, ly.core_k, ly.core_v, ly.count, ly.core_len, None,
-                          self.cws[l], self.cstatus[l], self.compress_flags if l > 0 else 0)
+                          self.cws[l], self.cstatus[l], 0)
 
-    def run_decode(self):
+    def run_decode(self, mode: str, steps: int | None = None, raw: bool = False):
         b, w = self.b, self.w
-        for s in range(w.decode_steps):
+        flag = {"chain": b.SC_FLAG_OVERLAP_CHAIN, "serial": 0, "independent": b.SC_FLAG_OVERLAP_PREV}[mode]
+        for s in range(steps or w.decode_steps):
             for l in range(w.L):
-                # layer 0 of each step is an ordinary launch (ordered after all earlier work); the other
-                # layers share no buffer with their predecessor and may overlap it
-                b.decode_attn(self.q[s, l], self.layers[l], out=self.out[s, l], workspace=self.dws[l],
-                              status=self.status[l], flags=self.decode_flags if l > 0 else 0)
+                q = self.q[s, l] if (l == 0 or mode == "independent") else self.out[s, l - 1]
+                # the first launch of a decode step is an ordinary one: it orders the step behind all earlier work
+                fl = flag if l > 0 else 0
+                if raw:
+                    b.sc_decode_attn(q, self.K[l], self.V[l], None, self.raw_len, self.out[s, l], self.raw_ws[l],
+                                     0.0, self.status[l], fl)
+                else:
+                    b.decode_attn(q, self.layers[l], out=self.out[s, l], workspace=self.dws[l],
+                                  status=self.status[l], flags=fl)
 
-    def capture(self):
+    def capture(self, modes=("chain",), short_steps: int | None = None):
+        """Warm-up pass, then one graph for the compress stage and one per decode mode.  The first mode
+        is captured with all decode steps; the others with ``short_steps`` (they are side measurements)."""
         self.run_compress()   # allocates the plan outside capture
-        self.run_decode()
         torch.cuda.synchronize(self.dev)
         self.b.check_status(self.plan.status, "warm-up pass")
         if int(self.cstatus.abs().max().item()) != 0:
             raise RuntimeError("sc_compress reported a device-side error in the warm-up pass")
-        self.g_compress, self.g_decode = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
         c0 = self.b.launch_counter()
+        self.g_compress = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.g_compress):
             self.run_compress()
-        c1 = self.b.launch_counter()
-        with torch.cuda.graph(self.g_decode):
-            self.run_decode()
-        self.launches_compress, self.launches_decode = c1 - c0, self.b.launch_counter() - c1
+        self.launches_compress = self.b.launch_counter() - c0
+        self.steps_of = {}
+        for i, mode in enumerate(modes):
+            steps = self.w.decode_steps if (i == 0 or not short_steps) else min(short_steps, self.w.decode_steps)
+            self.run_decode(mode, 1)
+            torch.cuda.synchronize(self.dev)
+            c0 = self.b.launch_counter()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self.run_decode(mode, steps)
+            self.g_decode[mode], self.launches_decode[mode], self.steps_of[mode] = g, self.b.launch_counter() - c0, steps
+        if self.raw:
+            steps = min(short_steps or self.w.decode_steps, self.w.decode_steps)
+            self.run_decode("chain", 1, raw=True)
+            torch.cuda.synchronize(self.dev)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                self.run_decode("chain", steps, raw=True)
+            self.g_decode["raw"], self.steps_of["raw"] = g, steps
         torch.cuda.synchronize(self.dev)
+        if int(self.status.abs().max().item()) != 0:
+            raise RuntimeError("sc_decode_attn reported a device-side error in the warm-up pass")
+
+    def time_graph(self, g, reps: int):
+        """Median device time (ms) of ``reps`` replays of a graph, one warm-up replay first."""
+        g.replay()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for a, z in ev:
+            a.record(); g.replay(); z.record()
+        torch.cuda.synchronize(self.dev)
+        return statistics.median(a.elapsed_time(z) for a, z in ev)
 
     def algorithmic_bytes(self):
-        """(compress bytes per step, decode bytes per decode step over all layers, per-layer list)."""
+        """(compress bytes per step, decode bytes per decode step over all layers, per-layer list, kept)."""
         w = self.w
         esz = self.K[0].element_size()
         lens = torch.stack([ly.core_len for ly in self.layers]).to(torch.int64).cpu()   # [L, B, Hkv]
@@ -185,6 +248,16 @@ class Pipeline:
         qo = w.L * w.B * w.Hq * w.d * esz * 2
         per_layer = [(lens[l].sum().item() * (2 * w.d * esz + 4) + qo // w.L) for l in range(w.L)]
         return kv_in + core_bytes, core_bytes + qo, per_layer, rows / (w.L * w.B * w.Hkv * w.n)
+
+
+def decode_mode_record(pipe: Pipeline, mode: str, ms: float, layer_bytes: float, peak: float):
+    """Per-launch time and achieved bandwidth of one decode graph replay that took ``ms``."""
+    w = pipe.w
+    launches = pipe.steps_of[mode] * w.L
+    us = ms * 1e3 / launches
+    gbs = layer_bytes / (us * 1e-6) / 1e9
+    return {"us_per_launch": us, "achieved_gbs": gbs, "frac": gbs / peak, "frac_of_nominal_8tbs": gbs / 8000.0,
+            "decode_tokens_per_s": w.B * pipe.steps_of[mode] / (ms * 1e-3), "decode_steps_timed": pipe.steps_of[mode]}
 
 
 def run_ours(args):
@@ -205,39 +278,35 @@ def run_ours(args):
     if distributed:
         w = scdist.rank_workload(w, rank)           # every rank owns an independent batch (weak scaling)
     pipe = Pipeline(w, dev)
-    # the per-layer decode calls of a step are independent (own q, out, workspace): let them overlap
-    pipe.decode_flags = 0 if args.no_overlap else binding.SC_FLAG_OVERLAP_PREV
-    # sc_compress also takes the flag, but overlapping consecutive layers gains 2 % on cfg1 and loses a factor
-    # of two on cfg3 (4 KV heads, 128K tokens): its layers are launched the ordinary way
-    pipe.compress_flags = 0
-    pipe.capture()
+    main_mode = "serial" if args.no_overlap else "chain"
+    side_modes = [m for m in DECODE_MODES if m != main_mode] if (args.gpus == 1 and not args.no_modes) else []
+    pipe.capture([main_mode] + side_modes, short_steps=max(8, min(32, w.decode_steps // 8)))
     cbytes, dbytes, per_layer, kept = pipe.algorithmic_bytes()
+    g_decode = pipe.g_decode[main_mode]
 
     def barrier():
         scdist.barrier(dev)
 
-    def one_step():
-        pipe.g_compress.replay()
-        pipe.g_decode.replay()
-
     for _ in range(max(args.warmup, 3)):
-        one_step()
+        pipe.g_compress.replay()
+        g_decode.replay()
     barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     barrier()
+    t_host0 = time.time()
     t_wall = time.perf_counter()
     for s in range(args.steps):
         ev[s][0].record()
         pipe.g_compress.replay()
         ev[s][1].record()
-        pipe.g_decode.replay()
+        g_decode.replay()
         ev[s][2].record()
     barrier()
     t_wall = time.perf_counter() - t_wall
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.summary(t_host0, time.time()) if rank == 0 else None
     binding.check_status(pipe.plan.status, "timed region")
     if int(pipe.status.abs().max().item()) != 0 or int(pipe.cstatus.abs().max().item()) != 0:
         raise RuntimeError("sc_compress / sc_decode_attn reported a device-side error")
@@ -248,7 +317,7 @@ def run_ours(args):
     value = scdist.whole_job_rate(w.B * w.decode_steps * args.steps, args.gpus, total_ms)
 
     # end to end through the public API with HOST buffers (copies inside the timed region)
-    e2e = run_e2e(pipe, args, barrier) if not args.no_e2e else None
+    e2e = run_e2e(pipe, args, barrier, g_decode) if not args.no_e2e else None
     if distributed and e2e is not None:
         e2e["value"] = scdist.whole_job_rate(w.B * w.decode_steps * e2e["_steps"], args.gpus,
                                              scdist.max_over_ranks([e2e["_ms"]], dev)[0])
@@ -264,39 +333,147 @@ def run_ours(args):
     achieved = layer_bytes / (dec_launch_us * 1e-6) / 1e9
     comp_ms = sum_c / args.steps
     comp_gbs = cbytes / (comp_ms * 1e-3) / 1e9
+    launch_text = {"chain": "cuda graphs; within a decode step layer l+1's query is layer l's output and the launches are "
+                            "chained (SC_FLAG_OVERLAP_CHAIN: cores prefetched under the previous layer, query read after it)",
+                   "serial": "cuda graphs; dependent per-layer launches in plain stream order"}[main_mode]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "n_ctx": w.n, "layers": w.L, "kv_heads": w.Hkv, "q_heads": w.Hq,
                    "head_dim": w.d, "tau": w.tau, "decode_steps": w.decode_steps, "kept_fraction": round(kept, 4),
-                   "l2": "inputs larger than L2 (every step streams all layers)", "launch": "cuda graphs" + ("" if args.no_overlap else "; the independent per-layer decode launches of a step overlap (programmatic stream serialization, no wait)"),
+                   "l2": "inputs larger than L2 (every step streams all layers)", "launch": launch_text,
                    "parallelism": f"replicas x{args.gpus}" if distributed else "single gpu"},
         "decode_tokens_per_s": w.B * w.decode_steps * args.gpus / (sum_d / args.steps * 1e-3),
         "decode_bytes_per_step": dbytes,
         "decode_gbs": dbytes * w.decode_steps / (sum_d / args.steps * 1e-3) / 1e9,
         "compress_ms_per_32k_ctx": comp_ms * 32768 / (w.B * w.n),
         "compress_gbs": comp_gbs, "compress_frac_of_peak": comp_gbs / peak,
-        "roofline": {"kernel": "sc_decode_attn (one layer per launch)", "bound": "hbm", "achieved": achieved,
-                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+        "roofline": {"kernel": "sc_decode_attn (one layer per launch, " + main_mode + " launches)", "bound": "hbm",
+                     "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8tbs": achieved / 8000.0, "bytes_per_launch": layer_bytes,
                      "us_per_launch": dec_launch_us,
-                     "traffic": args.traffic if args.traffic is not None else
-                     NCU_TRAFFIC.get(w.name, {}).get("decode")},
+                     "traffic": args.traffic if args.traffic is not None else recorded_traffic(w.name, "decode"),
+                     "traffic_source": "ncu capture recorded under profiles/ (not this run); null once the kernel source changed"},
         "roofline_compress": {"kernel": "sc_compress (one layer per launch)", "bound": "hbm", "achieved": comp_gbs,
                               "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": comp_gbs / peak,
                               "frac_of_nominal_8tbs": comp_gbs / 8000.0, "bytes_per_launch": cbytes / w.L,
                               "us_per_launch": comp_ms * 1e3 / w.L,
-                              "traffic": NCU_TRAFFIC.get(w.name, {}).get("compress")},
-        "gpu_launches": args.steps * (pipe.launches_compress + pipe.launches_decode),
-        "gpu_launches_per_step": {"chunk+compress": pipe.launches_compress, "decode": pipe.launches_decode},
+                              "traffic": recorded_traffic(w.name, "compress")},
+        "gpu_launches": args.steps * (pipe.launches_compress + pipe.launches_decode[main_mode]),
+        "gpu_launches_per_step": {"chunk+compress": pipe.launches_compress, "decode": pipe.launches_decode[main_mode]},
         "clocks": clocks, "e2e": e2e, "wall_s": t_wall,
     }
+    if side_modes:
+        # the same decode work under the other launch disciplines (decode graph alone, a few replays each)
+        modes = {main_mode: {"us_per_launch": dec_launch_us, "achieved_gbs": achieved, "frac": achieved / peak,
+                             "frac_of_nominal_8tbs": achieved / 8000.0,
+                             "decode_tokens_per_s": line["decode_tokens_per_s"], "decode_steps_timed": w.decode_steps,
+                             "timed": "inside the benchmark step"}}
+        for m in side_modes:
+            modes[m] = decode_mode_record(pipe, m, pipe.time_graph(pipe.g_decode[m], 5), layer_bytes, peak)
+        line["decode_launch_modes"] = {
+            "what": "chain = layer l+1's query is layer l's output, launches chained with SC_FLAG_OVERLAP_CHAIN (what a "
+                    "model's decode loop can use); serial = the same chain in plain stream order; independent = every "
+                    "layer has its own query, SC_FLAG_OVERLAP_PREV (an attention-only loop without the dependence)",
+            **modes}
+        line["decode_serial"] = modes["serial"]
+        line["decode_independent_overlap"] = modes["independent"]
     if args.gpus == 1:
         line["append"] = measure_append(pipe)
+    del pipe
+    torch.cuda.empty_cache()
+    if args.gpus == 1 and not args.no_sweep:
+        t0 = time.time()
+        line["configs"] = sweep_configs(args, dev, sampler, peak)
+        line["configs"]["wall_s"] = time.time() - t0
+    sampler.stop()
     if not args.no_cpu_baseline and args.gpus == 1:
         line["cpu_baseline"] = cpu_baseline(w, budget_s=args.cpu_budget)
     print(json.dumps(line))
+
+
+# ------------------------------------------------------------ the five workloads and their sweeps
+
+
+def measure_cell(w: synth.Workload, full_L: int, dev, sampler, peak, label: dict, raw: bool = False,
+                 decode_steps: int = 8, cap_frac: float = 0.5):
+    """Short pass of one workload cell on a reduced layer count: compress (median of 3 graph replays) and
+    chained decode (median of 3 replays of ``decode_steps`` steps), optionally exact attention over the raw
+    cache with the same kernel.  Rates are for the workload's full layer count ``full_L``."""
+    t0 = time.time()
+    w = w.replace(decode_steps=decode_steps)
+    pipe = Pipeline(w, dev, cap_frac=cap_frac, raw_comparator=raw)
+    pipe.capture(["chain"], short_steps=decode_steps)
+    cbytes, dbytes, per_layer, kept = pipe.algorithmic_bytes()
+    ms_c = pipe.time_graph(pipe.g_compress, 3)
+    ms_d = pipe.time_graph(pipe.g_decode["chain"], 3)
+    layer_bytes = sum(per_layer) / len(per_layer)
+    us_launch = ms_d * 1e3 / (decode_steps * w.L)
+    dgbs = layer_bytes / (us_launch * 1e-6) / 1e9
+    cgbs = cbytes / (ms_c * 1e-3) / 1e9
+    rec = dict(label)
+    rec.update({
+        "layers_run": w.L, "layers_full": full_L, "kept_fraction": round(kept, 4),
+        "achieved_reduction": round(1.0 / kept, 3) if kept > 0 else None,
+        "decode_tokens_per_s": w.B / (us_launch * 1e-6 * full_L), "decode_bytes_per_step": dbytes / w.L * full_L,
+        "decode_us_per_launch": us_launch, "decode_gbs": dgbs, "decode_frac": dgbs / peak,
+        "compress_ms_per_32k_ctx": ms_c / w.L * full_L * 32768 / (w.B * w.n), "compress_us_per_layer": ms_c * 1e3 / w.L,
+        "compress_gbs": cgbs, "compress_frac": cgbs / peak})
+    if raw:
+        ms_r = pipe.time_graph(pipe.g_decode["raw"], 3)
+        us_r = ms_r * 1e3 / (pipe.steps_of["raw"] * w.L)
+        raw_bytes = w.B * w.Hkv * w.n * 2 * w.d * pipe.K[0].element_size() + 2 * w.B * w.Hq * w.d * pipe.K[0].element_size()
+        rgbs = raw_bytes / (us_r * 1e-6) / 1e9
+        rec["uncompressed_exact_attention"] = {
+            "what": "the same decode kernel over the raw K/V (count = NULL, every head n rows)",
+            "decode_tokens_per_s": w.B / (us_r * 1e-6 * full_L), "decode_bytes_per_step": raw_bytes * full_L,
+            "decode_us_per_launch": us_r, "decode_gbs": rgbs, "decode_frac": rgbs / peak,
+            "speedup_of_compressed": us_r / us_launch, "bytes_ratio": raw_bytes / layer_bytes}
+    if int(pipe.status.abs().max().item()) != 0 or int(pipe.cstatus.abs().max().item()) != 0:
+        raise RuntimeError(f"device-side error in sweep cell {label}")
+    del pipe
+    torch.cuda.empty_cache()
+    rec["clocks"] = sampler.summary(t0, time.time())
+    rec["cell_wall_s"] = round(time.time() - t0, 2)
+    return rec
+
+
+def sweep_configs(args, dev, sampler, peak):
+    """Short passes over the other workloads and the sweeps two of them name (after the headline run).
+
+    Every cell runs a reduced number of layers whose cores still exceed the L2 by a wide margin (the
+    toy workload excepted: it is L2-resident by definition and its fractions are informational)."""
+    out = {"what": "per cell: chained decode and compress on a reduced layer count (layers_run), rates scaled to "
+                   "layers_full; fractions of the measured HBM copy peak", "peak_gbs": peak}
+    c0, c2, c3, c4 = (synth.config(i) for i in (0, 2, 3, 4))
+    out["cfg0"] = measure_cell(c0, c0.L, dev, sampler, peak, {"workload": c0.name, "note": "L2-resident toy"},
+                               decode_steps=32)
+    out["cfg2"] = measure_cell(c2.replace(L=2), c2.L, dev, sampler, peak, {"workload": c2.name})
+    # cfg3: noise swept at tau = 0.9 (the norm reading of the noise), plus the literal reading where nothing merges
+    cells = []
+    for sigma in (0.05, 0.15, 0.3):
+        cells.append(measure_cell(c3.replace(L=6, sigma=sigma, tau=0.9), c3.L, dev, sampler, peak,
+                                  {"workload": c3.name, "sigma": sigma, "tau": 0.9, "noise_reading": "norm"}))
+    cells.append(measure_cell(c3.replace(L=2, sigma=0.15, tau=0.9, noise_reading="literal"), c3.L, dev, sampler, peak,
+                              {"workload": c3.name, "sigma": 0.15, "tau": 0.9, "noise_reading": "literal (no merge)"},
+                              cap_frac=1.0))
+    out["cfg3_sigma_sweep"] = cells
+    # cfg4: mean chunk length x target reduction, with exact attention over the raw cache on the same inputs
+    grid = []
+    for mean_len in (8, 32, 128):
+        for r in (2, 4, 8):
+            wc = c4.replace(L=2, gap=("poisson", float(mean_len)), centroids=("ratio", float(r)))
+            rec = measure_cell(wc, c4.L, dev, sampler, peak,
+                               {"workload": c4.name, "mean_chunk_len": mean_len, "target_reduction": r}, raw=True,
+                               cap_frac=1.0 if r == 2 else 0.5)
+            best = (mean_len + 1) / 2.0     # one core per chunk plus its delimiter
+            rec["reachable"] = r <= best
+            if not rec["reachable"]:
+                rec["note"] = f"unreachable: at best {best:.1f}x (one core per chunk plus the delimiter)"
+            grid.append(rec)
+    out["cfg4_grid"] = grid
+    return out
 
 
 def measure_append(pipe, m: int = 256, layers: int = 4):
@@ -348,7 +525,7 @@ def measure_append(pipe, m: int = 256, layers: int = 4):
             "host_bound_us_per_call_storing": med(plain), "host_bound_us_per_call_finishing_a_chunk": med(closing)}
 
 
-def run_e2e(pipe, args, barrier):
+def run_e2e(pipe, args, barrier, g_decode):
     """Same step with inputs in pinned HOST memory: H2D of ids/K/V/q and D2H of the outputs timed."""
     w, dev = pipe.w, pipe.dev
     steps = max(1, min(args.steps, args.e2e_steps))
@@ -388,7 +565,7 @@ def run_e2e(pipe, args, barrier):
                           pipe.cws[l], pipe.cstatus[l], 0)
         ev_done.record(main)
         pipe.q.copy_(host_q, non_blocking=True)
-        pipe.g_decode.replay()
+        g_decode.replay()
         host_out.copy_(pipe.out, non_blocking=True)
         for l in range(w.L):
             host_len[l].copy_(pipe.layers[l].core_len, non_blocking=True)
@@ -437,7 +614,12 @@ def cpu_baseline(w: synth.Workload, budget_s: float = 20.0):
     t_c, t_d = oracle_sample(ws, n_decode=2)
     del budget_s
     step_s = w.B * (w.L * t_c + w.decode_steps * w.L * t_d)
-    return {"value": w.B * w.decode_steps / step_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    threads = oracle.num_threads()
+    # the oracle's loops run in parallel over (sequence, KV head) for chunk/GSC/merge and over (sequence, query
+    # head) for attention: no more threads than that have work on the one-sequence sample
+    busy_c, busy_a = min(threads, ws.B * ws.Hkv), min(threads, ws.B * ws.Hq)
+    return {"value": w.B * w.decode_steps / step_s, "unit": UNIT, "cores": max(busy_c, busy_a), "kind": "oracle",
+            "threads_available": threads, "cores_with_work": {"chunk_gsc_merge": busy_c, "attention": busy_a},
             "sample": f"layer 0 of {w.L}, sequence 0 of {w.B}: chunk+GSC+merge once ({t_c:.2f} s) and 2 of "
                       f"{w.decode_steps} decode steps ({t_d * 1e3:.1f} ms each), scaled linearly to the full step",
             "compress_s_per_layer": t_c, "decode_s_per_layer_step": t_d}
@@ -468,7 +650,8 @@ def run_reference(args):
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "B": w.B, "n_ctx": w.n, "layers": w.L, "kv_heads": w.Hkv, "q_heads": w.Hq,
                    "head_dim": w.d, "tau": w.tau, "decode_steps": w.decode_steps},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": min(oracle.num_threads(), ws.B * ws.Hq), "kind": "oracle",
+                         "threads_available": oracle.num_threads(), "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0}))
 
@@ -484,7 +667,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small profiling cases)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-overlap", action="store_true", help="plain launches (no programmatic dependent launch)")
+    ap.add_argument("--no-overlap", action="store_true", help="time the step with plain stream-ordered decode launches")
+    ap.add_argument("--no-modes", action="store_true", help="skip the side measurements of the other decode launch modes")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the short passes over the other workloads and sweeps")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--traffic", type=float, default=None,

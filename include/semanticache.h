@@ -10,11 +10,14 @@
  *
  * General rules
  *   - Every pointer is a DEVICE pointer unless its comment says HOST.  The caller owns all
- *     buffers; the library allocates nothing and keeps no state between calls.
+ *     buffers; the library allocates nothing.  The state it keeps between calls: the launch
+ *     counter, per-GPU launch geometry looked up on first use, and, for sc_decode_attn_static
+ *     only, its fixed scratch array with the per-GPU address of that array.
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
  *     Calls return after enqueueing; they never synchronise.
  *   - The return value reports host-side validation only (SC_OK, SC_ERR_INVALID_ARG,
- *     SC_ERR_UNSUPPORTED, SC_ERR_CUDA for a failed launch).  Conditions found on the device
+ *     SC_ERR_UNSUPPORTED, SC_ERR_CUDA for a failed launch; sc_decode_attn_static alone also
+ *     returns SC_ERR_CAPACITY from the host for a shape beyond its fixed scratch).  Conditions found on the device
  *     are written to the caller's `status` word (int32, device or pinned host memory, may be
  *     NULL): it is left untouched on success and set to SC_ERR_CAPACITY / SC_ERR_TIMEOUT
  *     otherwise (first error wins).  The caller zeroes it beforehand.  Kernels never trap.
@@ -55,14 +58,27 @@ typedef enum { SC_BF16 = 0, SC_F32 = 1 } sc_dtype;
 #define SC_FLAG_TWO_PASS 2u    /* fused compress: count pass + write pass instead of the
                                   single pass whose tiles look back for their output offset */
 #define SC_FLAG_OVERLAP_PREV 4u /* sc_decode_attn, sc_compress (fused bf16 path, single pass): launch with
-                                  programmatic stream serialization and
-                                  do not wait for the kernel enqueued just before on this stream.
-                                  The caller promises that that kernel and this call share no
-                                  buffer that either of them writes (q, out, workspace, status and
-                                  the cores all count).  Independent calls, e.g. the layers of an
-                                  attention-only benchmark with one workspace per layer, then run
-                                  back to back without the launch gap.  A call without the flag
-                                  orders itself after everything enqueued before it, as usual. */
+                                  programmatic stream serialization, so that this kernel may start while
+                                  the kernels enqueued before it on this stream are still running.  The
+                                  caller promises that nothing this call READS before it writes (q, cores,
+                                  count, core_len; for sc_compress K, V and the chunk plan) is written by
+                                  any kernel of the unbroken run of overlapped launches before it, nor by
+                                  the kernel just before that run.  Every write of the call (out,
+                                  workspace, status; for sc_compress also cores, count, core_len, assign)
+                                  is ordered behind the completion of the kernel before it, and so on
+                                  back along the run: sc_decode_attn calls of one run may therefore share
+                                  their workspace and out buffers; sc_compress calls of one run must not
+                                  share a workspace or outputs (it writes throughout).  Independent
+                                  calls, e.g. the layers of an attention-only benchmark, then run back to
+                                  back without the launch gap.  A call without the flag orders itself
+                                  after everything enqueued before it, as usual. */
+#define SC_FLAG_OVERLAP_CHAIN 8u /* sc_decode_attn only: as SC_FLAG_OVERLAP_PREV, except that q MAY be the
+                                  product of the kernel just before this call (layer l+1's query follows
+                                  from layer l's output).  The kernel starts early, sends its share of the
+                                  cores on its way (first tiles to shared memory, the rest to L2), waits
+                                  for the preceding kernel to complete and only then reads q.  The cores,
+                                  count and core_len are still read early and fall under the promise
+                                  above.  Ignored (ordinary launch) on the generic path. */
 
 typedef struct {
     float tau;             /* similarity threshold of Algorithm 1; merge iff Sim > tau (strict) */
@@ -82,7 +98,7 @@ SC_API const char* sc_version(void);
 
 /*
  * Statistics: number of kernels this library has launched (or recorded into a CUDA graph under
- * stream capture) since it was loaded.  The only state the library keeps; it affects nothing.
+ * stream capture) since it was loaded.  It affects nothing.
  */
 SC_API uint64_t sc_launch_counter(void);
 
@@ -174,7 +190,8 @@ SC_API sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides
  *   core_len   [B, Hkv] int32 (device), each <= cap
  *   scale      0 means 1/sqrt(d)
  *   out        [B, Hq, d] contiguous, dtype dt; a head with core_len 0 gets zeros
- *   flags      SC_FLAG_GENERIC forces the generic kernels; SC_FLAG_OVERLAP_PREV (see above); else 0
+ *   flags      SC_FLAG_GENERIC forces the generic kernels; SC_FLAG_OVERLAP_PREV or
+ *              SC_FLAG_OVERLAP_CHAIN (see above); else 0
  *   workspace  at least sc_decode_workspace_bytes(B, Hq, Hkv, d, cap) bytes.  It holds the
  *              split partials and a few arrival counters; the counters must be zero on entry
  *              and are left zero on exit, so zero the workspace once after allocating it.

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libsemanticache.so")
 
 SC_OK, SC_ERR_INVALID_ARG, SC_ERR_UNSUPPORTED, SC_ERR_CAPACITY, SC_ERR_CUDA, SC_ERR_TIMEOUT = range(6)
 SC_BF16, SC_F32 = 0, 1
-SC_FLAG_GENERIC, SC_FLAG_TWO_PASS, SC_FLAG_OVERLAP_PREV = 1, 2, 4
+SC_FLAG_GENERIC, SC_FLAG_TWO_PASS, SC_FLAG_OVERLAP_PREV, SC_FLAG_OVERLAP_CHAIN = 1, 2, 4, 8
 SC_MAX_CHUNK_LEN, SC_MAX_DELIMS, SC_TILE_ROWS = 256, 64, 128
 _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CAPACITY", "SC_ERR_CUDA",
                  "SC_ERR_TIMEOUT"]

@@ -73,29 +73,6 @@ static_assert(kSmemBytes <= 76800, "three blocks per SM need <= 75 KB each");
 enum Mode { kCountOnly = 0, kWriteWithCounts = 1, kLookBack = 2 };
 enum Geo { gB = 0, gH = 1, gT = 2, gNseg = 3, gRow0 = 4, gR = 5, gLast = 6 };
 
-// Per-phase cycle totals for a debugging harness; compiled out of the library.
-#ifdef SC_PHASE_TIMING
-__device__ unsigned long long g_phase_cycles[16];
-#define CF_T(i)                                                                 \
-    do {                                                                        \
-        if (threadIdx.x == 0) {                                                 \
-            const long long now_ = clock64();                                   \
-            atomicAdd(&g_phase_cycles[i], (unsigned long long)(now_ - t_prev)); \
-            t_prev = now_;                                                      \
-        }                                                                       \
-    } while (0)
-// the same for a span measured by one lane of any warp
-#define CF_SPAN_BEGIN() const long long span_t0_ = clock64()
-#define CF_SPAN_END(i)                                                                             \
-    do {                                                                                           \
-        if ((threadIdx.x & 31) == 0) atomicAdd(&g_phase_cycles[i], (unsigned long long)(clock64() - span_t0_)); \
-    } while (0)
-#else
-#define CF_T(i)
-#define CF_SPAN_BEGIN()
-#define CF_SPAN_END(i)
-#endif
-
 // cnts[seed row] while the cluster waits to be pooled: kPending | first row of its segment | (one past its last
 // row) << 9, the latter 0 for a segment of up to 32 tokens, whose member mask is one segment-relative word
 constexpr uint32_t kPending = 1u << 31;
@@ -649,7 +626,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     int max_nt = 0;                        // most tiles any sequence has (service warp)
 
     // Let the next kernel of the stream start beside this one if it was launched with programmatic stream
-    // serialization (a no-op otherwise); this kernel itself never waits for its predecessor.
+    // serialization (a no-op otherwise); this kernel waits for its predecessor only at its very end.
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     if (tid == 0) {
         mbar_init(bar_k, 1);
@@ -672,9 +649,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     __syncthreads();
 
     int buf = 0;
-#ifdef SC_PHASE_TIMING
-    long long t_prev = clock64();
-#endif
     for (;;) {
         const int* geo = geo_buf + buf * 8;
         const int16_t* segs = segs_buf + buf * kSegsStride;
@@ -692,7 +666,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
             stage_rows(sbase, hs, &p.map_k, row0, R, h, b, bar_k, lane);
             if (two_tensors) stage_rows(sbase + kVOff, hs, &p.map_v, row0, R, h, b, bar_v, lane);
         }
-        CF_T(1);
         // end of the segment each row is in (0 past the tile)
         // also: one-token segments (delimiters, lone tokens) are clusters of their own -- no key needed;
         // the others are listed for the warps
@@ -719,7 +692,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
             }
         }
         for (int r = R + tid; r < nrb * 32; r += kThreads) send[r] = (uint16_t)0;
-        CF_T(0);
         failed = !mbar_wait(bar_k, phase_k);   // K has landed
         phase_k ^= 1u;
         if (two_tensors && !failed) {
@@ -727,7 +699,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
             phase_v ^= 1u;
         }
         if (__syncthreads_or(failed)) { failed = true; break; }
-        CF_T(2);
 
         // ---- 2. segments of more than kWarpSegMax tokens: Gram blocks -> norms -> adjacency bits in shared memory ----
         const int longblocks = misc[2];
@@ -752,17 +723,13 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
             }
             __syncthreads();
         }
-        CF_T(4);
 
         // ---- 3. the service warp draws the block's next ticket; compute warps: Algorithm 1 per segment,
         //         one warp each, in registers up to 32 tokens, else on the bit rows ----
         unsigned char* lane_base = smem + (lane >> 4) * kVOff + ((lane >> 3) & 1) * hs;   // see rows_add
         if (service) {
-            CF_SPAN_BEGIN();
             fetch_tile(p, lane, max_nt, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
-            CF_SPAN_END(10);
         } else {
-            CF_SPAN_BEGIN();
             const int nmulti = misc[3];
             for (int k = warp; k < nmulti; k += kWarps) {
                 const int s = multi[k];
@@ -801,11 +768,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 }
                 if (seeds) atomicOr(&seedmask[lane], seeds);
             }
-            if (warp == 0) CF_SPAN_END(11);
-            if (warp == 7) CF_SPAN_END(12);
         }
         __syncthreads();
-        CF_T(5);
 
         // ---- 4. cluster count of the tile, published at once.  Service warp: output offset of the tile
         //         (look-back).  Compute warps: the seed row of every cluster, and Eq. 3 ----
@@ -827,9 +791,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 }
                 compute_warps_sync();   // the table of seed rows is complete
                 pool_clusters(lane_base, seedrow, P, adj, cnts, warp, lane, long_tile ? 16 : 32);
-                CF_T(7);
             } else {
-                CF_SPAN_BEGIN();
                 if (kMode == kLookBack && lane == 0)
                     atomicExch(&stt[t], (t == 0 ? kFlagPrefix : kFlagAggregate) | (uint32_t)P);
                 int base = 0;
@@ -882,10 +844,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                         if (base + P > p.cap) set_status(p.status, SC_ERR_CAPACITY);
                     }
                 }
-                CF_SPAN_END(13);
             }
             __syncthreads();
-            CF_T(8);
 
             // ---- compact, coalesced stores of the cores: cluster `row` of the tile sits in its seed's staged row ----
             const int base = misc[0];
@@ -926,7 +886,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
         fence_async_proxy();   // the next tile's copies overwrite what ordinary accesses read and wrote
         __syncthreads();
-        CF_T(9);
         buf ^= 1;
     }
 
@@ -939,6 +898,9 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         mbar_wait(bar_v, phase_v);
     }
     __syncthreads();
+    // Under an overlapped launch a block does not finish before the kernel enqueued ahead of this one has
+    // completed, so completion is transitive along a run of overlapped launches (a no-op otherwise).
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
     if (tid == 0) {
         __threadfence();
         const int done = atomicAdd(&p.ctl[1], 1);
@@ -1063,13 +1025,3 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
 
 }  // namespace sc
 
-#ifdef SC_PHASE_TIMING
-extern "C" __attribute__((visibility("default"))) int sc_debug_phase_cycles(unsigned long long* host16, int reset) {
-    cudaError_t e = cudaMemcpyFromSymbol(host16, sc::cf::g_phase_cycles, 16 * sizeof(unsigned long long));
-    if (e == cudaSuccess && reset) {
-        unsigned long long z[16] = {0};
-        e = cudaMemcpyToSymbol(sc::cf::g_phase_cycles, z, sizeof(z));
-    }
-    return (int)e;
-}
-#endif

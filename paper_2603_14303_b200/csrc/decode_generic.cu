@@ -50,7 +50,7 @@ decode_generic(const T* __restrict__ q, int B, int Hq, int Hkv, int d, const T* 
             if (c < d) s = fmaf(qv[u], Elem<T>::load(kr + c), s);
         }
         s = warp_sum(s);
-        if (count != nullptr) s += log2f((float)count[cbase + t]);  // ln s, in base-2 units
+        if (count != nullptr) s += log2f((float)max(count[cbase + t], 1));  // ln s, in base-2 units (a valid row has count >= 1)
         const float mn = fmaxf(m, s);
         const float corr = exp2f(m - mn);  // m = -inf on the first row gives 0
         const float pw = exp2f(s - mn);

@@ -5,12 +5,22 @@
 // ldmatrix is conflict free) and fold the whole GQA group into one pass:
 //     S^T[16 keys x 8 heads]   = K_tile . q^T                (mma.m16n8k16, keys on M, heads on N)
 //     x = S^T * scale*log2(e) + log2(count)                  (Proportional Attention, base 2)
-//     P^T = 2^(x - m)  (online softmax; the running max is per head and common to the warp)
-//     O^T[128 dims x 8 heads] += V_tile^T . P^T              (ldmatrix.trans, P^T via movmatrix)
-// Warps are merged in a fixed order through shared memory, the block writes one (m, l, O)
-// partial, and the last block of a head to arrive (atomic ticket, no waiting) merges the
-// splits in order and writes the output, so results are bit-reproducible.
-#include <cstdlib>
+//     P^T = 2^(x - m)  (online softmax; the running max is per head, common to the warp, and
+//                       raised only when a score overtakes it by a margin)
+//     O^T[128 dims x 8 heads] += V_tile^T . P^T              (ldmatrix.trans, P^T via movmatrix,
+//                                                             as a bf16 pair: leading part + remainder)
+// Warps are merged in a fixed order through shared memory into one (m, l, O) partial per block.
+// When the launch is about one wave of blocks, the splits of a head form a thread-block cluster
+// and fold their partials through distributed shared memory, each block its own slice of the
+// output (no partial leaves the SMs); otherwise, or when a head needs several clusters, partials go
+// to global memory and the last block of a head to arrive (atomic ticket, no waiting) merges them.
+// Every order is fixed, so results are bit-reproducible.
+//
+// Launch modes: ordinary; overlapped with the preceding kernel (programmatic stream
+// serialization), where every global write waits for that kernel's completion; and chained, where
+// in addition q is read only after that wait (q is the preceding kernel's product) while the cores
+// were requested before it.
+#include <cooperative_groups.h>
 
 #include "common.cuh"
 
@@ -18,22 +28,7 @@ namespace sc {
 
 namespace dm {
 
-// Phase timestamps for a debugging harness; compiled out of the library.
-#ifdef SC_TIMELINE
-__device__ long long* g_timeline = nullptr;   // [launch][block][16]
-__device__ const char* g_timeline_out0 = nullptr;
-__device__ long long g_timeline_stride = 1;
-#define SC_T(i)                                                                                         \
-    do {                                                                                                \
-        if (g_timeline && threadIdx.x == 0) {                                                           \
-            long long* t_ = g_timeline + ((size_t)tl_launch * 1024 + tl_block) * 16;                    \
-            if ((i) == 0) { unsigned long long gt_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_)); t_[15] = (long long)gt_; } \
-            t_[i] = clock64();                                                                          \
-        }                                                                                               \
-    } while (0)
-#else
-#define SC_T(i)
-#endif
+namespace cg = cooperative_groups;
 
 constexpr int kWarps = 4;
 constexpr int kStages = 3;
@@ -47,6 +42,9 @@ constexpr int kSmemBytes = kWarps * kWarpBytes;
 constexpr int kPartStride = 8 * kD + 16;        // floats per (b, h, split): acc[8 heads][128], m[8], l[8]
 constexpr int kCtasPerSm = 2;                   // two kernels (consecutive layers) can be co-resident
 constexpr size_t kL2PrefetchBytes = 512 * 1024;  // per tensor and block
+constexpr float kMaxSlack = 8.f;                // log2 units a score may exceed the running maximum before it is raised
+constexpr int kMergeGroup = 16;                 // cluster partials folded per round by the merging block
+constexpr int kMaxCluster = 16;                 // blocks per cluster (more than 8 needs the non-portable opt-in)
 constexpr int kCapRowsPerSplit = 1408;           // of capacity (heads are usually half full or less): about 700 rows a block
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -97,20 +95,40 @@ __device__ __forceinline__ float fast_log2(float x) {
     return y;
 }
 
-// Copies rows [row0, row0+16) of one head's cores into a stage; rows >= len are zero-filled.
+__device__ __forceinline__ void store_out4(__nv_bfloat16* dst, const float4& acc, float inv) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dst) = pk;
+}
+
+// Copies rows [row0, row0+16) of one head's cores into a stage; rows >= len are zero-filled.  Lane l
+// moves 16-byte chunk l & 15 of rows 2i + (l >> 4), i = 0..7, to its swizzled place soff[i] (the same
+// for every tile, so the caller computes the eight offsets once).  A tile that lies wholly inside the
+// head -- all but the last one -- needs no per-row test.
 __device__ __forceinline__ void issue_tile(uint32_t stage, const __nv_bfloat16* __restrict__ kh,
                                            const __nv_bfloat16* __restrict__ vh, const int32_t* __restrict__ ch,
-                                           int row0, int len, int lane) {
+                                           int row0, int len, int lane, const uint32_t (&soff)[8]) {
+    const size_t g0 = (size_t)(row0 + (lane >> 4)) * kD + (lane & 15) * 8;
+    if (row0 + kTile <= len) {
+        const __nv_bfloat16* ks = kh + g0;
+        const __nv_bfloat16* vs = vh + g0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            cp_async16(stage + soff[i], ks + i * 2 * kD, 16);
+            cp_async16(stage + kTileBytes + soff[i], vs + i * 2 * kD, 16);
+        }
+        if (ch != nullptr && lane < kTile) cp_async4(stage + 2 * kTileBytes + lane * 4, ch + row0 + lane, 4);
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const int idx = i * 32 + lane;          // 256 chunks of 16 B per tile
-        const int r = idx >> 4, c = idx & 15;
-        const int row = row0 + r;
-        const bool ok = row < len;
-        const size_t goff = (size_t)(ok ? row : 0) * kD + c * 8;
-        const uint32_t soff = r * kRowBytes + ((c ^ (r & 7)) << 4);
-        cp_async16(stage + soff, kh + goff, ok ? 16 : 0);
-        cp_async16(stage + kTileBytes + soff, vh + goff, ok ? 16 : 0);
+        const bool ok = row0 + 2 * i + (lane >> 4) < len;
+        const size_t goff = ok ? g0 + (size_t)i * 2 * kD : 0;
+        cp_async16(stage + soff[i], kh + goff, ok ? 16 : 0);
+        cp_async16(stage + kTileBytes + soff[i], vh + goff, ok ? 16 : 0);
     }
     if (ch != nullptr && lane < kTile) {
         const int row = row0 + lane;
@@ -122,7 +140,7 @@ __device__ __forceinline__ void issue_tile(uint32_t stage, const __nv_bfloat16* 
 __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
 decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __nv_bfloat16* __restrict__ core_k,
                   const __nv_bfloat16* __restrict__ core_v, const int32_t* __restrict__ count, int cap,
-                  const int32_t* __restrict__ core_len, float scale_log2, int n_split,
+                  const int32_t* __restrict__ core_len, float scale_log2, int n_split, int q_from_prev,
                   __nv_bfloat16* __restrict__ out, float* __restrict__ part, int32_t* __restrict__ tickets) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ float sh_m[kWarps][8];
@@ -132,18 +150,14 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, tig = lane & 3;
     const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-#ifdef SC_TIMELINE
-    const int tl_launch = (int)(((const char*)out - g_timeline_out0) / g_timeline_stride), tl_block = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
-#endif
-    SC_T(0);
     const int G = Hq / Hkv;
     const int bh = b * Hkv + h;
     // Let the next kernel of the stream start beside this one if it was launched with programmatic
-    // stream serialization (a no-op otherwise).
+    // stream serialization (a no-op otherwise).  Whatever this block reads before its own
+    // griddepcontrol.wait below (core_len, cores, counts) must not be written by a kernel that may
+    // still be running then; that is the caller's promise when it asks for an overlapped launch.
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     const int len = max(min(core_len[bh], cap), 0);
-
-    SC_T(1);
     const int tiles_total = (len + kTile - 1) / kTile;
     const int tiles_per_split = (tiles_total + n_split - 1) / n_split;
     const int t0 = min(split * tiles_per_split, tiles_total);
@@ -171,17 +185,24 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
         }
     }
 
+    uint32_t soff[8];   // this lane's eight chunk places inside a K or V tile (see issue_tile)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 2 * i + (lane >> 4), c = lane & 15;
+        soff[i] = r * kRowBytes + ((c ^ (r & 7)) << 4);
+    }
+
     // prologue: fill the ring
 #pragma unroll
     for (int s = 0; s < kStages - 1; ++s) {
-        if (s < my_tiles) issue_tile(wbase + s * kStageBytes, kh, vh, ch, (t0 + warp + s * kWarps) * kTile, len, lane);
+        if (s < my_tiles) issue_tile(wbase + s * kStageBytes, kh, vh, ch, (t0 + warp + s * kWarps) * kTile, len, lane, soff);
         cp_async_commit();
     }
 
-    // Under an overlapped launch the caller has promised that the preceding kernel shares no
-    // buffer with this call, so nothing is waited for; an ordinary launch is already ordered.
-    SC_T(2);
-    SC_T(3);
+    // Chained launch (SC_FLAG_OVERLAP_CHAIN): q is the preceding kernel's product.  The cores' first
+    // tiles are on their way to shared memory and the rest of the block's share to L2; only now wait
+    // for that kernel to complete (and its writes to be visible), then read q.
+    if (q_from_prev) asm volatile("griddepcontrol.wait;\n" ::: "memory");
 
     // q^T as the B operand of every k-step: b0 = q[head g][16ks + 2tig, +1], b1 = same + 8
     uint32_t qb[8][2];
@@ -189,12 +210,11 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
         const __nv_bfloat16* qh = q + ((size_t)b * Hq + (size_t)h * G + g) * kD;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-            qb[ks][0] = (g < G) ? *reinterpret_cast<const uint32_t*>(qh + ks * 16 + 2 * tig) : 0u;
-            qb[ks][1] = (g < G) ? *reinterpret_cast<const uint32_t*>(qh + ks * 16 + 2 * tig + 8) : 0u;
+            // read through L2: under a chained launch q was written while this kernel was already running
+            qb[ks][0] = (g < G) ? __ldcg(reinterpret_cast<const uint32_t*>(qh + ks * 16 + 2 * tig)) : 0u;
+            qb[ks][1] = (g < G) ? __ldcg(reinterpret_cast<const uint32_t*>(qh + ks * 16 + 2 * tig + 8)) : 0u;
         }
     }
-
-    SC_T(4);
     float o[8][4];
 #pragma unroll
     for (int mt = 0; mt < 8; ++mt) { o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f; }
@@ -208,7 +228,7 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
     for (int i = 0; i < my_tiles; ++i) {
         const int pre = i + kStages - 1;
         if (pre < my_tiles)
-            issue_tile(wbase + (pre % kStages) * kStageBytes, kh, vh, ch, (t0 + warp + pre * kWarps) * kTile, len, lane);
+            issue_tile(wbase + (pre % kStages) * kStageBytes, kh, vh, ch, (t0 + warp + pre * kWarps) * kTile, len, lane, soff);
         cp_async_commit();
         cp_async_wait<kStages - 1>();
         __syncwarp();
@@ -216,15 +236,18 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
         const uint32_t st = wbase + (i % kStages) * kStageBytes;
         const int row0 = (t0 + warp + i * kWarps) * kTile;
 
-        // S^T = K . q^T, two accumulator chains
+        // S^T = K . q^T, four accumulator chains
         float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+        float sc2[4] = {0.f, 0.f, 0.f, 0.f}, sd[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
             uint32_t a0, a1, a2, a3;
             const int c = 2 * ks + k_csel;
             ldmatrix_x4(st + k_row * kRowBytes + ((c ^ (k_row & 7)) << 4), a0, a1, a2, a3);
-            if (ks & 1) mma_bf16(sb, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
-            else mma_bf16(sa, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+            if ((ks & 3) == 0) mma_bf16(sa, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+            else if ((ks & 3) == 1) mma_bf16(sb, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+            else if ((ks & 3) == 2) mma_bf16(sc2, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+            else mma_bf16(sd, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
         }
         float lc_lo = 0.f, lc_hi = 0.f;
         if (ch != nullptr) {
@@ -233,29 +256,39 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
             lc_hi = fast_log2((float)max(cs[g + 8], 1));
         }
         const bool ok_lo = row0 + g < len, ok_hi = row0 + g + 8 < len;
-        const float x0 = ok_lo ? fmaf(sa[0] + sb[0], scale_log2, lc_lo) : -INFINITY;
-        const float x1 = ok_lo ? fmaf(sa[1] + sb[1], scale_log2, lc_lo) : -INFINITY;
-        const float x2 = ok_hi ? fmaf(sa[2] + sb[2], scale_log2, lc_hi) : -INFINITY;
-        const float x3 = ok_hi ? fmaf(sa[3] + sb[3], scale_log2, lc_hi) : -INFINITY;
-        float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
+        const float x0 = ok_lo ? fmaf((sa[0] + sb[0]) + (sc2[0] + sd[0]), scale_log2, lc_lo) : -INFINITY;
+        const float x1 = ok_lo ? fmaf((sa[1] + sb[1]) + (sc2[1] + sd[1]), scale_log2, lc_lo) : -INFINITY;
+        const float x2 = ok_hi ? fmaf((sa[2] + sb[2]) + (sc2[2] + sd[2]), scale_log2, lc_hi) : -INFINITY;
+        const float x3 = ok_hi ? fmaf((sa[3] + sb[3]) + (sc2[3] + sd[3]), scale_log2, lc_hi) : -INFINITY;
+        // The running maxima m0, m1 are common to the warp.  They are raised only when some lane meets a
+        // score more than kMaxSlack above them (one vote per tile instead of a shuffle reduction): the
+        // weights 2^(x - m) then stay below 2^kMaxSlack, which fp32 sums and bf16 weights carry without loss.
+        const float lx0 = fmaxf(x0, x2), lx1 = fmaxf(x1, x3);
+        if (__any_sync(kFull, (lx0 > m0 + kMaxSlack) || (lx1 > m1 + kMaxSlack))) {
+            float mx0 = lx0, mx1 = lx1;
 #pragma unroll
-        for (int off = 4; off < 32; off <<= 1) {
-            mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, off));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, off));
-        }
-        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: a tile has a valid row
-        if (__any_sync(kFull, (mn0 != m0) || (mn1 != m1))) {
+            for (int off = 4; off < 32; off <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, off));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, off));
+            }
+            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: a tile has a valid row
             const float c0 = fast_exp2(m0 - mn0), c1 = fast_exp2(m1 - mn1);
             l0 *= c0; l1 *= c1;
 #pragma unroll
             for (int mt = 0; mt < 8; ++mt) { o[mt][0] *= c0; o[mt][2] *= c0; o[mt][1] *= c1; o[mt][3] *= c1; }
             m0 = mn0; m1 = mn1;
         }
-        const uint32_t p_lo = pack_bf16x2(fast_exp2(x0 - m0), fast_exp2(x1 - m1));   // row g
-        const uint32_t p_hi = pack_bf16x2(fast_exp2(x2 - m0), fast_exp2(x3 - m1));   // row g + 8
-        l0 += bf16_lo(p_lo) + bf16_lo(p_hi);
-        l1 += bf16_hi(p_lo) + bf16_hi(p_hi);
+        // The weights enter the second product as bf16 pairs (leading part + remainder), which keeps
+        // sixteen bits of each: a single bf16 rounding of P would be the largest error of the whole path.
+        const float w0 = fast_exp2(x0 - m0), w1 = fast_exp2(x1 - m1);   // row g
+        const float w2 = fast_exp2(x2 - m0), w3 = fast_exp2(x3 - m1);   // row g + 8
+        const uint32_t p_lo = pack_bf16x2(w0, w1), p_hi = pack_bf16x2(w2, w3);
+        const uint32_t r_lo = pack_bf16x2(w0 - bf16_lo(p_lo), w1 - bf16_hi(p_lo));
+        const uint32_t r_hi = pack_bf16x2(w2 - bf16_lo(p_hi), w3 - bf16_hi(p_hi));
+        l0 += (bf16_lo(p_lo) + bf16_lo(r_lo)) + (bf16_lo(p_hi) + bf16_lo(r_hi));
+        l1 += (bf16_hi(p_lo) + bf16_hi(r_lo)) + (bf16_hi(p_hi) + bf16_hi(r_hi));
         const uint32_t pb0 = movmatrix_trans(p_lo), pb1 = movmatrix_trans(p_hi);
+        const uint32_t rb0 = movmatrix_trans(r_lo), rb1 = movmatrix_trans(r_hi);
 
         // O^T += V^T . P^T
 #pragma unroll
@@ -264,11 +297,11 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
             const int c = 2 * mt + v_csel;
             ldmatrix_x4_trans(st + kTileBytes + v_row * kRowBytes + ((c ^ (v_row & 7)) << 4), a0, a1, a2, a3);
             mma_bf16(o[mt], a0, a1, a2, a3, pb0, pb1);
+            mma_bf16(o[mt], a0, a1, a2, a3, rb0, rb1);
         }
         __syncwarp();
     }
     cp_async_wait<0>();
-    SC_T(5);
 
     // ---- merge the warps of this block (fixed order) ----
     // lane-local l covers rows g, g+8 of every tile: sum over the 8 row groups
@@ -297,15 +330,25 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
         slab[(2 * tig + 1) * kD + d0 + 8] = o[mt][3] * f1;
     }
     __syncthreads();
-    float* my_part = part + ((size_t)bh * n_split + split) * kPartStride;
+    // Nothing has been written to global memory so far.  Under an overlapped launch every write of
+    // this kernel (partials, arrival counters, out) is ordered behind the completion of the kernel
+    // before it, which ordered its own writes behind its predecessor in the same way: completion is
+    // transitive along a run of overlapped launches, and they may share workspace and out buffers.
+    // (A no-op for an ordinary launch and after the wait above.)
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+    // ---- block partial (m, l, O) into this block's shared memory, behind the warps' slabs ----
     const float* slabs = reinterpret_cast<const float*>(smem);
-    for (int e = threadIdx.x; e < G * kD; e += kWarps * 32) {
-        float acc = 0.f;
+    float* blk = reinterpret_cast<float*>(smem) + kWarps * (8 * kD);   // [8][128] O, [8] m, [8] l
+    for (int e4 = threadIdx.x; e4 < G * (kD / 4); e4 += kWarps * 32) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int w2 = 0; w2 < kWarps; ++w2) acc += slabs[w2 * (8 * kD) + e];
-        my_part[e] = acc;
+        for (int w2 = 0; w2 < kWarps; ++w2) {
+            const float4 v = *reinterpret_cast<const float4*>(slabs + w2 * (8 * kD) + e4 * 4);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        *reinterpret_cast<float4*>(blk + e4 * 4) = acc;
     }
-    if (threadIdx.x < G) {
+    if (threadIdx.x < 8) {
         const int hd = threadIdx.x;
         float bm = -INFINITY, bl = 0.f;
 #pragma unroll
@@ -315,68 +358,112 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
             const float mw = sh_m[w2][hd];
             bl += (mw == -INFINITY) ? 0.f : sh_l[w2][hd] * fast_exp2(mw - bm);
         }
-        my_part[8 * kD + hd] = bm;
-        my_part[8 * kD + 8 + hd] = bl;
+        blk[8 * kD + hd] = bm;
+        blk[8 * kD + 8 + hd] = bl;
     }
 
-    // ---- the last block of this head to arrive merges the splits ----
-    SC_T(6);
-    __threadfence();
-    __syncthreads();
-    SC_T(7);
+    // ---- the splits of one thread-block cluster are folded through distributed shared memory ----
+    // Every block of the cluster folds its own slice of the (head, column) pairs, reading that slice of
+    // every member's partial straight out of the member's shared memory (no trip through L2, no counter,
+    // and no single block pulling all partials through its own port); the members stay until all have read.
+    cg::cluster_group cluster = cg::this_cluster();
+    const int csize = (int)cluster.num_blocks(), crank = (int)cluster.block_rank();
+    const int n_clusters = n_split / csize, cidx = split / csize;   // clusters per head, this one's index
+    float* my_part = part + ((size_t)bh * n_clusters + cidx) * kPartStride;
+    const bool direct = n_clusters == 1;   // this cluster holds the whole head: its fold is the result
+    const int slice = (G * (kD / 4) + csize - 1) / csize;
+    cluster.sync();
+    for (int i = threadIdx.x; i < slice; i += kWarps * 32) {
+        const int e4 = crank * slice + i;
+        if (e4 >= G * (kD / 4)) break;
+        const int hd = e4 / (kD / 4), d4 = (e4 % (kD / 4)) * 4;
+        float mv[kMaxCluster], lv[kMaxCluster];
+        float4 ov[kMaxCluster];
+#pragma unroll
+        for (int j = 0; j < kMaxCluster; ++j) {
+            const float* pb = cluster.map_shared_rank(blk, j < csize ? j : 0);
+            mv[j] = j < csize ? pb[8 * kD + hd] : -INFINITY;
+            lv[j] = j < csize ? pb[8 * kD + 8 + hd] : 0.f;
+            ov[j] = j < csize ? *reinterpret_cast<const float4*>(pb + hd * kD + d4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float gm = mv[0];
+#pragma unroll
+        for (int j = 1; j < kMaxCluster; ++j) gm = fmaxf(gm, mv[j]);
+        float lsum = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < kMaxCluster; ++j) {
+            const float w = (mv[j] == -INFINITY) ? 0.f : fast_exp2(mv[j] - gm);
+            lsum = fmaf(w, lv[j], lsum);
+            acc.x = fmaf(w, ov[j].x, acc.x); acc.y = fmaf(w, ov[j].y, acc.y);
+            acc.z = fmaf(w, ov[j].z, acc.z); acc.w = fmaf(w, ov[j].w, acc.w);
+        }
+        if (direct) {
+            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+            store_out4(out + ((size_t)b * Hq + (size_t)h * G + hd) * kD + d4, acc, inv);
+        } else {
+            *reinterpret_cast<float4*>(my_part + hd * kD + d4) = acc;
+            if (d4 == 0) { my_part[8 * kD + hd] = gm; my_part[8 * kD + 8 + hd] = lsum; }
+        }
+    }
+    if (!direct) __threadfence();   // this block's slice of the cluster partial, before the cluster's ticket
+    cluster.sync();   // every member's shared memory has been read: they may leave
+    if (direct || crank != 0) return;
+
+    // ---- several clusters per head: the last of them to arrive merges their partials ----
+    // The cluster barrier above orders every member's (fenced) partial stores before this block's
+    // ticket, whose release makes them visible to whoever reads the ticket with acquire (the last
+    // cluster); that block's other threads are ordered behind its thread 0 by the barrier below and read
+    // the partials from L2.
     if (threadIdx.x == 0) {
-        const int t = atomicAdd(&tickets[bh], 1);
-        sh_last = (t == n_split - 1);
+        int t;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;\n" : "=r"(t) : "l"(tickets + bh) : "memory");
+        sh_last = (t == n_clusters - 1);
         if (sh_last) tickets[bh] = 0;   // leave the counter ready for the next call
     }
     __syncthreads();
-    SC_T(8);
     if (!sh_last) return;
-    __threadfence();
-    const float* hp = part + (size_t)bh * n_split * kPartStride;
-    float* wgt = reinterpret_cast<float*>(smem);            // [n_split][8] weights, then [8] 1/l
-    float* lraw = wgt + n_split * 8 + 8;                     // [n_split][8]
-    for (int idx = threadIdx.x; idx < n_split * 8; idx += kWarps * 32) {
-        const int s = idx >> 3, hd = idx & 7;
-        wgt[idx] = __ldcg(hp + (size_t)s * kPartStride + 8 * kD + hd);
-        lraw[idx] = __ldcg(hp + (size_t)s * kPartStride + 8 * kD + 8 + hd);
-    }
-    __syncthreads();
-    if (threadIdx.x < 8) {
-        const int hd = threadIdx.x;
-        float gm = -INFINITY;
-        for (int s = 0; s < n_split; ++s) gm = fmaxf(gm, wgt[s * 8 + hd]);
-        float lsum = 0.f;
-        for (int s = 0; s < n_split; ++s) {
-            const float ms = wgt[s * 8 + hd];
-            const float w = (ms == -INFINITY) ? 0.f : fast_exp2(ms - gm);
-            wgt[s * 8 + hd] = w;
-            lsum = fmaf(w, lraw[s * 8 + hd], lsum);
-        }
-        wgt[n_split * 8 + hd] = lsum > 0.f ? 1.f / lsum : 0.f;
-    }
-    __syncthreads();
+    // One thread per (head, four output columns); the partials are folded sixteen at a time, all of a
+    // group's loads in flight together (one round trip to L2 per group).
+    const float* hp = part + (size_t)bh * n_clusters * kPartStride;
     for (int e4 = threadIdx.x; e4 < G * (kD / 4); e4 += kWarps * 32) {
         const int hd = e4 / (kD / 4), d4 = (e4 % (kD / 4)) * 4;
-        const float* src = hp + hd * kD + d4;
+        float gm = -INFINITY, lsum = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 8
-        for (int s = 0; s < n_split; ++s) {
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(src + (size_t)s * kPartStride));
-            const float w = wgt[s * 8 + hd];
-            acc.x = fmaf(w, v.x, acc.x); acc.y = fmaf(w, v.y, acc.y);
-            acc.z = fmaf(w, v.z, acc.z); acc.w = fmaf(w, v.w, acc.w);
+        for (int s0 = 0; s0 < n_clusters; s0 += kMergeGroup) {
+            float mv[kMergeGroup], lv[kMergeGroup];
+            float4 ov[kMergeGroup];
+#pragma unroll
+            for (int j = 0; j < kMergeGroup; ++j) {
+                const bool ok = s0 + j < n_clusters;
+                const float* sp = hp + (size_t)(ok ? s0 + j : 0) * kPartStride;
+                mv[j] = ok ? __ldcg(sp + 8 * kD + hd) : -INFINITY;
+                lv[j] = ok ? __ldcg(sp + 8 * kD + 8 + hd) : 0.f;
+                ov[j] = ok ? __ldcg(reinterpret_cast<const float4*>(sp + hd * kD + d4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            float cm = mv[0];
+#pragma unroll
+            for (int j = 1; j < kMergeGroup; ++j) cm = fmaxf(cm, mv[j]);
+            const float ngm = fmaxf(gm, cm);
+            if (ngm == -INFINITY) continue;   // nothing but empty splits so far
+            const float c = (gm == -INFINITY) ? 0.f : fast_exp2(gm - ngm);
+            lsum *= c; acc.x *= c; acc.y *= c; acc.z *= c; acc.w *= c;
+            gm = ngm;
+#pragma unroll
+            for (int j = 0; j < kMergeGroup; ++j) {
+                const float w = (mv[j] == -INFINITY) ? 0.f : fast_exp2(mv[j] - gm);
+                lsum = fmaf(w, lv[j], lsum);
+                acc.x = fmaf(w, ov[j].x, acc.x); acc.y = fmaf(w, ov[j].y, acc.y);
+                acc.z = fmaf(w, ov[j].z, acc.z); acc.w = fmaf(w, ov[j].w, acc.w);
+            }
         }
-        const float inv = wgt[n_split * 8 + hd];
-        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-        __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-        uint2 pk;
-        pk.x = *reinterpret_cast<uint32_t*>(&lo);
-        pk.y = *reinterpret_cast<uint32_t*>(&hi);
-        *reinterpret_cast<uint2*>(out + ((size_t)b * Hq + (size_t)h * G + hd) * kD + d4) = pk;
+        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+        store_out4(out + ((size_t)b * Hq + (size_t)h * G + hd) * kD + d4, acc, inv);
     }
-    SC_T(9);
 }
+
+// Block split of one head: how many blocks stream it, and how they are grouped into clusters.
+struct SplitPlan { int n_split, cluster; };
 
 inline int splits_for(int B, int Hkv, int cap, int sms) {
     const int heads = B * Hkv;
@@ -391,11 +478,30 @@ inline int splits_for(int B, int Hkv, int cap, int sms) {
     return s < 1 ? 1 : s;
 }
 
+// Splits are grouped into clusters whose blocks fold their partials through distributed shared memory
+// when the whole launch is about one wave of blocks (few heads: the latency of the merge is then a large
+// part of the launch).  One cluster per head (no partial ever leaves the SMs) whenever the wanted split count is within a
+// quarter of the largest cluster; otherwise as few equal clusters as cover it.
+inline SplitPlan plan_for(int B, int Hkv, int cap, int sms, int cmax) {
+    const int s0 = splits_for(B, Hkv, cap, sms);
+    if (s0 <= 1 || cmax <= 1) return {s0, 1};
+    // Several waves of blocks (many heads): a block that waits at a cluster barrier holds an SM slot the next
+    // wave wants, and the merge is a small part of such a launch; there every block is a cluster of its own,
+    // leaves its partial in global memory and goes (measured: clusters of 6 cost 7 % at 128 heads x 8K rows).
+    if ((long long)B * Hkv * s0 > 2LL * sms) return {s0, 1};
+    if (s0 <= cmax + cmax / 4) { const int c = s0 < cmax ? s0 : cmax; return {c, c}; }
+    const int k = (s0 + cmax - 1) / cmax, c = s0 / k;
+    return {c * k, c};
+}
+
 }  // namespace dm
 
 bool decode_mma_supported(const DecodeArgs& a) {
     return a.dt == SC_BF16 && a.d == dm::kD && (a.Hq / a.Hkv) <= 8 && a.cap > 0 && a.Hkv <= 65535 && a.B <= 65535;
 }
+
+// Bytes at the front of the workspace that hold the arrival counters (zero between calls).
+size_t decode_mma_counter_bytes(int32_t B, int32_t Hkv) { return sizeof(int32_t) * (((size_t)B * Hkv + 63) / 64 * 64); }
 
 size_t decode_mma_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap) {
     (void)Hq; (void)d;
@@ -403,15 +509,13 @@ size_t decode_mma_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_
     const int s = dm::splits_for(B, Hkv, cap, 256);
     const int s2 = dm::splits_for(B, Hkv, cap, 132);
     int smax = s > s2 ? s : s2;
-#ifdef SC_TUNE
-    if (smax < 64) smax = 64;
-#endif
-    return 256 + sizeof(int32_t) * (((size_t)B * Hkv + 63) / 64 * 64) +
+    return 256 + decode_mma_counter_bytes(B, Hkv) +
            sizeof(float) * (size_t)B * Hkv * smax * dm::kPartStride;
 }
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
-    static int sms_of[64] = {0};   // per device: SM count, and the opt-in to large dynamic shared memory
+    // per device: SM count, the opt-in to large dynamic shared memory, and the largest cluster that can be scheduled
+    static int sms_of[64] = {0}, cmax_of[64] = {0};
     int dev = 0;
     cudaGetDevice(&dev);
     dev &= 63;
@@ -419,30 +523,46 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
         int v = 0;
         cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
         cudaFuncSetAttribute(dm::decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dm::kSmemBytes);
+        int cmax = 8;   // the portable cluster size
+        if (cudaFuncSetAttribute(dm::decode_mma_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+            cudaLaunchConfig_t probe = {};
+            probe.gridDim = dim3(dm::kMaxCluster, 1, 1);
+            probe.blockDim = dim3(dm::kWarps * 32);
+            probe.dynamicSmemBytes = dm::kSmemBytes;
+            cudaLaunchAttribute pa[1];
+            pa[0].id = cudaLaunchAttributeClusterDimension;
+            pa[0].val.clusterDim.x = dm::kMaxCluster; pa[0].val.clusterDim.y = 1; pa[0].val.clusterDim.z = 1;
+            probe.attrs = pa;
+            probe.numAttrs = 1;
+            int n_clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&n_clusters, dm::decode_mma_kernel, &probe) == cudaSuccess && n_clusters > 0)
+                cmax = dm::kMaxCluster;
+        }
+        (void)cudaGetLastError();   // a refused opt-in or probe is not an error of this call
+        cmax_of[dev] = cmax;
         sms_of[dev] = v > 256 ? 256 : (v < 1 ? 1 : v);
     }
-    const int sms = sms_of[dev];
-    int n_split = dm::splits_for(a.B, a.Hkv, a.cap, sms);
-#ifdef SC_TUNE   // tuning harness only
-    if (const char* e = getenv("SC_DEC_SPLITS")) n_split = atoi(e);
-#endif
+    const dm::SplitPlan plan = dm::plan_for(a.B, a.Hkv, a.cap, sms_of[dev], cmax_of[dev]);
     int32_t* tickets = (int32_t*)a.ws;
-    float* part = (float*)((char*)a.ws + sizeof(int32_t) * (((size_t)a.B * a.Hkv + 63) / 64 * 64));
+    float* part = (float*)((char*)a.ws + decode_mma_counter_bytes(a.B, a.Hkv));
     const float scale = (a.scale == 0.f ? 1.f / sqrtf((float)a.d) : a.scale) * 1.4426950408889634f;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(n_split, a.Hkv, a.B);
+    cfg.gridDim = dim3(plan.n_split, a.Hkv, a.B);
     cfg.blockDim = dim3(dm::kWarps * 32);
     cfg.dynamicSmemBytes = dm::kSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = plan.cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (a.flags & SC_FLAG_OVERLAP_PREV) ? 1 : 0;
+    cfg.numAttrs = (a.flags & (SC_FLAG_OVERLAP_PREV | SC_FLAG_OVERLAP_CHAIN)) ? 2 : 1;
+    const int q_from_prev = (a.flags & SC_FLAG_OVERLAP_CHAIN) ? 1 : 0;
     note_launches(1);
     return cudaLaunchKernelEx(&cfg, dm::decode_mma_kernel, (const __nv_bfloat16*)a.q, a.Hq, a.Hkv,
                               (const __nv_bfloat16*)a.core_k, (const __nv_bfloat16*)a.core_v, a.count, a.cap,
-                              a.core_len, scale, n_split, (__nv_bfloat16*)a.out, part, tickets);
+                              a.core_len, scale, plan.n_split, q_from_prev, (__nv_bfloat16*)a.out, part, tickets);
 }
 
 }  // namespace sc

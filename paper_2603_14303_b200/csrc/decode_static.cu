@@ -42,22 +42,38 @@ cudaError_t static_scratch(void** out) {
 
 }  // namespace
 
+namespace sc {
+bool decode_mma_supported(const DecodeArgs& a);
+size_t decode_mma_counter_bytes(int32_t B, int32_t Hkv);
+}  // namespace sc
+
 extern "C" sc_status sc_decode_attn_static(const void* q, sc_dtype dt, int32_t B, int32_t Hq, int32_t Hkv,
                                            int32_t d, const void* core_k, const void* core_v,
                                            const int32_t* count, int32_t cap, const int32_t* core_len,
                                            float scale, uint32_t flags, void* out, int32_t* status,
                                            void* stream) {
-    if (B < 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || cap < 0) return SC_ERR_INVALID_ARG;
-    // The overlapped launch relies on one workspace per in-flight call; here there is only one.
-    if (flags & SC_FLAG_OVERLAP_PREV) return SC_ERR_INVALID_ARG;
+    // The same checks, in the same order, as sc_decode_attn makes before it looks at its workspace.
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || cap < 0 || (Hq % Hkv) != 0) return SC_ERR_INVALID_ARG;
+    if (dt != SC_BF16 && dt != SC_F32) return SC_ERR_UNSUPPORTED;
+    if (d < 8 || d > 256 || (d % 8) != 0) return SC_ERR_UNSUPPORTED;
+    if (!(scale == scale) || scale < 0.f) return SC_ERR_INVALID_ARG;
+    // An overlapped launch would run beside its neighbour's clearing of the one shared array.
+    if (flags & (SC_FLAG_OVERLAP_PREV | SC_FLAG_OVERLAP_CHAIN)) return SC_ERR_INVALID_ARG;
+    if (B == 0) return SC_OK;
     const size_t need = sc_decode_workspace_bytes(B, Hq, Hkv, d, cap);
     if (need > (size_t)SC_STATIC_SCRATCH_BYTES) return SC_ERR_CAPACITY;   // problem too large for the fixed array
-    if (B == 0) return SC_OK;
     void* scratch = nullptr;
     if (static_scratch(&scratch) != cudaSuccess) return SC_ERR_CUDA;
-    // The array still holds whatever the previous call (or an aborted one) left: the arrival
-    // counters must start at zero, so the part this call uses is cleared first, in stream order.
-    if (cudaMemsetAsync(scratch, 0, need, (cudaStream_t)stream) != cudaSuccess) return SC_ERR_CUDA;
+    // The array still holds whatever the previous call (or an aborted one) left.  Only the arrival
+    // counters at its front must start at zero (the tensor-core kernel's; the generic kernels keep
+    // none): every split partial is written by its block before the merging block reads it.  They
+    // are cleared here, in stream order, before the kernel runs.
+    sc::DecodeArgs probe = {};
+    probe.dt = dt; probe.B = B; probe.Hq = Hq; probe.Hkv = Hkv; probe.d = d; probe.cap = cap;
+    if (!(flags & SC_FLAG_GENERIC) && sc::decode_mma_supported(probe)) {
+        if (cudaMemsetAsync(scratch, 0, sc::decode_mma_counter_bytes(B, Hkv), (cudaStream_t)stream) != cudaSuccess)
+            return SC_ERR_CUDA;
+    }
     return sc_decode_attn(q, dt, B, Hq, Hkv, d, core_k, core_v, count, cap, core_len, scale, flags, out, scratch,
                           (size_t)SC_STATIC_SCRATCH_BYTES, status, stream);
 }

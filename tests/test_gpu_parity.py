@@ -453,3 +453,79 @@ def test_overlapped_independent_layer_launches_match_ordinary_ones():
         assert_close_vectors(to_f64(plain[2, l]), want, 1e-2, f"layer {l}")
     for x in ws:
         assert int(x.view(torch.int32)[:64].abs().max()) == 0, "arrival counters are left at zero"
+
+
+def _bf16_bits(x64: np.ndarray) -> np.ndarray:
+    """float64 -> bf16 bit patterns (uint16), via torch's round-to-nearest-even conversion."""
+    return torch.from_numpy(x64).to(torch.float32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("share_workspace", [False, True])
+def test_chained_layer_launches_where_each_query_is_the_previous_output(share_workspace):
+    """SC_FLAG_OVERLAP_CHAIN: layer l+1's query IS layer l's output (same shape), the launches go back to
+    back.  The chained launches must equal ordinary stream-ordered launches bit for bit, and the oracle run
+    as the same chain (its output rounded to bf16 between layers) within the bf16 tolerance.  Along a run
+    of overlapped launches every write is ordered behind the preceding kernel's completion, so the calls
+    may also share one workspace."""
+    w = synth.config(0, n=8192, L=6)
+    ids, run_id, run_lens = synth.token_ids(w)
+    plan = binding.chunk(ids.to(DEV), w.delims)
+    layers, refs = [], []
+    for l in range(w.L):
+        K, V = synth.layer_kv(w, l, run_id, run_lens)
+        refs.append(oracle_compress(ids, K, V, w.delims, w.tau, cap=w.n // 2))
+        layers.append(binding.compress(K.to(DEV), V.to(DEV), plan, w.tau, cap=w.n // 2))
+    n_ws = 1 if share_workspace else w.L
+    ws = [binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, w.n // 2, DEV) for _ in range(n_ws)]
+    st = torch.zeros(1, dtype=torch.int32, device=DEV)
+    q0 = (4.0 * synth.queries(w, 0, 0)).to(DEV)     # sharper softmax than N(0,1) queries give
+    # x[0] = q0, x[l + 1] = attention of layer l on x[l]
+    plain = torch.zeros((w.L + 1, w.B, w.Hq, w.d), dtype=q0.dtype, device=DEV)
+    plain[0] = q0
+    for l in range(w.L):
+        binding.decode_attn(plain[l], layers[l], out=plain[l + 1], workspace=ws[l % n_ws], status=st)
+    torch.cuda.synchronize()
+    for rep in range(4):
+        chain = torch.zeros_like(plain)
+        chain[0] = q0
+        torch.cuda.synchronize()
+        for l in range(w.L):
+            binding.decode_attn(chain[l], layers[l], out=chain[l + 1], workspace=ws[l % n_ws], status=st,
+                                flags=binding.SC_FLAG_OVERLAP_CHAIN if l > 0 else 0)
+        torch.cuda.synchronize()
+        assert torch.equal(plain, chain), f"repeat {rep}"
+    assert int(st.item()) == 0
+    x = synth.to_numpy_bits(q0.cpu())
+    for l in range(w.L):
+        r = refs[l]
+        want = oracle.attn(x, r["core_k"], r["core_v"], r["count"], r["core_len"])
+        assert_close_vectors(to_f64(plain[l + 1]), want, 1e-2, f"chain, layer {l}")
+        x = _bf16_bits(want)
+    for x in ws:
+        assert int(x.view(torch.int32)[:64].abs().max()) == 0, "arrival counters are left at zero"
+
+
+def test_overlapped_launches_two_apart_may_share_a_workspace():
+    """Two workspaces used alternately by a run of SC_FLAG_OVERLAP_PREV launches: launch l and launch l+2
+    write the same scratch, which is safe because a kernel's writes wait for its predecessor's completion
+    and that one waited for its own predecessor."""
+    w = synth.config(0, n=4096, L=6)
+    ids, run_id, run_lens = synth.token_ids(w)
+    plan = binding.chunk(ids.to(DEV), w.delims)
+    layers = []
+    for l in range(w.L):
+        K, V = synth.layer_kv(w, l, run_id, run_lens)
+        layers.append(binding.compress(K.to(DEV), V.to(DEV), plan, w.tau))
+    q = torch.stack([synth.queries(w, 1, l) for l in range(w.L)]).to(DEV)
+    ws = [binding.decode_workspace(w.B, w.Hq, w.Hkv, w.d, w.n, DEV) for _ in range(2)]
+    plain, fast = torch.empty_like(q), torch.empty_like(q)
+    for l in range(w.L):
+        binding.decode_attn(q[l], layers[l], out=plain[l], workspace=ws[l % 2])
+    torch.cuda.synchronize()
+    for rep in range(5):
+        fast.zero_()
+        for l in range(w.L):
+            binding.decode_attn(q[l], layers[l], out=fast[l], workspace=ws[l % 2],
+                                flags=binding.SC_FLAG_OVERLAP_PREV if l > 0 else 0)
+        torch.cuda.synchronize()
+        assert torch.equal(plain, fast), f"repeat {rep}"
