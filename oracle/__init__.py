@@ -159,6 +159,42 @@ def attn(q: np.ndarray, core_k: np.ndarray, core_v: np.ndarray, count: np.ndarra
     return out
 
 
+def attn_multi(q: np.ndarray, core_k: np.ndarray, core_v: np.ndarray, count: np.ndarray | None,
+               core_len: np.ndarray, scale: float | None = None, causal: bool = False) -> np.ndarray:
+    """Eq. 4 with a block of m queries per head.  q: [B, Hq, m, d].  Returns float64 [B, Hq, m, d].
+
+    causal: the last m rows of the cache are the queries' own tokens; query i sees rows
+    t < core_len - (m - 1 - i)."""
+    q = np.ascontiguousarray(q)
+    core_k = np.ascontiguousarray(core_k)
+    core_v = np.ascontiguousarray(core_v)
+    B, Hq, m, d = q.shape
+    _, Hkv, cap, _ = core_k.shape
+    assert Hq % Hkv == 0 and q.dtype == core_k.dtype == core_v.dtype
+    if count is not None:
+        count = np.ascontiguousarray(count, dtype=np.int32)
+    core_len = np.ascontiguousarray(core_len, dtype=np.int32)
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    out = np.zeros((B, Hq, m, d), dtype=np.float64)
+    _load().oracle_attn_multi(_p(q), ctypes.c_int32(_dtype_code(q)), ctypes.c_int32(B), ctypes.c_int32(Hq),
+                              ctypes.c_int32(Hkv), ctypes.c_int32(m), ctypes.c_int32(d), _p(core_k), _p(core_v),
+                              _p(count), ctypes.c_int32(cap), _p(core_len), ctypes.c_double(scale),
+                              ctypes.c_int32(1 if causal else 0), _p(out))
+    return out
+
+
+def compress_global(K, V, tau, cap=None):
+    """The paper's "no chunking" ablation arm (Table 4a): Algorithm 1 over each whole sequence as one
+    chunk (delimiters get no special treatment), then Eq. 3.  Same products as ``compress``."""
+    B, Hkv, n, _ = K.shape
+    seg_off = (np.arange(B + 1, dtype=np.int64) * n).astype(np.int32)
+    seq_seg_off = np.arange(B + 1, dtype=np.int32)
+    assign, margin = gsc(K, seg_off, seq_seg_off, tau)
+    core_k, core_v, count, core_len = merge(K, V, assign, cap)
+    return dict(seg_off=seg_off, seq_seg_off=seq_seg_off, assign=assign, margin=margin,
+                core_k=core_k, core_v=core_v, count=count, core_len=core_len)
+
+
 def compress(token_ids, delim_ids, K, V, tau, max_chunk_len=256, cap=None):
     """chunk -> gsc -> merge, the whole compress stage.  Returns a dict of every product."""
     seg_off, seq_seg_off = chunk(token_ids, delim_ids, max_chunk_len)
@@ -216,3 +252,62 @@ def append(state: dict, token_ids_new, k_new: np.ndarray, v_new: np.ndarray, del
                 tlen[b, h] += 1
                 if tlen[b, h] == max_chunk_len:
                     finish(b, h)
+
+
+def tau_grid(tau_lo: float, tau_hi: float, n_grid: int) -> np.ndarray:
+    """The thresholds a budget search may choose from: tau_i = tau_lo + i * ((tau_hi - tau_lo) / (n_grid - 1)),
+    every operation rounded to float32 (the threshold of Algorithm 1 is a float32 parameter)."""
+    lo, hi = np.float32(tau_lo), np.float32(tau_hi)
+    step = np.float32(hi - lo) / np.float32(n_grid - 1)
+    return np.array([np.float32(lo + np.float32(np.float32(i) * step)) for i in range(n_grid)], dtype=np.float32)
+
+
+def budget(token_ids, delim_ids, K, V, target_kept: float, tau_lo: float, tau_hi: float, n_grid: int,
+           max_chunk_len: int = 256, cap=None):
+    """Compress one layer to a KV budget (the kept fractions of Table 1; Table 4b: a lower threshold keeps less).
+
+    The paper states budgets and a threshold but not how one is turned into the other.  The reading
+    taken: the threshold is searched on a grid of ``n_grid`` values between ``tau_lo`` and ``tau_hi``
+    for the one whose number of cores (all sequences and heads of the layer together) comes nearest
+    to ``target_kept`` times the number of tokens, assuming that the count does not fall as the
+    threshold rises:
+      1. the two ends are evaluated; if even the lowest threshold keeps at least the target, it is
+         chosen; if even the highest keeps less than the target, that one is;
+      2. otherwise the interval is halved (middle index, rounded down) until its ends are adjacent,
+         keeping "fewer than the target" at the lower end and "at least the target" at the upper;
+      3. of the two ends the one whose count is nearer the target is chosen, the lower on a tie.
+    Returns the compress products at the chosen threshold plus ``tau``, ``index``, ``target_cores``
+    and ``visited`` (list of (index, cores) in evaluation order)."""
+    seg_off, seq_seg_off = chunk(token_ids, delim_ids, max_chunk_len)
+    B, Hkv, n, _ = K.shape
+    grid = tau_grid(tau_lo, tau_hi, n_grid)
+    target = int(np.floor(float(target_kept) * (B * Hkv * n) + 0.5))
+    pos = np.arange(n, dtype=np.int32)
+    visited, margins = [], []
+
+    def cores(i):
+        assign, margin = gsc(K, seg_off, seq_seg_off, float(grid[i]))
+        c = int((assign == pos).sum())
+        visited.append((i, c))
+        margins.append(margin)
+        return c
+
+    lo, hi = 0, n_grid - 1
+    k_lo, k_hi = cores(lo), cores(hi)
+    if k_lo >= target:
+        pick = lo
+    elif k_hi < target:
+        pick = hi
+    else:
+        while hi - lo > 1:
+            mid = (lo + hi) // 2
+            k = cores(mid)
+            if k >= target:
+                hi, k_hi = mid, k
+            else:
+                lo, k_lo = mid, k
+        pick = hi if (k_hi - target) < (target - k_lo) else lo
+    out = compress(token_ids, delim_ids, K, V, float(grid[pick]), max_chunk_len, cap)
+    out.update(tau=float(grid[pick]), index=pick, target_cores=target, visited=visited,
+               search_margin=min(margins))
+    return out

@@ -9,13 +9,18 @@
  *   oracle_chunk   Sec. 2.2, Eq. 1     delimiter-bounded chunking
  *   oracle_gsc     Sec. 2.3, Eq. 2 + Algorithm 1   greedy seed-based clustering
  *   oracle_merge   Sec. 2.4, Eq. 3     mean-pool each cluster into a semantic core
- *   oracle_attn    Sec. 2.4, Eq. 4     proportional attention over the cores
+ *   oracle_attn    Sec. 2.4, Eq. 4     proportional attention over the cores (one query per head)
+ *   oracle_attn_multi  Sec. 2.4, Eq. 4 as printed (Q in R^{m x d}): a block of queries per head
+ * The front end (__init__.py) adds, on top of these: the incremental path, the "no chunking" ablation
+ * arm of Table 4a (oracle_gsc with one chunk per sequence) and the budget search (Table 1 budgets).
  *
  * Pins (all in tests/, none re-types these formulas): hand-worked fixtures with
  * angles whose cosines are known in closed form, the lexicographically-first
  * maximal independent set found by brute force over all subsets, partition
  * invariants, tau >= 1 reducing Eq. 4 to textbook softmax attention (numpy),
- * and a cluster of identical (k, v) reproducing uncompressed attention.
+ * a cluster of identical (k, v) reproducing uncompressed attention, one query
+ * of a block being the decode step, and a closed-form kept fraction on pairs at
+ * known angles for the budget search.
  * The paper prints no worked numeric example, so the whole path against printed
  * values is "parity unpinned"; every function below has at least one of the pins
  * above.
@@ -320,6 +325,55 @@ void oracle_attn(const void *q, int32_t dtype, int32_t B, int32_t Hq, int32_t Hk
             for (int32_t t = 0; t < len; ++t) {
                 double w = x[t] / denom;
                 for (int32_t c = 0; c < d; ++c) o[c] += w * load_elem(core_v, dtype, (cbase + t) * d + c);
+            }
+            free(x);
+        }
+    }
+}
+
+/*
+ * Eq. 4 with a block of queries (Q in R^{m x d}, the form the paper prints): for every
+ * sequence b, query head hq (KV head = hq / (Hq/Hkv)) and query i of the m,
+ *   x_t = scale * <q_i, k_hat_t> + ln(count_t),   o_i = sum_t softmax(x)_t * v_hat_t.
+ * q and out are [B, Hq, m, d].  causal == 0: every query sees all core_len[b, kvh] rows.
+ * causal != 0: the last m rows of the cache are the queries' own tokens (appended with count 1),
+ * and query i sees rows t < core_len - (m - 1 - i): itself and everything before it.  A query
+ * that sees no row gives zeros.
+ */
+void oracle_attn_multi(const void *q, int32_t dtype, int32_t B, int32_t Hq, int32_t Hkv, int32_t m, int32_t d,
+                       const void *core_k, const void *core_v, const int32_t *count, int32_t cap,
+                       const int32_t *core_len, double scale, int32_t causal, double *out) {
+    const int32_t G = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int32_t b = 0; b < B; ++b) {
+        for (int32_t hq = 0; hq < Hq; ++hq) {
+            const int32_t h = hq / G;
+            const int32_t len = core_len[(int64_t)b * Hkv + h];
+            const int64_t cbase = ((int64_t)b * Hkv + h) * cap;
+            double *x = (double *)malloc(sizeof(double) * (size_t)(len > 0 ? len : 1));
+            for (int32_t i = 0; i < m; ++i) {
+                const int64_t qbase = (((int64_t)b * Hq + hq) * m + i) * d;
+                double *o = out + qbase;
+                for (int32_t c = 0; c < d; ++c) o[c] = 0.0;
+                const int32_t vis = causal ? len - (m - 1 - i) : len; /* rows this query sees */
+                if (vis <= 0) continue;
+                double mx = -INFINITY;
+                for (int32_t t = 0; t < vis; ++t) {
+                    double s = 0.0;
+                    for (int32_t c = 0; c < d; ++c)
+                        s += load_elem(q, dtype, qbase + c) * load_elem(core_k, dtype, (cbase + t) * d + c);
+                    x[t] = scale * s + (count ? log((double)count[cbase + t]) : 0.0);
+                    if (x[t] > mx) mx = x[t];
+                }
+                double denom = 0.0;
+                for (int32_t t = 0; t < vis; ++t) {
+                    x[t] = exp(x[t] - mx);
+                    denom += x[t];
+                }
+                for (int32_t t = 0; t < vis; ++t) {
+                    double w = x[t] / denom;
+                    for (int32_t c = 0; c < d; ++c) o[c] += w * load_elem(core_v, dtype, (cbase + t) * d + c);
+                }
             }
             free(x);
         }
