@@ -177,6 +177,52 @@ SC_API sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides
                       int32_t* status, void* stream);
 
 /*
+ * Compress one layer to a KV budget (the paper evaluates budgets of 20 / 35 / 50 % kept, Table 1, and
+ * shows that a lower threshold keeps fewer entries, Table 4b; how a budget is turned into a threshold
+ * it does not say).  This library's reading: the threshold of Algorithm 1 is searched on a grid
+ *     tau_i = tau_lo + i * ((tau_hi - tau_lo) / (n_grid - 1)),  i = 0 .. n_grid - 1   (float32 arithmetic)
+ * for the value whose number of cores, all sequences and KV heads of the layer together, comes
+ * nearest to target = floor(target_kept * B * Hkv * n + 0.5), assuming that the count does not fall
+ * as the threshold rises:
+ *   1. the lowest threshold is counted; if it already keeps at least the target it is chosen;
+ *      else the highest is counted; if even that keeps less than the target it is chosen;
+ *   2. otherwise the interval is halved (middle index, rounded down) until its ends are adjacent,
+ *      with "fewer than the target" at the lower end and "at least the target" at the upper;
+ *   3. of the two ends the one whose count is nearer the target is chosen, the lower on a tie.
+ * Everything runs on the device without a host round trip: at most 2 + ceil(log2(n_grid - 1))
+ * counting passes (Eq. 2 + Algorithm 1 on the keys alone, no Eq. 3, nothing written but counts),
+ * each followed by a one-block step that moves the search on, then one ordinary compress pass at
+ * the chosen threshold.  Counting passes enqueued after the choice is made return at once.
+ *
+ *   K .. n_tile_cap, core_k .. assign, status   as for sc_compress; params->tau is ignored;
+ *               params->flags may hold SC_FLAG_GENERIC only.  B, n > 0.
+ *   budget      HOST: target_kept in [0, 1], tau_lo < tau_hi, n_grid in [2, SC_BUDGET_MAX_GRID]
+ *   tau_out     out [1] float (device), may be NULL: the chosen threshold
+ *   search_out  out [2] int32 (device), may be NULL: the chosen grid index, and the number of
+ *               counting passes that did work
+ *   workspace   at least sc_compress_budget_workspace_bytes(B, Hkv, n) bytes, zeroed once after
+ *               allocation like sc_compress's (and left ready for the next call)
+ */
+typedef struct {
+    float target_kept;     /* wanted cores / tokens of the layer */
+    float tau_lo, tau_hi;  /* ends of the threshold grid */
+    int32_t n_grid;        /* number of grid points */
+} sc_budget;
+
+#define SC_BUDGET_MAX_GRID 65
+
+SC_API size_t sc_compress_budget_workspace_bytes(int32_t B, int32_t Hkv, int32_t n);
+
+SC_API sc_status sc_compress_budget(const void* K, const void* V, sc_strides kv_strides, sc_dtype dt,
+                             int32_t B, int32_t Hkv, int32_t n, int32_t d,
+                             const int32_t* seg_off, const int32_t* seq_seg_off, const int32_t* n_seg,
+                             const int32_t* tile_seg, const int32_t* seq_tile_cnt, int32_t n_tile_cap,
+                             const sc_gsc_params* params /*HOST*/, const sc_budget* budget /*HOST*/,
+                             void* core_k, void* core_v, int32_t* count, int32_t cap, int32_t* core_len,
+                             int32_t* assign, float* tau_out, int32_t* search_out,
+                             void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
  * One decode step of Proportional Attention (Sec. 2.4, Eq. 4) for one layer.  For every query
  * head hq of sequence b, with KV head h = hq / (Hq/Hkv):
  *     x_t = scale * <q, k_hat_t> + ln(count_t),  out = sum_t softmax(x)_t * v_hat_t

@@ -24,7 +24,8 @@ _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CA
 
 EXPORTS = ["sc_version", "sc_launch_counter", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
            "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn",
-           "sc_decode_attn_static", "sc_append"]
+           "sc_decode_attn_static", "sc_append", "sc_compress_budget_workspace_bytes", "sc_compress_budget"]
+SC_BUDGET_MAX_GRID = 65
 SC_STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -36,6 +37,11 @@ class ScError(RuntimeError):
 
 class _GscParams(ctypes.Structure):
     _fields_ = [("tau", ctypes.c_float), ("max_chunk_len", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class _Budget(ctypes.Structure):
+    _fields_ = [("target_kept", ctypes.c_float), ("tau_lo", ctypes.c_float), ("tau_hi", ctypes.c_float),
+                ("n_grid", ctypes.c_int32)]
 
 
 class _Strides(ctypes.Structure):
@@ -69,6 +75,12 @@ def lib() -> ctypes.CDLL:
         L.sc_compress.restype = _i32
         L.sc_compress.argtypes = [_vp, _vp, _Strides, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32,
                                   ctypes.POINTER(_GscParams), _vp, _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp, _vp]
+        L.sc_compress_budget_workspace_bytes.restype = _sz
+        L.sc_compress_budget_workspace_bytes.argtypes = [_i32, _i32, _i32]
+        L.sc_compress_budget.restype = _i32
+        L.sc_compress_budget.argtypes = [_vp, _vp, _Strides, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32,
+                                         ctypes.POINTER(_GscParams), ctypes.POINTER(_Budget), _vp, _vp, _vp, _i32, _vp,
+                                         _vp, _vp, _vp, _vp, _sz, _vp, _vp]
         L.sc_decode_attn.restype = _i32
         L.sc_decode_attn.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, ctypes.c_float,
                                      ctypes.c_uint32, _vp, _vp, _sz, _vp, _vp]
@@ -154,6 +166,28 @@ def sc_compress(K, V, plan: "ChunkPlan", tau, core_k, core_v, count, core_len, a
                              _ptr(assign), _ptr(workspace), workspace.numel() * workspace.element_size(),
                              _ptr(status), _stream(K))
     _check("sc_compress", code)
+
+
+def sc_compress_budget(K, V, plan: "ChunkPlan", target_kept, tau_lo, tau_hi, n_grid, core_k, core_v, count, core_len,
+                       tau_out, search_out, workspace, assign=None, status=None, flags=0):
+    """Raw sc_compress_budget for one layer: the threshold is searched on the device for the kept fraction."""
+    _need_cuda(K, V, core_k, core_v, count, core_len, assign, workspace, tau_out, search_out)
+    B, Hkv, n, d = K.shape
+    assert V.shape == K.shape and V.stride() == K.stride() and V.dtype == K.dtype and K.stride(3) == 1
+    assert core_k.is_contiguous() and core_v.is_contiguous() and count.is_contiguous()
+    assert tau_out is None or tau_out.dtype == torch.float32
+    assert search_out is None or (search_out.dtype == torch.int32 and search_out.numel() >= 2)
+    cap = core_k.shape[2]
+    prm = _GscParams(0.0, int(plan.max_chunk_len), int(flags))
+    bud = _Budget(float(target_kept), float(tau_lo), float(tau_hi), int(n_grid))
+    st = _Strides(K.stride(0), K.stride(1), K.stride(2))
+    code = lib().sc_compress_budget(_ptr(K), _ptr(V), st, _dt(K), B, Hkv, n, d, _ptr(plan.seg_off),
+                                    _ptr(plan.seq_seg_off), _ptr(plan.n_seg), _ptr(plan.tile_seg),
+                                    _ptr(plan.seq_tile_cnt), plan.n_tile_cap, ctypes.byref(prm), ctypes.byref(bud),
+                                    _ptr(core_k), _ptr(core_v), _ptr(count), cap, _ptr(core_len), _ptr(assign),
+                                    _ptr(tau_out), _ptr(search_out), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _ptr(status), _stream(K))
+    _check("sc_compress_budget", code)
 
 
 def sc_decode_attn(q, core_k, core_v, count, core_len, out, workspace, scale=0.0, status=None, flags=0):
@@ -250,6 +284,15 @@ def chunk(token_ids: torch.Tensor, delim_ids, max_chunk_len: int = SC_MAX_CHUNK_
     return plan
 
 
+def chunk_fixed(token_ids: torch.Tensor, size: int = 64) -> ChunkPlan:
+    """Fixed-size chunking, the paper's ablation arm (Table 4a compares semantic chunks with chunks of 64
+    tokens): every `size` tokens form a chunk and delimiters play no role -- sc_chunk with an empty
+    delimiter set and max_chunk_len = size.  The plan is used like any other."""
+    if not 1 <= size <= SC_MAX_CHUNK_LEN:
+        raise ValueError(f"chunk size must be in 1..{SC_MAX_CHUNK_LEN}")
+    return chunk(token_ids, (), size)
+
+
 def compress_workspace(B, Hkv, n, device) -> torch.Tensor:
     """Zero-initialised workspace for sc_compress (its status words and counters must start at zero)."""
     return torch.zeros(lib().sc_compress_workspace_bytes(B, Hkv, n), dtype=torch.uint8, device=device)
@@ -272,6 +315,26 @@ def compress(K, V, plan: ChunkPlan, tau: float, cap: int | None = None, want_ass
     sc_compress(K, V, plan, tau, out.core_k, out.core_v, out.count, out.core_len, out.assign, workspace,
                 plan.status, flags)
     return out
+
+
+def compress_to_budget(K, V, plan: ChunkPlan, target_kept: float, tau_lo: float = 0.5, tau_hi: float = 0.9,
+                       n_grid: int = 17, cap: int | None = None, want_assign: bool = False, flags: int = 0):
+    """Allocate the outputs and run sc_compress_budget.  Returns (CompressedLayer, tau [1] float32,
+    search [2] int32: grid index, counting passes) -- all on the device, nothing synchronises."""
+    B, Hkv, n, d = K.shape
+    dev = K.device
+    cap = n if cap is None else cap
+    out = CompressedLayer(torch.empty((B, Hkv, cap, d), dtype=K.dtype, device=dev),
+                          torch.empty((B, Hkv, cap, d), dtype=K.dtype, device=dev),
+                          torch.zeros((B, Hkv, cap), dtype=torch.int32, device=dev),
+                          torch.zeros((B, Hkv), dtype=torch.int32, device=dev),
+                          torch.empty((B, Hkv, n), dtype=torch.int32, device=dev) if want_assign else None)
+    ws = torch.zeros(lib().sc_compress_budget_workspace_bytes(B, Hkv, n), dtype=torch.uint8, device=dev)
+    tau = torch.zeros(1, dtype=torch.float32, device=dev)
+    search = torch.zeros(2, dtype=torch.int32, device=dev)
+    sc_compress_budget(K, V, plan, target_kept, tau_lo, tau_hi, n_grid, out.core_k, out.core_v, out.count, out.core_len,
+                       tau, search, ws, out.assign, plan.status, flags)
+    return out, tau, search
 
 
 def decode_workspace(B, Hq, Hkv, d, cap, device) -> torch.Tensor:

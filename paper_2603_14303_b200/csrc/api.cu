@@ -1,4 +1,6 @@
 // C-ABI entry points: argument validation and dispatch.  See include/semanticache.h.
+#include <math.h>
+
 #include "common.cuh"
 
 using namespace sc;
@@ -11,6 +13,9 @@ size_t compress_fused_ws_bytes(int32_t B, int32_t Hkv, int32_t n);
 bool decode_mma_supported(const DecodeArgs& a);
 cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st);
 size_t decode_mma_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap);
+size_t budget_state_bytes();
+cudaError_t launch_compress_budget(CompressArgs a, void* ws_compress, void* ws_generic, const float* grid, int n_grid,
+                                   long long target, float* tau_out, int32_t* search_out, cudaStream_t st);
 }  // namespace sc
 
 #include <atomic>
@@ -109,6 +114,7 @@ sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dt
     a.tau = params->tau; a.max_chunk_len = params->max_chunk_len; a.flags = params->flags;
     a.core_k = core_k; a.core_v = core_v; a.count = count; a.cap = cap; a.core_len = core_len;
     a.assign = assign; a.ws = workspace; a.status = status;
+    a.tau_dev = nullptr; a.skip = nullptr; a.count_only = 0;
     cudaError_t e;
     e = cudaErrorNotSupported;
     if (!(a.flags & SC_FLAG_GENERIC) && compress_fused_supported(a)) e = launch_compress_fused(a, st);
@@ -116,6 +122,59 @@ sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dt
         a.ws = (char*)workspace + fused_region_bytes(B, Hkv, n);   // never touches the fused kernel's words
         e = launch_compress_generic(a, st);
     }
+    return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
+size_t sc_compress_budget_workspace_bytes(int32_t B, int32_t Hkv, int32_t n) {
+    return budget_state_bytes() + sc_compress_workspace_bytes(B, Hkv, n);
+}
+
+sc_status sc_compress_budget(const void* K, const void* V, sc_strides kv_strides, sc_dtype dt, int32_t B, int32_t Hkv,
+                             int32_t n, int32_t d, const int32_t* seg_off, const int32_t* seq_seg_off,
+                             const int32_t* n_seg, const int32_t* tile_seg, const int32_t* seq_tile_cnt,
+                             int32_t n_tile_cap, const sc_gsc_params* params, const sc_budget* budget, void* core_k,
+                             void* core_v, int32_t* count, int32_t cap, int32_t* core_len, int32_t* assign,
+                             float* tau_out, int32_t* search_out, void* workspace, size_t workspace_bytes,
+                             int32_t* status, void* stream) {
+    if (B <= 0 || Hkv <= 0 || n <= 0 || cap < 0 || !params || !budget || !core_len) return SC_ERR_INVALID_ARG;
+    if (dt != SC_BF16 && dt != SC_F32) return SC_ERR_UNSUPPORTED;
+    if (d < 8 || d > 256 || (d % 8) != 0) return SC_ERR_UNSUPPORTED;
+    if (params->max_chunk_len < 1 || params->max_chunk_len > SC_MAX_CHUNK_LEN) return SC_ERR_INVALID_ARG;
+    if (params->flags & (SC_FLAG_TWO_PASS | SC_FLAG_OVERLAP_PREV | SC_FLAG_OVERLAP_CHAIN)) return SC_ERR_INVALID_ARG;
+    if (budget->n_grid < 2 || budget->n_grid > SC_BUDGET_MAX_GRID) return SC_ERR_INVALID_ARG;
+    if (!(budget->target_kept >= 0.f && budget->target_kept <= 1.f)) return SC_ERR_INVALID_ARG;
+    if (!(budget->tau_lo < budget->tau_hi)) return SC_ERR_INVALID_ARG;   // also refuses NaN
+    if (!K || !V || !seg_off || !seq_seg_off || !n_seg || !tile_seg || !seq_tile_cnt) return SC_ERR_INVALID_ARG;
+    if (!core_k || !core_v || !count || !workspace) return SC_ERR_INVALID_ARG;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(core_k) || !aligned16(core_v)) return SC_ERR_INVALID_ARG;
+    const size_t esz = dt == SC_BF16 ? 2 : 4;
+    if ((kv_strides.b * esz) % 16 || (kv_strides.h * esz) % 16 || (kv_strides.n * esz) % 16) return SC_ERR_INVALID_ARG;
+    if (kv_strides.n < d) return SC_ERR_INVALID_ARG;
+    if ((int64_t)B * n > 0x7fffffff - 1) return SC_ERR_INVALID_ARG;
+    if (n_tile_cap < 1 || n_tile_cap > tile_cap_for(n)) return SC_ERR_INVALID_ARG;
+    if (workspace_bytes < sc_compress_budget_workspace_bytes(B, Hkv, n)) return SC_ERR_INVALID_ARG;
+    // the grid of thresholds, in float32 arithmetic: tau_i = tau_lo + i * ((tau_hi - tau_lo) / (n_grid - 1))
+    float grid[SC_BUDGET_MAX_GRID];
+    {
+        volatile float step = (budget->tau_hi - budget->tau_lo) / (float)(budget->n_grid - 1);
+        for (int i = 0; i < budget->n_grid; ++i) {
+            volatile float prod = (float)i * step;   // rounded on its own: no fused multiply-add
+            grid[i] = budget->tau_lo + prod;
+        }
+    }
+    // the target as a number of cores of the whole layer, rounded half up
+    const long long target = (long long)floor((double)budget->target_kept * ((double)B * Hkv * n) + 0.5);
+    CompressArgs a;
+    a.K = K; a.V = V; a.st = kv_strides; a.dt = dt; a.B = B; a.Hkv = Hkv; a.n = n; a.d = d;
+    a.seg_off = seg_off; a.seq_seg_off = seq_seg_off; a.n_seg = n_seg;
+    a.tile_seg = tile_seg; a.seq_tile_cnt = seq_tile_cnt; a.n_tile_cap = n_tile_cap;
+    a.tau = grid[0]; a.max_chunk_len = params->max_chunk_len; a.flags = params->flags;
+    a.core_k = core_k; a.core_v = core_v; a.count = count; a.cap = cap; a.core_len = core_len;
+    a.assign = assign; a.ws = workspace; a.status = status;
+    a.tau_dev = nullptr; a.skip = nullptr; a.count_only = 0;
+    char* wsc = (char*)workspace + budget_state_bytes();
+    cudaError_t e = launch_compress_budget(a, wsc, wsc + fused_region_bytes(B, Hkv, n), grid, budget->n_grid, target,
+                                           tau_out, search_out, (cudaStream_t)stream);
     return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
 

@@ -91,6 +91,10 @@ struct CompressArgs {
     float tau; int32_t max_chunk_len; uint32_t flags;
     void* core_k; void* core_v; int32_t* count; int32_t cap; int32_t* core_len;
     int32_t* assign; void* ws; int32_t* status;
+    // budget search (all null / 0 for an ordinary call): the threshold is read from device memory; a pass
+    // may be told to do nothing by a device flag; a counting pass only adds each head's cluster count to
+    // core_len (which the caller zeroed) and writes nothing else
+    const float* tau_dev; const int32_t* skip; int32_t count_only;
 };
 cudaError_t launch_compress_generic(const CompressArgs& a, cudaStream_t st);
 size_t compress_generic_ws_bytes(int32_t B, int32_t Hkv, int32_t n);

@@ -444,6 +444,9 @@ struct Params {
     int32_t* ctl;            // [0] ticket counter, [1] blocks finished
     uint32_t* tile_state;    // [B*Hkv][n_tile_cap]
     int32_t* status;
+    const float* tau_dev;    // threshold in device memory (budget search), or null: use tau
+    const int32_t* skip;     // device flag: nonzero = this launch has nothing to do (budget search), or null
+    int count_into_len;      // kCountOnly: add the tile's cluster count to core_len instead of recording it per tile
     CUtensorMap map_k, map_v;   // [B, Hkv, n, 128] bf16, boxes of 32 rows x 64 columns, 128-byte swizzle
 };
 
@@ -625,6 +628,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     const bool service = warp == kWarps;   // the ninth warp
     int max_nt = 0;                        // most tiles any sequence has (service warp)
 
+    if (p.skip != nullptr && *p.skip != 0) return;   // uniform over the grid: nothing touched, nothing to clean
+    const float tau = p.tau_dev != nullptr ? *p.tau_dev : p.tau;
     // Let the next kernel of the stream start beside this one if it was launched with programmatic stream
     // serialization (a no-op otherwise); this kernel waits for its predecessor only at its very end.
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
@@ -711,15 +716,15 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
             }
             __syncthreads();
             if (have) {
-                if (p.tau < 0.f) threshold_block<true, true>(acc, warp, warp, lane, p.tau, norm, send, adj);
-                else threshold_block<false, true>(acc, warp, warp, lane, p.tau, norm, send, adj);
+                if (tau < 0.f) threshold_block<true, true>(acc, warp, warp, lane, tau, norm, send, adj);
+                else threshold_block<false, true>(acc, warp, warp, lane, tau, norm, send, adj);
             }
             for (int k = service ? 28 : warp; k < 28; k += kWarps) {
                 const int rb = kOffDiag[k] >> 4, cb = kOffDiag[k] & 15;
                 if (cb >= nrb || !((longblocks >> rb) & 1) || cb > reach[rb]) continue;
                 gram_block<false>(sbase, hs, rb, cb, lane, acc);
-                if (p.tau < 0.f) threshold_block<true, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
-                else threshold_block<false, false>(acc, rb, cb, lane, p.tau, norm, send, adj);
+                if (tau < 0.f) threshold_block<true, false>(acc, rb, cb, lane, tau, norm, send, adj);
+                else threshold_block<false, false>(acc, rb, cb, lane, tau, norm, send, adj);
             }
             __syncthreads();
         }
@@ -735,13 +740,13 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 const int s = multi[k];
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a <= 32) {
-                    if (p.tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
-                    else gsc_short_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
+                    if (tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
+                    else gsc_short_segment<false>(sbase, hs, a, e - a, tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
                     continue;
                 }
                 if (e - a <= kWarpSegMax) {   // the warp builds the segment's bit rows itself
-                    if (p.tau < 0.f) gram_mid_segment<true>(sbase, hs, a, e - a, p.tau, norm + warp * 64, adj, lane);
-                    else gram_mid_segment<false>(sbase, hs, a, e - a, p.tau, norm + warp * 64, adj, lane);
+                    if (tau < 0.f) gram_mid_segment<true>(sbase, hs, a, e - a, tau, norm + warp * 64, adj, lane);
+                    else gram_mid_segment<false>(sbase, hs, a, e - a, tau, norm + warp * 64, adj, lane);
                 }
                 const int w1 = (e - 1) >> 5;
                 uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
@@ -778,7 +783,10 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         for (int w = 0; w < kNW; ++w) P += __popc(seedmask[w]);
         uint32_t* stt = p.tile_state + (size_t)bh * p.n_tile_cap;
         if (kMode == kCountOnly) {
-            if (tid == 0) stt[t] = (uint32_t)P;
+            if (tid == 0) {
+                if (p.count_into_len) atomicAdd(&p.core_len[bh], P);
+                else stt[t] = (uint32_t)P;
+            }
         } else {
             if (!service) {
                 if (tid < R) {
@@ -987,6 +995,7 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
     p.B = a.B; p.Hkv = a.Hkv; p.n = a.n;
     p.seg_off = a.seg_off; p.tile_seg = a.tile_seg; p.seq_tile_cnt = a.seq_tile_cnt; p.n_tile_cap = a.n_tile_cap;
     p.tau = a.tau;
+    p.tau_dev = a.tau_dev; p.skip = a.skip; p.count_into_len = a.count_only ? 1 : 0;
     p.core_k = (__nv_bfloat16*)a.core_k; p.core_v = (__nv_bfloat16*)a.core_v; p.count = a.count; p.cap = a.cap;
     p.core_len = a.core_len; p.assign = a.assign;
     p.ctl = (int32_t*)a.ws;
@@ -997,7 +1006,10 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
     // no more blocks than there can be tiles
     const int64_t max_tiles = (int64_t)a.B * a.Hkv * a.n_tile_cap;
     const int grid = (int)(max_tiles < grid_of[dev] ? max_tiles : grid_of[dev]);
-    if (a.flags & SC_FLAG_TWO_PASS) {
+    if (a.count_only) {   // budget search: per-head cluster counts only
+        cf::compress_fused_kernel<cf::kCountOnly><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
+        note_launches(1);
+    } else if (a.flags & SC_FLAG_TWO_PASS) {
         cf::Params pc = p;
         pc.assign = nullptr;
         cf::compress_fused_kernel<cf::kCountOnly><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(pc);

@@ -15,8 +15,11 @@ template <typename T>
 __global__ void __launch_bounds__(kGenWarps * 32)
 gsc_generic(const T* __restrict__ K, sc_strides st, int B, int Hkv, int n, int d,
             const int32_t* __restrict__ seg_off, const int32_t* __restrict__ n_seg_p, int seg_stride,
-            float tau, int32_t* __restrict__ assign, int32_t* __restrict__ seg_p) {
+            float tau_host, const float* __restrict__ tau_dev, const int32_t* __restrict__ skip,
+            int32_t* __restrict__ assign, int32_t* __restrict__ seg_p) {
     __shared__ float norms[kGenWarps][SC_MAX_CHUNK_LEN];
+    if (skip != nullptr && *skip != 0) return;
+    const float tau = tau_dev != nullptr ? *tau_dev : tau_host;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int n_seg = min(*n_seg_p, seg_stride);
     const int64_t items = (int64_t)n_seg * Hkv;
@@ -80,8 +83,10 @@ gsc_generic(const T* __restrict__ K, sc_strides st, int B, int Hkv, int n, int d
 __global__ void __launch_bounds__(256)
 scan_generic(int Hkv, const int32_t* __restrict__ seq_seg_off, int seg_stride,
              const int32_t* __restrict__ seg_p, int32_t* __restrict__ seg_core_off,
-             int32_t* __restrict__ core_len, int cap, int32_t* status) {
+             int32_t* __restrict__ core_len, int cap, int32_t* status, const int32_t* __restrict__ skip,
+             int count_only) {
     __shared__ int wt[8];
+    if (skip != nullptr && *skip != 0) return;
     const int b = blockIdx.x / Hkv, h = blockIdx.x % Hkv;
     const int s0 = min(seq_seg_off[b], seg_stride), s1 = min(seq_seg_off[b + 1], seg_stride);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -100,7 +105,7 @@ scan_generic(int Hkv, const int32_t* __restrict__ seq_seg_off, int seg_stride,
     }
     if (threadIdx.x == 0) {
         core_len[b * Hkv + h] = carry;
-        if (carry > cap) set_status(status, SC_ERR_CAPACITY);
+        if (carry > cap && !count_only) set_status(status, SC_ERR_CAPACITY);
     }
 }
 
@@ -168,16 +173,20 @@ static cudaError_t run(const CompressArgs& a, cudaStream_t st) {
     int32_t* ws = (int32_t*)a.ws;
     int32_t* seg_p = ws;
     int32_t* seg_core_off = ws + per;
-    int32_t* assign = a.assign ? a.assign : ws + 2 * per;
+    int32_t* assign = (a.assign && !a.count_only) ? a.assign : ws + 2 * per;
     const int seg_stride = a.B * a.n;  // capacity of the segment axis
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int grid = sms * 8;
     gsc_generic<T><<<grid, kGenWarps * 32, 0, st>>>((const T*)a.K, a.st, a.B, a.Hkv, a.n, a.d, a.seg_off, a.n_seg,
-                                                    seg_stride, a.tau, assign, seg_p);
+                                                    seg_stride, a.tau, a.tau_dev, a.skip, assign, seg_p);
     scan_generic<<<a.B * a.Hkv, 256, 0, st>>>(a.Hkv, a.seq_seg_off, seg_stride, seg_p, seg_core_off, a.core_len,
-                                              a.cap, a.status);
+                                              a.cap, a.status, a.skip, a.count_only);
+    if (a.count_only) {   // budget search: per-head cluster counts only
+        note_launches(2);
+        return cudaGetLastError();
+    }
     merge_generic<T><<<grid, kGenWarps * 32, 0, st>>>((const T*)a.K, (const T*)a.V, a.st, a.B, a.Hkv, a.n, a.d,
                                                       a.seg_off, a.n_seg, seg_stride, assign, seg_core_off,
                                                       (T*)a.core_k, (T*)a.core_v, a.count, a.cap);

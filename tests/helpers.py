@@ -88,3 +88,31 @@ def layer_from_oracle(ref: dict, dtype, device) -> binding.CompressedLayer:
             return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).to(device)
         return torch.from_numpy(a).to(device)
     return binding.CompressedLayer(dev(ref["core_k"]), dev(ref["core_v"]), dev(ref["count"]), dev(ref["core_len"]))
+
+
+def assert_valid_run_of_algorithm1(assign: np.ndarray, Kb: np.ndarray, seg_off, tau: float, clear: float = 1e-5):
+    """Where similarities come within rounding of tau, fp32 (GPU) and fp64 (oracle) may decide differently
+    and both partitions are valid runs of Algorithm 1.  What is unique is checked exactly: replaying
+    Algorithm 1 along the given partition (assign[b, h, t] = seed position), every comparison whose
+    similarity is clear of tau by `clear` must have been decided as Eq. 2 says, the lowest unassigned token
+    of a chunk must be a seed, and every token must end up assigned.  seg_off is over the flattened [B*n] axis."""
+    B, Hkv, n = assign.shape
+    for s in range(len(seg_off) - 1):
+        a, e = int(seg_off[s]), int(seg_off[s + 1])
+        b, a, e = a // n, a - (a // n) * n, e - (a // n) * n
+        for h in range(Hkv):
+            taken = np.zeros(e - a, dtype=bool)
+            for i in range(a, e):
+                if taken[i - a]:
+                    continue
+                assert assign[b, h, i] == i, "the lowest unassigned token must be a seed"
+                taken[i - a] = True
+                for j in range(i + 1, e):
+                    if taken[j - a]:
+                        continue
+                    joined = assign[b, h, j] == i
+                    sim = oracle.sim(Kb[b, h], i, j)
+                    if abs(sim - tau) > clear:
+                        assert joined == (sim > tau), (b, h, i, j, sim)
+                    taken[j - a] |= joined
+            assert taken.all()
