@@ -223,6 +223,35 @@ SC_API sc_status sc_compress_budget(const void* K, const void* V, sc_strides kv_
                              void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
 
 /*
+ * Compress one layer WITHOUT chunking: the "none / global" arm of the paper's chunking ablation
+ * (Table 4a).  Algorithm 1 (Sec. 2.3) runs over each whole sequence as a single chunk -- delimiters
+ * get no special treatment, a token may join a seed anywhere before it -- and every cluster is then
+ * mean-pooled by Eq. 3 (Sec. 2.4) exactly as in sc_compress: cores in position order of their seeds,
+ * count = |S_t|, fp32 sums in token order, one rounding.
+ *
+ * Algorithm 1 over n tokens is evaluated through its closed form (the seeds are the first maximal
+ * independent set, in index order, of the graph Sim > tau; every other token joins its lowest adjacent
+ * seed): all pairwise similarities of a head are thresholded into a bit matrix (tensor cores for
+ * SC_BF16 with d = 128, CUDA cores otherwise), then seeds and members are decided in parallel rounds.
+ * The result is the one a sequential run gives.  Cost grows with n^2: about n^2 / 16 bytes of
+ * workspace per (sequence, head) and n^2 * d multiply-adds.
+ *
+ *   K, V, kv_strides, dt, core_k .. assign, status   as for sc_compress (assign: position of each token's seed)
+ *   n          at most SC_GLOBAL_MAX_TOKENS;  B * Hkv at most 65535
+ *   flags      SC_FLAG_GENERIC forces the CUDA-core similarity kernel; else 0
+ *   workspace  at least sc_compress_global_workspace_bytes(B, Hkv, n) bytes, 16-byte aligned; no
+ *              initialisation needed, nothing persists between calls
+ */
+#define SC_GLOBAL_MAX_TOKENS 131072
+
+SC_API size_t sc_compress_global_workspace_bytes(int32_t B, int32_t Hkv, int32_t n);
+
+SC_API sc_status sc_compress_global(const void* K, const void* V, sc_strides kv_strides, sc_dtype dt,
+                             int32_t B, int32_t Hkv, int32_t n, int32_t d, float tau, uint32_t flags,
+                             void* core_k, void* core_v, int32_t* count, int32_t cap, int32_t* core_len,
+                             int32_t* assign, void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
  * One decode step of Proportional Attention (Sec. 2.4, Eq. 4) for one layer.  For every query
  * head hq of sequence b, with KV head h = hq / (Hq/Hkv):
  *     x_t = scale * <q, k_hat_t> + ln(count_t),  out = sum_t softmax(x)_t * v_hat_t

@@ -24,7 +24,8 @@ _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CA
 
 EXPORTS = ["sc_version", "sc_launch_counter", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
            "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn",
-           "sc_decode_attn_static", "sc_append", "sc_compress_budget_workspace_bytes", "sc_compress_budget"]
+           "sc_decode_attn_static", "sc_append", "sc_compress_budget_workspace_bytes", "sc_compress_budget",
+           "sc_compress_global_workspace_bytes", "sc_compress_global"]
 SC_BUDGET_MAX_GRID = 65
 SC_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -81,6 +82,11 @@ def lib() -> ctypes.CDLL:
         L.sc_compress_budget.argtypes = [_vp, _vp, _Strides, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32,
                                          ctypes.POINTER(_GscParams), ctypes.POINTER(_Budget), _vp, _vp, _vp, _i32, _vp,
                                          _vp, _vp, _vp, _vp, _sz, _vp, _vp]
+        L.sc_compress_global_workspace_bytes.restype = _sz
+        L.sc_compress_global_workspace_bytes.argtypes = [_i32, _i32, _i32]
+        L.sc_compress_global.restype = _i32
+        L.sc_compress_global.argtypes = [_vp, _vp, _Strides, _i32, _i32, _i32, _i32, _i32, ctypes.c_float, ctypes.c_uint32,
+                                         _vp, _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp, _vp]
         L.sc_decode_attn.restype = _i32
         L.sc_decode_attn.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, ctypes.c_float,
                                      ctypes.c_uint32, _vp, _vp, _sz, _vp, _vp]
@@ -188,6 +194,20 @@ def sc_compress_budget(K, V, plan: "ChunkPlan", target_kept, tau_lo, tau_hi, n_g
                                     _ptr(tau_out), _ptr(search_out), _ptr(workspace),
                                     workspace.numel() * workspace.element_size(), _ptr(status), _stream(K))
     _check("sc_compress_budget", code)
+
+
+def sc_compress_global(K, V, tau, core_k, core_v, count, core_len, workspace, assign=None, status=None, flags=0):
+    """Raw sc_compress_global for one layer: Algorithm 1 over whole sequences (no chunking), then Eq. 3."""
+    _need_cuda(K, V, core_k, core_v, count, core_len, assign, workspace)
+    B, Hkv, n, d = K.shape
+    assert V.shape == K.shape and V.stride() == K.stride() and V.dtype == K.dtype and K.stride(3) == 1
+    assert core_k.is_contiguous() and core_v.is_contiguous() and count.is_contiguous()
+    st = _Strides(K.stride(0), K.stride(1), K.stride(2))
+    code = lib().sc_compress_global(_ptr(K), _ptr(V), st, _dt(K), B, Hkv, n, d, float(tau), int(flags), _ptr(core_k),
+                                    _ptr(core_v), _ptr(count), core_k.shape[2], _ptr(core_len), _ptr(assign),
+                                    _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status),
+                                    _stream(K))
+    _check("sc_compress_global", code)
 
 
 def sc_decode_attn(q, core_k, core_v, count, core_len, out, workspace, scale=0.0, status=None, flags=0):
@@ -335,6 +355,23 @@ def compress_to_budget(K, V, plan: ChunkPlan, target_kept: float, tau_lo: float 
     sc_compress_budget(K, V, plan, target_kept, tau_lo, tau_hi, n_grid, out.core_k, out.core_v, out.count, out.core_len,
                        tau, search, ws, out.assign, plan.status, flags)
     return out, tau, search
+
+
+def compress_global(K, V, tau: float, cap: int | None = None, want_assign: bool = False, flags: int = 0,
+                    status: torch.Tensor | None = None, workspace: torch.Tensor | None = None):
+    """Allocate the outputs (and the workspace) and run sc_compress_global for one layer."""
+    B, Hkv, n, d = K.shape
+    dev = K.device
+    cap = n if cap is None else cap
+    out = CompressedLayer(torch.empty((B, Hkv, cap, d), dtype=K.dtype, device=dev),
+                          torch.empty((B, Hkv, cap, d), dtype=K.dtype, device=dev),
+                          torch.zeros((B, Hkv, cap), dtype=torch.int32, device=dev),
+                          torch.zeros((B, Hkv), dtype=torch.int32, device=dev),
+                          torch.empty((B, Hkv, n), dtype=torch.int32, device=dev) if want_assign else None)
+    if workspace is None:
+        workspace = torch.empty(lib().sc_compress_global_workspace_bytes(B, Hkv, n), dtype=torch.uint8, device=dev)
+    sc_compress_global(K, V, tau, out.core_k, out.core_v, out.count, out.core_len, workspace, out.assign, status, flags)
+    return out
 
 
 def decode_workspace(B, Hq, Hkv, d, cap, device) -> torch.Tensor:

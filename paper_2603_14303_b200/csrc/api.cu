@@ -178,6 +178,36 @@ sc_status sc_compress_budget(const void* K, const void* V, sc_strides kv_strides
     return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
 
+size_t sc_compress_global_workspace_bytes(int32_t B, int32_t Hkv, int32_t n) {
+    if (B <= 0 || Hkv <= 0 || n <= 0) return 256;
+    return compress_global_ws_bytes(B, Hkv, n);
+}
+
+sc_status sc_compress_global(const void* K, const void* V, sc_strides kv_strides, sc_dtype dt, int32_t B, int32_t Hkv,
+                             int32_t n, int32_t d, float tau, uint32_t flags, void* core_k, void* core_v, int32_t* count,
+                             int32_t cap, int32_t* core_len, int32_t* assign, void* workspace, size_t workspace_bytes,
+                             int32_t* status, void* stream) {
+    if (B < 0 || Hkv <= 0 || n < 0 || cap < 0 || !core_len) return SC_ERR_INVALID_ARG;
+    if (dt != SC_BF16 && dt != SC_F32) return SC_ERR_UNSUPPORTED;
+    if (d < 8 || d > 256 || (d % 8) != 0) return SC_ERR_UNSUPPORTED;
+    if (!(tau == tau) || (flags & ~SC_FLAG_GENERIC)) return SC_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (B == 0) return SC_OK;
+    if (n == 0) return cudaMemsetAsync(core_len, 0, sizeof(int32_t) * (size_t)B * Hkv, st) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+    if (n > SC_GLOBAL_MAX_TOKENS || (int64_t)B * Hkv > 65535) return SC_ERR_UNSUPPORTED;
+    if (!K || !V || !core_k || !core_v || !count || !workspace) return SC_ERR_INVALID_ARG;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(core_k) || !aligned16(core_v) || !aligned16(workspace)) return SC_ERR_INVALID_ARG;
+    const size_t esz = dt == SC_BF16 ? 2 : 4;
+    if ((kv_strides.b * esz) % 16 || (kv_strides.h * esz) % 16 || (kv_strides.n * esz) % 16) return SC_ERR_INVALID_ARG;
+    if (kv_strides.n < d) return SC_ERR_INVALID_ARG;
+    if (workspace_bytes < sc_compress_global_workspace_bytes(B, Hkv, n)) return SC_ERR_INVALID_ARG;
+    GlobalArgs a;
+    a.K = K; a.V = V; a.st = kv_strides; a.dt = dt; a.B = B; a.Hkv = Hkv; a.n = n; a.d = d; a.tau = tau; a.flags = flags;
+    a.core_k = core_k; a.core_v = core_v; a.count = count; a.cap = cap; a.core_len = core_len; a.assign = assign;
+    a.ws = workspace; a.status = status;
+    return launch_compress_global(a, st) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
 size_t sc_decode_workspace_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap) {
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || cap < 0) return 256;
     size_t a = decode_generic_ws_bytes(B, Hq, Hkv, d, cap), b = decode_mma_ws_bytes(B, Hq, Hkv, d, cap);

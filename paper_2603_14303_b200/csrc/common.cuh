@@ -99,6 +99,15 @@ struct CompressArgs {
 cudaError_t launch_compress_generic(const CompressArgs& a, cudaStream_t st);
 size_t compress_generic_ws_bytes(int32_t B, int32_t Hkv, int32_t n);
 
+struct GlobalArgs {   // clustering of whole sequences (no chunking)
+    const void* K; const void* V; sc_strides st; sc_dtype dt; int32_t B, Hkv, n, d;
+    float tau; uint32_t flags;
+    void* core_k; void* core_v; int32_t* count; int32_t cap; int32_t* core_len; int32_t* assign;
+    void* ws; int32_t* status;
+};
+cudaError_t launch_compress_global(const GlobalArgs& a, cudaStream_t st);
+size_t compress_global_ws_bytes(int32_t B, int32_t Hkv, int32_t n);
+
 struct DecodeArgs {
     const void* q; sc_dtype dt; int32_t B, Hq, Hkv, d;
     const void* core_k; const void* core_v; const int32_t* count; int32_t cap;
