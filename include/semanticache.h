@@ -80,6 +80,9 @@ typedef enum { SC_BF16 = 0, SC_F32 = 1 } sc_dtype;
                                   count and core_len are still read early and fall under the promise
                                   above.  Ignored (ordinary launch) on the generic path. */
 
+#define SC_FLAG_CAUSAL_TAIL 16u /* sc_prefill_attn only: the last m rows of every head are the m queries' own
+                                  tokens; query i attends to rows t < core_len - (m - 1 - i) */
+
 typedef struct {
     float tau;             /* similarity threshold of Algorithm 1; merge iff Sim > tau (strict) */
     int32_t max_chunk_len; /* must equal the value given to sc_chunk; 1..SC_MAX_CHUNK_LEN */
@@ -277,6 +280,29 @@ SC_API sc_status sc_decode_attn(const void* q, sc_dtype dt, int32_t B, int32_t H
                          const void* core_k, const void* core_v, const int32_t* count, int32_t cap,
                          const int32_t* core_len, float scale, uint32_t flags, void* out,
                          void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
+ * Proportional Attention for a block of m queries per head (Sec. 2.4, Eq. 4 as the paper prints it, with
+ * Q in R^{m x d}): chunked prefill, or verification of m speculated tokens, over a compressed cache.  For
+ * every sequence b, query head hq (KV head h = hq / (Hq/Hkv)) and query i:
+ *     x_t = scale * <q_i, k_hat_t> + ln(count_t),  out_i = sum_t softmax(x)_t * v_hat_t
+ * over the rows t the query attends to: all t < core_len[b, h], or, with SC_FLAG_CAUSAL_TAIL, only
+ * t < core_len[b, h] - (m - 1 - i) (the cache then already holds the m queries' own tokens as its last m
+ * rows, stored with count 1, and each query sees itself and what precedes it).  A query that attends to
+ * no row gets zeros.  With m = 1 this is sc_decode_attn.
+ * The G*m query rows that share a KV head are one dense contraction against that head's cores: SC_BF16
+ * with d = 128 runs on the tensor cores (scores and accumulators in tensor memory), other types and
+ * head sizes on a CUDA-core kernel.  No workspace.
+ *
+ *   q, out     [B, Hq, m, d] contiguous, dtype dt
+ *   core_k/v, count (or NULL for all ones), cap, core_len, scale   as for sc_decode_attn
+ *   flags      SC_FLAG_CAUSAL_TAIL, SC_FLAG_GENERIC (forces the CUDA-core kernel), or 0
+ *   status     SC_ERR_TIMEOUT if a bounded wait inside the kernel gave up
+ */
+SC_API sc_status sc_prefill_attn(const void* q, sc_dtype dt, int32_t B, int32_t Hq, int32_t Hkv, int32_t m, int32_t d,
+                          const void* core_k, const void* core_v, const int32_t* count, int32_t cap,
+                          const int32_t* core_len, float scale, uint32_t flags, void* out,
+                          int32_t* status, void* stream);
 
 /*
  * One generated token joins a layer's compressed cache (incremental form of Sec. 2.2-2.4).

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libsemanticache.so")
 
 SC_OK, SC_ERR_INVALID_ARG, SC_ERR_UNSUPPORTED, SC_ERR_CAPACITY, SC_ERR_CUDA, SC_ERR_TIMEOUT = range(6)
 SC_BF16, SC_F32 = 0, 1
-SC_FLAG_GENERIC, SC_FLAG_TWO_PASS, SC_FLAG_OVERLAP_PREV, SC_FLAG_OVERLAP_CHAIN = 1, 2, 4, 8
+SC_FLAG_GENERIC, SC_FLAG_TWO_PASS, SC_FLAG_OVERLAP_PREV, SC_FLAG_OVERLAP_CHAIN, SC_FLAG_CAUSAL_TAIL = 1, 2, 4, 8, 16
 SC_MAX_CHUNK_LEN, SC_MAX_DELIMS, SC_TILE_ROWS = 256, 64, 128
 _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CAPACITY", "SC_ERR_CUDA",
                  "SC_ERR_TIMEOUT"]
@@ -25,7 +25,7 @@ _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CA
 EXPORTS = ["sc_version", "sc_launch_counter", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
            "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn",
            "sc_decode_attn_static", "sc_append", "sc_compress_budget_workspace_bytes", "sc_compress_budget",
-           "sc_compress_global_workspace_bytes", "sc_compress_global"]
+           "sc_compress_global_workspace_bytes", "sc_compress_global", "sc_prefill_attn"]
 SC_BUDGET_MAX_GRID = 65
 SC_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -90,6 +90,9 @@ def lib() -> ctypes.CDLL:
         L.sc_decode_attn.restype = _i32
         L.sc_decode_attn.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, ctypes.c_float,
                                      ctypes.c_uint32, _vp, _vp, _sz, _vp, _vp]
+        L.sc_prefill_attn.restype = _i32
+        L.sc_prefill_attn.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, ctypes.c_float,
+                                      ctypes.c_uint32, _vp, _vp, _vp]
         L.sc_decode_attn_static.restype = _i32
         L.sc_decode_attn_static.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp,
                                             ctypes.c_float, ctypes.c_uint32, _vp, _vp, _vp]
@@ -220,6 +223,18 @@ def sc_decode_attn(q, core_k, core_v, count, core_len, out, workspace, scale=0.0
                                 _ptr(core_len), float(scale), int(flags), _ptr(out), _ptr(workspace),
                                 workspace.numel() * workspace.element_size(), _ptr(status), _stream(q))
     _check("sc_decode_attn", code)
+
+
+def sc_prefill_attn(q, core_k, core_v, count, core_len, out, scale=0.0, status=None, flags=0):
+    """Raw sc_prefill_attn: Proportional Attention for a block of m queries per head, q/out [B, Hq, m, d]."""
+    _need_cuda(q, core_k, core_v, count, core_len, out)
+    B, Hq, m, d = q.shape
+    _, Hkv, cap, _ = core_k.shape
+    assert q.is_contiguous() and out.is_contiguous() and core_k.is_contiguous() and core_v.is_contiguous()
+    assert out.shape == q.shape and out.dtype == q.dtype
+    code = lib().sc_prefill_attn(_ptr(q), _dt(q), B, Hq, Hkv, m, d, _ptr(core_k), _ptr(core_v), _ptr(count), cap,
+                                 _ptr(core_len), float(scale), int(flags), _ptr(out), _ptr(status), _stream(q))
+    _check("sc_prefill_attn", code)
 
 
 def sc_decode_attn_static(q, core_k, core_v, count, core_len, out, scale=0.0, status=None, flags=0):
@@ -371,6 +386,16 @@ def compress_global(K, V, tau: float, cap: int | None = None, want_assign: bool 
     if workspace is None:
         workspace = torch.empty(lib().sc_compress_global_workspace_bytes(B, Hkv, n), dtype=torch.uint8, device=dev)
     sc_compress_global(K, V, tau, out.core_k, out.core_v, out.count, out.core_len, workspace, out.assign, status, flags)
+    return out
+
+
+def prefill_attn(q, layer: CompressedLayer, out=None, scale: float = 0.0, status=None, causal: bool = False,
+                 flags: int = 0, use_count: bool = True):
+    """Proportional Attention of a block of queries q [B, Hq, m, d] over one layer's cores."""
+    if out is None:
+        out = torch.empty_like(q)
+    sc_prefill_attn(q, layer.core_k, layer.core_v, layer.count if use_count else None, layer.core_len, out, scale,
+                    status, flags | (SC_FLAG_CAUSAL_TAIL if causal else 0))
     return out
 
 

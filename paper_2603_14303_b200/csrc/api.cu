@@ -237,6 +237,23 @@ sc_status sc_decode_attn(const void* q, sc_dtype dt, int32_t B, int32_t Hq, int3
     return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
 
+sc_status sc_prefill_attn(const void* q, sc_dtype dt, int32_t B, int32_t Hq, int32_t Hkv, int32_t m, int32_t d,
+                          const void* core_k, const void* core_v, const int32_t* count, int32_t cap,
+                          const int32_t* core_len, float scale, uint32_t flags, void* out, int32_t* status, void* stream) {
+    if (B < 0 || Hq <= 0 || Hkv <= 0 || m < 0 || cap < 0 || (Hq % Hkv) != 0) return SC_ERR_INVALID_ARG;
+    if (dt != SC_BF16 && dt != SC_F32) return SC_ERR_UNSUPPORTED;
+    if (d < 8 || d > 256 || (d % 8) != 0) return SC_ERR_UNSUPPORTED;
+    if (!(scale == scale) || scale < 0.f || (flags & ~(SC_FLAG_GENERIC | SC_FLAG_CAUSAL_TAIL))) return SC_ERR_INVALID_ARG;
+    if (B == 0 || m == 0) return SC_OK;
+    if (!q || !out || !core_len) return SC_ERR_INVALID_ARG;
+    if (cap > 0 && (!core_k || !core_v)) return SC_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(out) || !aligned16(core_k) || !aligned16(core_v)) return SC_ERR_INVALID_ARG;
+    PrefillArgs a;
+    a.q = q; a.dt = dt; a.B = B; a.Hq = Hq; a.Hkv = Hkv; a.m = m; a.d = d; a.core_k = core_k; a.core_v = core_v;
+    a.count = count; a.cap = cap; a.core_len = core_len; a.scale = scale; a.flags = flags; a.out = out; a.status = status;
+    return launch_prefill(a, (cudaStream_t)stream) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
 sc_status sc_append(const void* k_new, const void* v_new, sc_dtype dt, int32_t B, int32_t Hkv, int32_t d,
                     const int32_t* token_ids, const int32_t* delim_ids, int32_t n_delim, int32_t max_chunk_len,
                     float tau, void* core_k, void* core_v, int32_t* count, int32_t cap, int32_t* core_len,

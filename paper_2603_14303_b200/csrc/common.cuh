@@ -116,6 +116,13 @@ struct DecodeArgs {
 cudaError_t launch_decode_generic(const DecodeArgs& a, cudaStream_t st);
 size_t decode_generic_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap);
 
+struct PrefillArgs {   // Eq. 4 with a block of m queries per head
+    const void* q; sc_dtype dt; int32_t B, Hq, Hkv, m, d;
+    const void* core_k; const void* core_v; const int32_t* count; int32_t cap;
+    const int32_t* core_len; float scale; uint32_t flags; void* out; int32_t* status;
+};
+cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st);
+
 struct AppendArgs {
     const void* k_new; const void* v_new; sc_dtype dt; int32_t B, Hkv, d;
     const int32_t* token_ids; int32_t delim[SC_MAX_DELIMS]; int32_t n_delim; int32_t max_chunk_len; float tau;

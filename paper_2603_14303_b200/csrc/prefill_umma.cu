@@ -1,0 +1,403 @@
+// Multi-query Proportional Attention (Sec. 2.4, Eq. 4 as printed, with a block of m queries per head):
+//     O = softmax(Q K_c^T * scale + ln s) V_c      Q: [m, d] per query head, K_c/V_c: the head's cores
+// for chunked prefill or speculative decoding over a compressed cache.  Unlike the one-query decode
+// step this is a dense contraction: the G query heads that share a KV head times the m queries give
+// G*m rows against the same cores, so it runs on the tcgen05 tensor cores (bf16, d = 128):
+//   one CTA = 128 query rows of one (sequence, KV head), walking the head's cores 128 at a time;
+//   warp 0     TMA: the query tile once, then K and V tiles into a two-stage ring (128-byte swizzle);
+//   warp 1     issues the MMAs: S = Q K^T into one of two score buffers in tensor memory (so the next
+//              tile's scores are computed while this tile's are being exponentiated), then O += P V,
+//              V read as an MN-major operand straight from its [keys x dims] tile;
+//   warps 2-5  softmax, one thread per query row (= tensor-memory lane, so no cross-thread reduction):
+//              x = S * scale*log2(e) + log2(count), masks (head length, optional causal tail), running
+//              maximum raised lazily (the accumulator row is rescaled in tensor memory only then),
+//              P = 2^(x - m) written to shared memory as a bf16 pair (leading part + remainder) in
+//              the swizzled K-major layout the second MMA reads; finally O / l -> bf16 -> global.
+// Every wait is bounded; a wait that gives up is reported through the status word.
+// A CUDA-core kernel (one warp per query) serves other dtypes and head sizes.
+#include "common.cuh"
+#include "umma.cuh"
+
+namespace sc {
+
+namespace pf {
+
+using namespace umma;
+
+constexpr int kT = 128;                       // query rows per CTA, keys per tile
+constexpr int kHalf = kT * 128;               // 16384 bytes: one 64-column half of a [128 x 128] bf16 tile
+constexpr int kTile = 2 * kHalf;              // 32768
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;                // S0 | S1 | O (128 columns each), rounded up to a power of two
+constexpr int kColS = 0, kColO = 256;
+constexpr int kSmQ = 0, kSmK = kTile, kSmV = 3 * kTile, kSmP = 5 * kTile, kSmLc = 7 * kTile, kSmBar = kSmLc + 2 * kT * 4;
+constexpr int kSmemBytes = kSmBar + 256 + 1024;
+constexpr float kMaxSlack = 8.f;              // log2 units a score may exceed the running maximum before it is raised
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+
+struct Params {
+    CUtensorMap map_q, map_k, map_v;          // rows x 128 bf16, boxes of 128 rows x 64 columns
+    const int32_t* count; const int32_t* core_len;
+    __nv_bfloat16* out;
+    int Hq, Hkv, m, cap, causal;
+    float scale_log2;
+    int32_t* status;
+};
+
+__device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float lg2(float x) { float y; asm("lg2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+__global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_constant__ Params p) {
+    extern __shared__ unsigned char smem_raw[];
+    const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int G = p.Hq / p.Hkv, bh = b * p.Hkv + h;
+    const int rows_total = G * p.m;                           // query rows of this (sequence, KV head)
+    const int len = max(min(p.core_len[bh], p.cap), 0);
+    const int nt = (len + kT - 1) / kT;                       // key tiles
+    const long long q_row0 = ((long long)b * p.Hq + (long long)h * G) * p.m + (long long)qt * kT;
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* smem = smem_raw + (sbase - smem_u32(smem_raw));
+    float* lc_s = reinterpret_cast<float*>(smem + kSmLc);     // [2][128] log2(count) of the tile's keys
+    const uint32_t bar0 = sbase + kSmBar;
+    const uint32_t q_full = bar0, kv_full0 = bar0 + 8, kv_empty0 = bar0 + 24, s_full0 = bar0 + 40, s_empty0 = bar0 + 56,
+                   p_full = bar0 + 72, p_empty = bar0 + 80;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kSmBar + 96);
+    volatile int* sh_fail = reinterpret_cast<volatile int*>(smem + kSmBar + 100);
+    volatile int* sh_fail_sm = reinterpret_cast<volatile int*>(smem + kSmBar + 104);   // set by the softmax warps only
+    volatile int* sh_issued = reinterpret_cast<volatile int*>(smem + kSmBar + 108);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        mbar_init(q_full, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(kv_full0 + 8 * s, 1);
+            mbar_init(kv_empty0 + 8 * s, 1);
+            mbar_init(s_full0 + 8 * s, 1);
+            mbar_init(s_empty0 + 8 * s, 4);
+        }
+        mbar_init(p_full, 4);
+        mbar_init(p_empty, 1);
+        mbar_fence_init();
+        *sh_fail = 0; *sh_fail_sm = 0; *sh_issued = 0;
+    }
+    if (warp == 1) tmem_alloc(sbase + kSmBar + 96, kTmemCols);
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0 && nt > 0) {   // ---- TMA producer ----
+            mbar_expect_tx(q_full, kTile);
+            tma_load_4d(sbase + kSmQ, &p.map_q, 0, (int)q_row0, 0, 0, q_full);
+            tma_load_4d(sbase + kSmQ + kHalf, &p.map_q, 64, (int)q_row0, 0, 0, q_full);
+            const int row_base = bh * p.cap;
+            for (int t = 0; t < nt; ++t) {
+                const int s = t & 1;
+                if (t >= 2 && !mbar_wait(kv_empty0 + 8 * s, ((t >> 1) - 1) & 1)) { *sh_fail = 1; break; }
+                mbar_expect_tx(kv_full0 + 8 * s, 2 * kTile);
+                const uint32_t dk = sbase + kSmK + s * kTile, dv = sbase + kSmV + s * kTile;
+                tma_load_4d(dk, &p.map_k, 0, row_base + t * kT, 0, 0, kv_full0 + 8 * s);
+                tma_load_4d(dk + kHalf, &p.map_k, 64, row_base + t * kT, 0, 0, kv_full0 + 8 * s);
+                tma_load_4d(dv, &p.map_v, 0, row_base + t * kT, 0, 0, kv_full0 + 8 * s);
+                tma_load_4d(dv + kHalf, &p.map_v, 64, row_base + t * kT, 0, 0, kv_full0 + 8 * s);
+                *sh_issued = t + 1;
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && nt > 0) {   // ---- MMA issuer ----
+            constexpr uint32_t idesc_qk = instr_desc_bf16(kT, kT, false, false);   // Q and K both K-major
+            constexpr uint32_t idesc_pv = instr_desc_bf16(kT, kT, false, true);    // P K-major, V MN-major
+            const uint32_t aq = sbase + kSmQ;
+            auto issue_qk = [&](int t) {
+                const int s = t & 1;
+                const uint32_t bk = sbase + kSmK + s * kTile;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
+                    mma_bf16_ss(tmem + kColS + s * kT, smem_desc_sw128(aq + off, 16, 1024), smem_desc_sw128(bk + off, 16, 1024),
+                                idesc_qk, ks > 0);
+                }
+                mma_commit(s_full0 + 8 * s);
+            };
+            bool ok = mbar_wait(q_full, 0) && mbar_wait(kv_full0, 0);
+            if (ok) { fence_after_sync(); issue_qk(0); }
+            for (int t = 0; t < nt && ok; ++t) {
+                const int s = t & 1;
+                if (t + 1 < nt) {   // next tile's scores, into the other buffer
+                    const int s1 = (t + 1) & 1;
+                    ok = mbar_wait(kv_full0 + 8 * s1, ((t + 1) >> 1) & 1);
+                    if (ok && t + 1 >= 2) ok = mbar_wait(s_empty0 + 8 * s1, (((t + 1) >> 1) - 1) & 1);
+                    if (!ok) break;
+                    fence_after_sync();
+                    issue_qk(t + 1);
+                }
+                ok = mbar_wait(p_full, t & 1);
+                if (!ok) break;
+                fence_after_sync();
+                const uint32_t bv = sbase + kSmV + s * kTile;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {   // sixteen keys per instruction
+                    const uint32_t offp = (ks >> 2) * kHalf + (ks & 3) * 32;            // P: K-major, keys along the row
+                    const uint64_t vdesc = smem_desc_sw128(bv + ks * 16 * 128, kHalf, 1024);   // V: MN-major, 16 key rows down
+                    mma_bf16_ss(tmem + kColO, smem_desc_sw128(sbase + kSmP + offp, 16, 1024), vdesc, idesc_pv, t > 0 || ks > 0);
+                    mma_bf16_ss(tmem + kColO, smem_desc_sw128(sbase + kSmP + kTile + offp, 16, 1024), vdesc, idesc_pv, true);
+                }
+                mma_commit(kv_empty0 + 8 * s);   // K and V of this stage are spent
+                mma_commit(p_empty);             // P may be overwritten, O may be read
+            }
+            if (!ok) *sh_fail = 1;
+        }
+    } else {
+        // ---- softmax: thread = one query row ----
+        const int q = warp & 3, r = q * 32 + lane;
+        const int row = qt * kT + r;                          // row among the G*m of this head group
+        const bool row_ok = row < rows_total;
+        const int qi = row % p.m;                             // which of the m queries
+        const int vis = p.causal ? len - (p.m - 1 - qi) : len;   // keys this row sees: [0, vis)
+        const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+        const int32_t* cnt = p.count ? p.count + (size_t)bh * p.cap : nullptr;
+        float m_run = -INFINITY, l_run = 0.f;
+        bool failed = false;
+        for (int t = 0; t < nt; ++t) {
+            const int s = t & 1, j0 = t * kT;
+            lc_s[s * kT + r] = (cnt != nullptr && j0 + r < len) ? lg2((float)max(cnt[j0 + r], 1)) : 0.f;
+            if (!mbar_wait(s_full0 + 8 * s, (t >> 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
+            fence_after_sync();
+            asm volatile("bar.sync 1, 128;\n" ::: "memory");   // the four softmax warps: log2(count) is in place
+            if (*sh_fail_sm) { failed = true; break; }
+            // Rows of the stage past the head's end hold whatever lies behind the cores (0 * NaN would poison
+            // the second product): this row's thread clears its V row.  K rows need nothing, their scores are masked.
+            if (j0 + r >= len) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    *reinterpret_cast<uint4*>(smem + kSmV + s * kTile + r * 128 + u * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    *reinterpret_cast<uint4*>(smem + kSmV + s * kTile + kHalf + r * 128 + u * 16) = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+            // pass 1: the row's largest score in this tile
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t g[32];
+                tmem_ld32(lane_addr + kColS + s * kT + c * 32, g);
+                tmem_ld_wait();
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                    const float x = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + c * 32 + k]);
+                    if (j0 + c * 32 + k < vis) mx = fmaxf(mx, x);
+                }
+            }
+            // P and O belong to the previous tile's second product until it is complete
+            if (t > 0 && !mbar_wait(p_empty, (t - 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
+            fence_after_sync();
+            const bool raise = mx > m_run + kMaxSlack;      // also the first finite score (m_run = -inf)
+            if (__any_sync(kFull, raise)) {
+                const float f = raise ? ex2(m_run - mx) : 1.f;   // 0 when nothing had been seen
+                if (t > 0) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(lane_addr + kColO + c * 32, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * f);
+                        tmem_st32(lane_addr + kColO + c * 32, o);
+                    }
+                    tmem_st_wait();
+                }
+                l_run *= f;
+                if (raise) m_run = mx;
+            }
+            // pass 2: weights, as bf16 pairs (leading part + remainder), into the swizzled K-major P tiles
+            const float mref = m_run == -INFINITY ? 0.f : m_run;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t g[32];
+                tmem_ld32(lane_addr + kColS + s * kT + c * 32, g);
+                tmem_ld_wait();
+                uint32_t hi[16], lo[16];
+#pragma unroll
+                for (int k = 0; k < 32; k += 2) {
+                    const float x0 = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + c * 32 + k]);
+                    const float x1 = fmaf(__uint_as_float(g[k + 1]), p.scale_log2, lc_s[s * kT + c * 32 + k + 1]);
+                    const float w0 = (j0 + c * 32 + k < vis) ? ex2(x0 - mref) : 0.f;
+                    const float w1 = (j0 + c * 32 + k + 1 < vis) ? ex2(x1 - mref) : 0.f;
+                    const uint32_t ph = pack2(w0, w1);
+                    const uint32_t pl = pack2(w0 - bf_lo(ph), w1 - bf_hi(ph));
+                    l_run += (bf_lo(ph) + bf_lo(pl)) + (bf_hi(ph) + bf_hi(pl));
+                    hi[k >> 1] = ph; lo[k >> 1] = pl;
+                }
+                // 32 keys = four 16-byte chunks of this row; chunk cc of the 64-key half sits at cc ^ (row & 7)
+                const int half = c >> 1;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int cc = (c & 1) * 4 + u;
+                    const uint32_t off = half * kHalf + r * 128 + ((cc ^ (r & 7)) << 4);
+                    *reinterpret_cast<uint4*>(smem + kSmP + off) = make_uint4(hi[4 * u], hi[4 * u + 1], hi[4 * u + 2], hi[4 * u + 3]);
+                    *reinterpret_cast<uint4*>(smem + kSmP + kTile + off) = make_uint4(lo[4 * u], lo[4 * u + 1], lo[4 * u + 2], lo[4 * u + 3]);
+                }
+            }
+            fence_before_sync();      // this thread's reads of the score buffer
+            fence_async_proxy();      // this thread's P stores, for the tensor core's reads
+            __syncwarp();
+            if (lane == 0) { mbar_arrive(s_empty0 + 8 * s); mbar_arrive(p_full); }
+        }
+        // ---- O / l -> bf16 -> global ----
+        if (!failed && nt > 0) {
+            if (!mbar_wait(p_empty, (nt - 1) & 1)) { *sh_fail = 1; failed = true; }
+            fence_after_sync();
+        }
+        __nv_bfloat16* orow = p.out + (size_t)(q_row0 + r) * 128;
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            if (nt > 0 && !failed) {
+                tmem_ld32(lane_addr + kColO + c * 32, o);
+                tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int k = 0; k < 32; ++k) o[k] = 0u;
+            }
+            if (row_ok) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    uint4 v;
+                    v.x = pack2(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
+                    v.y = pack2(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
+                    v.z = pack2(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
+                    v.w = pack2(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
+                    *reinterpret_cast<uint4*>(orow + c * 32 + u * 8) = v;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (*sh_fail) {   // a wait gave up: report it and give copies still in flight one more bounded wait
+        if (tid == 0) {
+            set_status(p.status, SC_ERR_TIMEOUT);
+            const int issued = *sh_issued;
+            if (nt > 0) mbar_wait(q_full, 0);
+            for (int t = max(issued - 2, 0); t < issued; ++t) mbar_wait(kv_full0 + 8 * (t & 1), (t >> 1) & 1);
+        }
+        __syncthreads();
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+}
+
+// Any dtype, any d <= 256: one warp per (sequence, query head, query), online softmax in fp32.
+template <typename T>
+__global__ void __launch_bounds__(128) prefill_generic_kernel(const T* __restrict__ q, int B, int Hq, int Hkv, int m, int d,
+                                                              const T* __restrict__ core_k, const T* __restrict__ core_v,
+                                                              const int32_t* __restrict__ count, int cap,
+                                                              const int32_t* __restrict__ core_len, float scale_log2, int causal,
+                                                              T* __restrict__ out) {
+    const int lane = threadIdx.x & 31;
+    const long long it = (long long)blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (it >= (long long)B * Hq * m) return;
+    const int i = (int)(it % m), hq = (int)((it / m) % Hq), b = (int)(it / ((long long)m * Hq));
+    const int h = hq / (Hq / Hkv);
+    const int len = max(min(core_len[b * Hkv + h], cap), 0);
+    const int vis = causal ? len - (m - 1 - i) : len;
+    const T* qr = q + it * d;
+    const long long cbase = ((long long)b * Hkv + h) * cap;
+    float qv[8], acc[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int c = lane + 32 * u;
+        qv[u] = c < d ? Elem<T>::load(qr + c) * scale_log2 : 0.f;
+        acc[u] = 0.f;
+    }
+    float mx = -INFINITY, lsum = 0.f;
+    for (int t = 0; t < vis; ++t) {
+        const T* kr = core_k + (cbase + t) * d;
+        const T* vr = core_v + (cbase + t) * d;
+        float s = 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int c = lane + 32 * u;
+            if (c < d) s = fmaf(qv[u], Elem<T>::load(kr + c), s);
+        }
+        s = warp_sum(s);
+        if (count != nullptr) s += log2f((float)max(count[cbase + t], 1));
+        const float mn = fmaxf(mx, s);
+        const float corr = exp2f(mx - mn), pw = exp2f(s - mn);
+        lsum = lsum * corr + pw;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int c = lane + 32 * u;
+            if (c < d) acc[u] = acc[u] * corr + pw * Elem<T>::load(vr + c);
+        }
+        mx = mn;
+    }
+    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int c = lane + 32 * u;
+        if (c < d) Elem<T>::store(out + it * d + c, acc[u] * inv);
+    }
+}
+
+}  // namespace pf
+
+cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
+    using namespace pf;
+    const float scale_log2 = (a.scale == 0.f ? 1.f / sqrtf((float)a.d) : a.scale) * 1.4426950408889634f;
+    const int causal = (a.flags & SC_FLAG_CAUSAL_TAIL) ? 1 : 0;
+    const int G = a.Hq / a.Hkv;
+    const long long q_rows = (long long)a.B * a.Hq * a.m, c_rows = (long long)a.B * a.Hkv * a.cap;
+    if (a.dt == SC_BF16 && a.d == 128 && !(a.flags & SC_FLAG_GENERIC) && a.cap > 0 && q_rows < 0x7fffffff &&
+        c_rows < 0x7fffffff && a.Hkv <= 65535 && a.B <= 65535) {
+        static bool attr_set[64] = {false};
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (!attr_set[dev & 63]) {
+            cudaFuncSetAttribute(prefill_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+            attr_set[dev & 63] = true;
+        }
+        Params p;
+        p.count = a.count; p.core_len = a.core_len; p.out = (__nv_bfloat16*)a.out;
+        p.Hq = a.Hq; p.Hkv = a.Hkv; p.m = a.m; p.cap = a.cap; p.causal = causal; p.scale_log2 = scale_log2; p.status = a.status;
+        if (make_map_bf16_rows(&p.map_q, a.q, 0, 0, 128, 1, 1, q_rows, kT) &&
+            make_map_bf16_rows(&p.map_k, a.core_k, 0, 0, 128, 1, 1, c_rows, kT) &&
+            make_map_bf16_rows(&p.map_v, a.core_v, 0, 0, 128, 1, 1, c_rows, kT)) {
+            const dim3 grid((unsigned)((G * a.m + kT - 1) / kT), a.Hkv, a.B);
+            prefill_umma_kernel<<<grid, kThreads, kSmemBytes, st>>>(p);
+            note_launches(1);
+            return cudaGetLastError();
+        }
+    }
+    const unsigned blocks = (unsigned)((q_rows + 3) / 4);
+    if (a.dt == SC_BF16)
+        prefill_generic_kernel<__nv_bfloat16><<<blocks, 128, 0, st>>>((const __nv_bfloat16*)a.q, a.B, a.Hq, a.Hkv, a.m, a.d,
+            (const __nv_bfloat16*)a.core_k, (const __nv_bfloat16*)a.core_v, a.count, a.cap, a.core_len, scale_log2, causal,
+            (__nv_bfloat16*)a.out);
+    else
+        prefill_generic_kernel<float><<<blocks, 128, 0, st>>>((const float*)a.q, a.B, a.Hq, a.Hkv, a.m, a.d, (const float*)a.core_k,
+            (const float*)a.core_v, a.count, a.cap, a.core_len, scale_log2, causal, (float*)a.out);
+    note_launches(1);
+    return cudaGetLastError();
+}
+
+}  // namespace sc
