@@ -61,6 +61,15 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
+def measured_tensor_peak():
+    """Dense bf16 TFLOP/s: the sustained figure (kernels here are timed inside loops of many launches)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+    return 1400.0, "fallback (sustained)"
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while timed regions run."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -387,6 +396,9 @@ def run_ours(args):
         t0 = time.time()
         line["configs"] = sweep_configs(args, dev, sampler, peak)
         line["configs"]["wall_s"] = time.time() - t0
+        t0 = time.time()
+        line["extras"] = measure_extras(dev, sampler, peak)
+        line["extras"]["wall_s"] = time.time() - t0
     sampler.stop()
     if not args.no_cpu_baseline and args.gpus == 1:
         line["cpu_baseline"] = cpu_baseline(w, budget_s=args.cpu_budget)
@@ -439,6 +451,132 @@ def measure_cell(w: synth.Workload, full_L: int, dev, sampler, peak, label: dict
     return rec
 
 
+def time_calls(fn, reps: int = 10):
+    """Median device time (ms) of fn() launched `reps` times after one warm-up call."""
+    fn()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, z in ev:
+        a.record(); fn(); z.record()
+    torch.cuda.synchronize()
+    return statistics.median(a.elapsed_time(z) for a, z in ev)
+
+
+def measure_extras(dev, sampler, peak):
+    """The rows beyond the three main calls, each on the Llama-3-8B 32K shape (a few layers): multi-query
+    Proportional Attention, clustering without chunking, fixed-size chunks, compression to a budget."""
+    from paper_2603_14303_b200 import binding as b
+    out = {}
+    tpeak, tkind = measured_tensor_peak()
+    w = synth.config(1, L=4)
+    pipe = Pipeline(w, dev)
+    pipe.run_compress()
+    torch.cuda.synchronize()
+    lens = torch.stack([ly.core_len for ly in pipe.layers]).to(torch.int64)
+    rows_per_layer = lens.sum().item() / w.L
+
+    # -- sc_prefill_attn: m queries per head against the compressed cache, one launch per layer
+    t0 = time.time()
+    pre = {"what": "sc_prefill_attn: a block of m queries per head over the compressed cache, one launch per layer; "
+                   "flops = 4 * (G*m) * core rows * d per KV head (scores + weighted sum)", "peak_tflops": tpeak,
+           "peak_kind": tkind, "cells": []}
+    for m in (128, 512, 2048):
+        q = torch.randn((w.L, w.B, w.Hq, m, w.d), device=dev).to(torch.bfloat16)
+        o = torch.empty_like(q)
+        st = torch.zeros(1, dtype=torch.int32, device=dev)
+
+        def run():
+            for l in range(w.L):
+                b.sc_prefill_attn(q[l], pipe.layers[l].core_k, pipe.layers[l].core_v, pipe.layers[l].count,
+                                  pipe.layers[l].core_len, o[l], 0.0, st)
+        ms = time_calls(run) / w.L
+        flops = 4.0 * w.G * m * rows_per_layer * w.d
+        tf = flops / (ms * 1e-3) / 1e12
+        pre["cells"].append({"m": m, "query_rows_per_kv_head": w.G * m, "us_per_layer": ms * 1e3, "tflops": tf,
+                             "frac_of_tensor_peak": tf / tpeak, "query_tokens_per_s": w.B * m / (ms * 1e-3 * 32)})
+        if int(st.item()) != 0:
+            raise RuntimeError("sc_prefill_attn reported a device-side error")
+        del q, o
+    pre["roofline"] = {"bound": "tensor", "achieved": max(c["tflops"] for c in pre["cells"]), "peak": tpeak,
+                       "unit": "TFLOP/s", "frac": max(c["frac_of_tensor_peak"] for c in pre["cells"]),
+                       "traffic": recorded_traffic(w.name, "prefill")}
+    pre["clocks"] = sampler.summary(t0, time.time())
+    out["prefill_attn"] = pre
+
+    # -- fixed-size chunks of 64 tokens (Table 4a's second arm): same kernels, other plan
+    t0 = time.time()
+    plan64 = b.chunk_fixed(pipe.ids_dev, 64)
+    lay = pipe.layers
+
+    def run_fixed():
+        for l in range(w.L):
+            b.sc_compress(pipe.K[l], pipe.V[l], plan64, w.tau, lay[l].core_k, lay[l].core_v, lay[l].count, lay[l].core_len,
+                          None, pipe.cws[l], pipe.cstatus[l], 0)
+    ms = time_calls(run_fixed) / w.L
+    kept = torch.stack([ly.core_len for ly in lay]).sum().item() / (w.L * w.B * w.Hkv * w.n)
+    cbytes = w.B * w.Hkv * w.n * w.d * 2 * 2 * (1 + kept) + 4 * kept * w.B * w.Hkv * w.n
+    out["fixed_chunks_64"] = {"what": "sc_chunk with no delimiters and max_chunk_len 64, then sc_compress", "layers_run": w.L,
+                              "kept_fraction": round(kept, 4), "compress_us_per_layer": ms * 1e3,
+                              "compress_ms_per_32k_ctx": ms * 32 * 32768 / (w.B * w.n),
+                              "compress_frac": cbytes / (ms * 1e-3) / 1e9 / peak, "clocks": sampler.summary(t0, time.time())}
+    pipe.run_compress()      # back to the semantic plan's cores
+
+    # -- clustering without chunking (Table 4a's third arm)
+    t0 = time.time()
+    gws = torch.empty(b.lib().sc_compress_global_workspace_bytes(w.B, w.Hkv, w.n), dtype=torch.uint8, device=dev)
+    gl_layers = 2
+
+    def run_global():
+        for l in range(gl_layers):
+            b.sc_compress_global(pipe.K[l], pipe.V[l], w.tau, lay[l].core_k, lay[l].core_v, lay[l].count, lay[l].core_len,
+                                 gws, None, pipe.cstatus[l], 0)
+    ms = time_calls(run_global, 5) / gl_layers
+    kept = torch.stack([ly.core_len for ly in lay[:gl_layers]]).sum().item() / (gl_layers * w.B * w.Hkv * w.n)
+    pair_flops = float(w.B * w.Hkv) * w.n * w.n * w.d       # n^2 / 2 pairs, 2 d flops each
+    out["global_clustering"] = {"what": "sc_compress_global: Algorithm 1 over whole sequences; pairwise stage = n^2/2 * 2d flops per head",
+                                "layers_run": gl_layers, "kept_fraction": round(kept, 4), "ms_per_layer": ms,
+                                "ms_per_32k_ctx": ms * 32 * 32768 / (w.B * w.n), "pairwise_tflops_if_all_time": pair_flops / (ms * 1e-3) / 1e12,
+                                "workspace_mb": gws.numel() / 1e6, "clocks": sampler.summary(t0, time.time())}
+    del gws
+    if int(pipe.cstatus.abs().max().item()) != 0:
+        raise RuntimeError("device-side error in the ablation arms")
+    del pipe
+    torch.cuda.empty_cache()
+
+    # -- compression to a budget: keys noisy enough that the kept fraction depends on the threshold
+    t0 = time.time()
+    wb = synth.config(1, L=4, sigma=0.6)
+    pipe = Pipeline(wb, dev, cap_frac=1.0)
+    pipe.run_compress()
+    bws = [torch.zeros(b.lib().sc_compress_budget_workspace_bytes(wb.B, wb.Hkv, wb.n), dtype=torch.uint8, device=dev)
+           for _ in range(wb.L)]
+    tau = torch.zeros((wb.L, 1), dtype=torch.float32, device=dev)
+    srch = torch.zeros((wb.L, 2), dtype=torch.int32, device=dev)
+    lay = pipe.layers
+    cells = []
+    for target in (0.35, 0.5):
+        def run_budget():
+            for l in range(wb.L):
+                b.sc_compress_budget(pipe.K[l], pipe.V[l], pipe.plan, target, 0.5, 0.9, 17, lay[l].core_k, lay[l].core_v,
+                                     lay[l].count, lay[l].core_len, tau[l], srch[l], bws[l], None, pipe.cstatus[l], 0)
+        ms = time_calls(run_budget, 5) / wb.L
+        ms_plain = time_calls(lambda: [b.sc_compress(pipe.K[l], pipe.V[l], pipe.plan, 0.7, lay[l].core_k, lay[l].core_v,
+                                                     lay[l].count, lay[l].core_len, None, pipe.cws[l], pipe.cstatus[l], 0)
+                                       for l in range(wb.L)], 3) / wb.L
+        run_budget()
+        torch.cuda.synchronize()
+        kept = torch.stack([ly.core_len for ly in lay]).sum().item() / (wb.L * wb.B * wb.Hkv * wb.n)
+        cells.append({"target_kept": target, "achieved_kept": round(kept, 4), "tau_chosen": [round(float(x), 4) for x in tau.flatten().tolist()],
+                      "counting_passes": srch[:, 1].tolist(), "us_per_layer": ms * 1e3, "ms_per_32k_ctx": ms * 32 * 32768 / (wb.B * wb.n),
+                      "plain_compress_us_per_layer": ms_plain * 1e3})
+    out["budget"] = {"what": "sc_compress_budget on keys with noise 0.6 (kept fraction varies over the grid), grid of 17 thresholds in [0.5, 0.9]",
+                     "layers_run": wb.L, "cells": cells, "clocks": sampler.summary(t0, time.time())}
+    if int(pipe.cstatus.abs().max().item()) != 0:
+        raise RuntimeError("device-side error in the budget search")
+    del pipe
+    torch.cuda.empty_cache()
+    return out
+
+
 def sweep_configs(args, dev, sampler, peak):
     """Short passes over the other workloads and the sweeps two of them name (after the headline run).
 
@@ -449,7 +587,7 @@ def sweep_configs(args, dev, sampler, peak):
     c0, c2, c3, c4 = (synth.config(i) for i in (0, 2, 3, 4))
     out["cfg0"] = measure_cell(c0, c0.L, dev, sampler, peak, {"workload": c0.name, "note": "L2-resident toy"},
                                decode_steps=32)
-    out["cfg2"] = measure_cell(c2.replace(L=2), c2.L, dev, sampler, peak, {"workload": c2.name})
+    out["cfg2"] = measure_cell(c2.replace(L=4), c2.L, dev, sampler, peak, {"workload": c2.name})
     # cfg3: noise swept at tau = 0.9 (the norm reading of the noise), plus the literal reading where nothing merges
     cells = []
     for sigma in (0.05, 0.15, 0.3):
@@ -463,7 +601,7 @@ def sweep_configs(args, dev, sampler, peak):
     grid = []
     for mean_len in (8, 32, 128):
         for r in (2, 4, 8):
-            wc = c4.replace(L=2, gap=("poisson", float(mean_len)), centroids=("ratio", float(r)))
+            wc = c4.replace(L=3, gap=("poisson", float(mean_len)), centroids=("ratio", float(r)))
             rec = measure_cell(wc, c4.L, dev, sampler, peak,
                                {"workload": c4.name, "mean_chunk_len": mean_len, "target_reduction": r}, raw=True,
                                cap_frac=1.0 if r == 2 else 0.5)
@@ -670,6 +808,8 @@ def main():
     ap.add_argument("--no-overlap", action="store_true", help="time the step with plain stream-ordered decode launches")
     ap.add_argument("--no-modes", action="store_true", help="skip the side measurements of the other decode launch modes")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short passes over the other workloads and sweeps")
+    ap.add_argument("--extras-only", action="store_true",
+                    help="run only the measurements of sc_prefill_attn, the ablation arms and the budget search (a small case for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=20.0)
     ap.add_argument("--traffic", type=float, default=None,
@@ -677,6 +817,16 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.extras_only:
+        from paper_2603_14303_b200 import build
+        build.build()
+        dev = torch.device("cuda:0")
+        torch.cuda.set_device(dev)
+        sampler = ClockSampler(0)
+        sampler.start()
+        extras = measure_extras(dev, sampler, measured_peaks()[0])
+        sampler.stop()
+        print(json.dumps({"extras": extras}))
     else:
         run_ours(args)
 

@@ -200,45 +200,48 @@ chunk_write(const int32_t* __restrict__ token_ids, int n, int tps, DelimSet D, i
 }
 
 // Kernel 5: one block per sequence packs consecutive segments into work tiles: as many whole
-// segments as fit in SC_TILE_ROWS tokens, or one longer segment alone.  The chain
-// tile -> next tile is sequential, so the sequence's offsets are staged through shared memory
-// in windows and one warp walks them.
+// segments as fit in SC_TILE_ROWS tokens, or one longer segment alone.  The chain tile -> next tile is
+// sequential, but where a tile that starts at segment s ends does not depend on the chain: the
+// sequence's offsets are staged through shared memory in windows, every thread finds the end of the
+// tile that would start at its segments (a binary search over the monotone offsets), and one thread then
+// walks the chain with a single shared-memory lookup per tile.
 __global__ void __launch_bounds__(kChunkThreads)
 chunk_pack_tiles(const int32_t* __restrict__ seg_off, const int32_t* __restrict__ seq_seg_off, int n_seg_cap,
                  int32_t* __restrict__ tile_seg, int n_tile_cap, int32_t* __restrict__ seq_tile_cnt,
                  int32_t* status) {
     __shared__ int buf[kPackWindow + 1];
+    __shared__ int nxt[kPackWindow];       // window index of the segment the next tile starts at
     __shared__ int sh_cur, sh_nt;
     const int b = blockIdx.x;
     const int s0 = seq_seg_off[b];
     const int s1 = min(seq_seg_off[b + 1], n_seg_cap);  // clamped when sc_chunk overflowed
     int32_t* out = tile_seg + (int64_t)b * (n_tile_cap + 1);
     int cur = s0, nt = 0;
-    const int lane = threadIdx.x & 31;
     while (cur < s1) {
         const int ws = cur;
         const int cnt = min(kPackWindow, s1 - ws);
         for (int i = threadIdx.x; i <= cnt; i += kChunkThreads) buf[i] = seg_off[ws + i];
         __syncthreads();
-        if (threadIdx.x < 32) {
+        for (int i = threadIdx.x; i < cnt; i += kChunkThreads) {
+            // largest e in (i, cnt] with buf[e] - buf[i] <= SC_TILE_ROWS, or i + 1 for a segment longer than a tile
+            const int limit = buf[i] + SC_TILE_ROWS;
+            int lo = i + 1, hi = min(cnt, i + SC_TILE_ROWS);   // a segment holds at least one token
+            while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (buf[mid] <= limit) lo = mid; else hi = mid - 1;
+            }
+            nxt[i] = lo;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            // a tile's end is known for sure only if SC_TILE_ROWS + 1 offsets behind its start are in the window
             const bool last_window = (ws + cnt == s1);
             while (cur < s1 && (last_window || cur - ws + SC_TILE_ROWS + 1 <= cnt)) {
-                const int base = buf[cur - ws];
-                int e = cur;
-                for (;;) {
-                    int idx = e + 1 + lane;
-                    bool ok = (idx - ws <= cnt) && (buf[idx - ws] - base <= SC_TILE_ROWS);
-                    unsigned m = __ballot_sync(kFull, ok);
-                    int c = (m == kFull) ? 32 : (__ffs(~m) - 1);
-                    e += c;
-                    if (c < 32) break;
-                }
-                if (e == cur) e = cur + 1;  // one segment longer than a tile
-                if (lane == 0 && nt < n_tile_cap) out[nt] = cur;
+                if (nt < n_tile_cap) out[nt] = cur;
                 ++nt;
-                cur = e;
+                cur = ws + nxt[cur - ws];
             }
-            if (lane == 0) { sh_cur = cur; sh_nt = nt; }
+            sh_cur = cur; sh_nt = nt;
         }
         __syncthreads();
         cur = sh_cur; nt = sh_nt;

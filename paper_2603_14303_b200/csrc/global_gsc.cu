@@ -17,7 +17,8 @@
 //      number of rounds is enqueued (clustered keys need three or four); rounds that find nothing left
 //      return at once, and a last kernel finishes whatever is left one head per block;
 //   4. every member's seed (its lowest adjacent seed), the seeds' ranks (prefix sum) and core_len;
-//   5. Eq. 3: one warp per cluster sums its members in token order (fp32), divides once, rounds once.
+//   5. Eq. 3: the tokens are binned by cluster (sizes, prefix sum, fill), then one warp per cluster puts
+//      its members in token order and sums them (fp32), divides once, rounds once.
 #include "common.cuh"
 #include "umma.cuh"
 
@@ -384,60 +385,132 @@ __global__ void __launch_bounds__(256) assign_kernel(const uint32_t* __restrict_
     }
 }
 
-// Step 5 (Eq. 3): one warp per token; a seed's warp walks the tokens behind it and pools its members in order.
-template <typename T>
-__global__ void __launch_bounds__(256) merge_kernel(const T* __restrict__ K, const T* __restrict__ V, sc_strides st, int Hkv, int n,
-                                                    int d, int heads, const uint32_t* __restrict__ seed,
-                                                    const int32_t* __restrict__ rank_base, const int32_t* __restrict__ assign,
-                                                    T* __restrict__ core_k, T* __restrict__ core_v, int32_t* __restrict__ count, int cap) {
-    const int lane = threadIdx.x & 31;
+// Step 5a: cluster index of a token = rank of its seed among the head's seeds.
+__device__ __forceinline__ int cluster_of(const uint32_t* __restrict__ seed, const int32_t* __restrict__ rank_base, int seed_pos) {
+    const uint32_t sw = seed[seed_pos >> 5];
+    return rank_base[seed_pos >> 5] + __popc(sw & ((1u << (seed_pos & 31)) - 1u));
+}
+
+// Step 5b: cluster sizes (phase 0), then every token into its cluster's slice of the member list (phase 1).
+// The order inside a slice is whatever the atomics gave; the pooling kernel puts it right.
+__global__ void __launch_bounds__(256) members_kernel(int n, int heads, const uint32_t* __restrict__ seed,
+                                                      const int32_t* __restrict__ rank_base, const int32_t* __restrict__ assign,
+                                                      int32_t* __restrict__ csize, const int32_t* __restrict__ coff,
+                                                      int32_t* __restrict__ cursor, int32_t* __restrict__ members, int phase) {
     const int nw = (n + 31) >> 5;
     const long long rows = (long long)heads * n;
-    for (long long rid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); rid < rows; rid += (long long)gridDim.x * 8) {
-        const int bh = (int)(rid / n), i = (int)(rid - (long long)bh * n);
-        const uint32_t sw = seed[(size_t)bh * nw + (i >> 5)];
-        if (!((sw >> (i & 31)) & 1u)) continue;
-        const int rank = rank_base[(size_t)bh * nw + (i >> 5)] + __popc(sw & ((1u << (i & 31)) - 1u));
-        if (rank >= cap) continue;
+    for (long long rid = (long long)blockIdx.x * blockDim.x + threadIdx.x; rid < rows; rid += (long long)gridDim.x * blockDim.x) {
+        const int bh = (int)(rid / n), j = (int)(rid - (long long)bh * n);
+        const int c = cluster_of(seed + (size_t)bh * nw, rank_base + (size_t)bh * nw, assign[rid]);
+        if (phase == 0) atomicAdd(&csize[(size_t)bh * n + c], 1);
+        else members[(size_t)bh * n + coff[(size_t)bh * n + c] + atomicAdd(&cursor[(size_t)bh * n + c], 1)] = j;
+    }
+}
+
+// Step 5c: exclusive prefix sum of the cluster sizes per head.
+__global__ void __launch_bounds__(1024) offsets_kernel(int n, const int32_t* __restrict__ core_len, const int32_t* __restrict__ csize,
+                                                       int32_t* __restrict__ coff) {
+    __shared__ int wsum[32];
+    const int bh = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int S = min(core_len[bh], n);
+    int carry = 0;
+    for (int base = 0; base < S; base += 1024) {
+        const int c = base + threadIdx.x;
+        const int v = c < S ? csize[(size_t)bh * n + c] : 0;
+        const int incl = warp_scan_add(v, lane);
+        if (lane == 31) wsum[warp] = incl;
+        __syncthreads();
+        int pre = 0, tot = 0;
+        for (int k = 0; k < 32; ++k) { if (k < warp) pre += wsum[k]; tot += wsum[k]; }
+        __syncthreads();
+        if (c < S) coff[(size_t)bh * n + c] = carry + pre + incl - v;
+        carry += tot;
+    }
+}
+
+// Step 5d (Eq. 3): one warp per cluster pools its members in token order (fp32 sums, one divide, one rounding).
+// Up to 32 members are ordered in registers; up to kMidCluster by repeatedly taking the next larger position;
+// beyond that the warp walks the head's assignment array, which is already in token order.
+constexpr int kMidCluster = 1024;
+template <typename T>
+__device__ __forceinline__ void add_row(const T* __restrict__ Kh, const T* __restrict__ Vh, long long sn, int jj, int d, int lane,
+                                        float (&sk)[8], float (&sv)[8]) {
+    const T* kr = Kh + (long long)jj * sn;
+    const T* vr = Vh + (long long)jj * sn;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int c = lane + 32 * u;
+        if (c < d) { sk[u] += Elem<T>::load(kr + c); sv[u] += Elem<T>::load(vr + c); }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) merge_kernel(const T* __restrict__ K, const T* __restrict__ V, sc_strides st, int Hkv, int n,
+                                                    int d, int heads, const int32_t* __restrict__ core_len,
+                                                    const int32_t* __restrict__ csize, const int32_t* __restrict__ coff,
+                                                    const int32_t* __restrict__ members, const int32_t* __restrict__ assign,
+                                                    T* __restrict__ core_k, T* __restrict__ core_v, int32_t* __restrict__ count, int cap) {
+    const int lane = threadIdx.x & 31;
+    const long long slots = (long long)heads * n;
+    for (long long sid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); sid < slots; sid += (long long)gridDim.x * 8) {
+        const int bh = (int)(sid / n), c = (int)(sid - (long long)bh * n);
+        if (c >= min(core_len[bh], cap)) continue;
         const T* Kh = K + (bh / Hkv) * st.b + (bh % Hkv) * st.h;
         const T* Vh = V + (bh / Hkv) * st.b + (bh % Hkv) * st.h;
-        const int32_t* as = assign + (size_t)bh * n;
+        const int cnt = csize[(size_t)bh * n + c];
+        const int32_t* mem = members + (size_t)bh * n + coff[(size_t)bh * n + c];
         float sk[8], sv[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) sk[u] = sv[u] = 0.f;
-        int cnt = 0;
-        for (int j0 = i & ~31; j0 < n; j0 += 32) {
-            const int j = j0 + lane;
-            uint32_t mem = __ballot_sync(kFull, j < n && j >= i && as[j] == i);
-            cnt += __popc(mem);
-            while (mem) {
-                const int jj = j0 + __ffs(mem) - 1;
-                mem &= mem - 1;
-                const T* kr = Kh + (long long)jj * st.n;
-                const T* vr = Vh + (long long)jj * st.n;
+        if (cnt <= 32) {
+            const int mine = lane < cnt ? mem[lane] : 0x7fffffff;
+            int pos = 0;
+            for (int k = 0; k < cnt; ++k) pos += __shfl_sync(kFull, mine, k) < mine;
+            for (int t = 0; t < cnt; ++t) {
+                const int src = __ffs(__ballot_sync(kFull, lane < cnt && pos == t)) - 1;
+                add_row<T>(Kh, Vh, st.n, __shfl_sync(kFull, mine, src), d, lane, sk, sv);
+            }
+        } else if (cnt <= kMidCluster) {
+            int last = -1;
+            for (int t = 0; t < cnt; ++t) {
+                int best = 0x7fffffff;
+                for (int k = lane; k < cnt; k += 32) { const int v = mem[k]; if (v > last && v < best) best = v; }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int c = lane + 32 * u;
-                    if (c < d) { sk[u] += Elem<T>::load(kr + c); sv[u] += Elem<T>::load(vr + c); }
+                for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(kFull, best, o));
+                add_row<T>(Kh, Vh, st.n, best, d, lane, sk, sv);
+                last = best;
+            }
+        } else {
+            const int32_t* as = assign + (size_t)bh * n;
+            int seed_pos = 0x7fffffff;   // the cluster's seed is its smallest member
+            for (int k = lane; k < cnt; k += 32) seed_pos = min(seed_pos, mem[k]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) seed_pos = min(seed_pos, __shfl_xor_sync(kFull, seed_pos, o));
+            for (int j0 = seed_pos & ~31; j0 < n; j0 += 32) {
+                const int j = j0 + lane;
+                uint32_t hit = __ballot_sync(kFull, j < n && as[j] == seed_pos);
+                while (hit) {
+                    add_row<T>(Kh, Vh, st.n, j0 + __ffs(hit) - 1, d, lane, sk, sv);
+                    hit &= hit - 1;
                 }
             }
         }
-        const size_t o = ((size_t)bh * cap + rank) * d;
+        const size_t o = ((size_t)bh * cap + c) * d;
         const float fc = (float)cnt;
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const int c = lane + 32 * u;
-            if (c < d) {
-                Elem<T>::store(core_k + o + c, sk[u] / fc);
-                Elem<T>::store(core_v + o + c, sv[u] / fc);
+            const int col = lane + 32 * u;
+            if (col < d) {
+                Elem<T>::store(core_k + o + col, sk[u] / fc);
+                Elem<T>::store(core_v + o + col, sv[u] / fc);
             }
         }
-        if (lane == 0) count[(size_t)bh * cap + rank] = cnt;
+        if (lane == 0) count[(size_t)bh * cap + c] = cnt;
     }
 }
 
 struct Layout {   // workspace: every part 256-byte aligned
-    size_t norms, bits, seed, member, rank, assign, ctl, total;
+    size_t norms, bits, seed, member, rank, assign, csize, coff, members, ctl, total;
 };
 inline Layout layout_for(int B, int Hkv, int n) {
     const size_t heads = (size_t)B * Hkv, nb = (n + kT - 1) / kT, nw = (n + 31) / 32;
@@ -450,6 +523,9 @@ inline Layout layout_for(int B, int Hkv, int n) {
     L.member = off; off += up(4 * heads * nw);
     L.rank = off; off += up(4 * heads * nw);
     L.assign = off; off += up(4 * heads * n);
+    L.csize = off; off += 2 * up(4 * heads * n);      // cluster sizes, then the fill cursors (cleared together)
+    L.coff = off; off += up(4 * heads * n);
+    L.members = off; off += up(4 * heads * n);
     L.ctl = off; off += 256;
     L.total = off;
     return L;
@@ -503,9 +579,19 @@ static cudaError_t run_global(const GlobalArgs& a, cudaStream_t st) {
     finish_kernel<<<heads, 1024, 0, st>>>(bits, a.n, nb, m);
     rank_kernel<<<heads, 1024, 0, st>>>(m.seed, a.n, rank_base, a.core_len, a.cap, a.status);
     assign_kernel<<<round_grid, 256, 0, st>>>(bits, a.n, nb, heads, m.seed, assign);
-    merge_kernel<T><<<round_grid, 256, 0, st>>>((const T*)a.K, (const T*)a.V, a.st, a.Hkv, a.n, a.d, heads, m.seed, rank_base,
-                                                assign, (T*)a.core_k, (T*)a.core_v, a.count, a.cap);
-    note_launches(launched + kRounds + 4);
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    int32_t* csize = (int32_t*)(ws + L.csize);
+    int32_t* cursor = (int32_t*)(ws + L.csize + up(4 * (size_t)heads * a.n));
+    int32_t* coff = (int32_t*)(ws + L.coff);
+    int32_t* members = (int32_t*)(ws + L.members);
+    cudaMemsetAsync(csize, 0, 2 * up(4 * (size_t)heads * a.n), st);
+    const int tok_grid = (int)(rows / 256 < (long long)sms * 8 ? (rows + 255) / 256 : (long long)sms * 8);
+    members_kernel<<<tok_grid, 256, 0, st>>>(a.n, heads, m.seed, rank_base, assign, csize, coff, cursor, members, 0);
+    offsets_kernel<<<heads, 1024, 0, st>>>(a.n, a.core_len, csize, coff);
+    members_kernel<<<tok_grid, 256, 0, st>>>(a.n, heads, m.seed, rank_base, assign, csize, coff, cursor, members, 1);
+    merge_kernel<T><<<round_grid, 256, 0, st>>>((const T*)a.K, (const T*)a.V, a.st, a.Hkv, a.n, a.d, heads, a.core_len, csize, coff,
+                                                members, assign, (T*)a.core_k, (T*)a.core_v, a.count, a.cap);
+    note_launches(launched + kRounds + 7);
     return cudaGetLastError();
 }
 

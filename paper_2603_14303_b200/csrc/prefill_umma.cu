@@ -8,7 +8,8 @@
 //   warp 1     issues the MMAs: S = Q K^T into one of two score buffers in tensor memory (so the next
 //              tile's scores are computed while this tile's are being exponentiated), then O += P V,
 //              V read as an MN-major operand straight from its [keys x dims] tile;
-//   warps 2-5  softmax, one thread per query row (= tensor-memory lane, so no cross-thread reduction):
+//   warps 2-9  softmax, two threads per query row (= tensor-memory lane; each owns half of a tile's keys and
+//              half of the accumulator's columns, the row maximum is exchanged through shared memory):
 //              x = S * scale*log2(e) + log2(count), masks (head length, optional causal tail), running
 //              maximum raised lazily (the accumulator row is rescaled in tensor memory only then),
 //              P = 2^(x - m) written to shared memory as a bf16 pair (leading part + remainder) in
@@ -27,11 +28,12 @@ using namespace umma;
 constexpr int kT = 128;                       // query rows per CTA, keys per tile
 constexpr int kHalf = kT * 128;               // 16384 bytes: one 64-column half of a [128 x 128] bf16 tile
 constexpr int kTile = 2 * kHalf;              // 32768
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                 // warp 0: TMA, warp 1: MMA + tensor memory, warps 2-9: softmax
 constexpr int kTmemCols = 512;                // S0 | S1 | O (128 columns each), rounded up to a power of two
 constexpr int kColS = 0, kColO = 256;
-constexpr int kSmQ = 0, kSmK = kTile, kSmV = 3 * kTile, kSmP = 5 * kTile, kSmLc = 7 * kTile, kSmBar = kSmLc + 2 * kT * 4;
-constexpr int kSmemBytes = kSmBar + 256 + 1024;
+constexpr int kSmQ = 0, kSmK = kTile, kSmV = 3 * kTile, kSmP = 5 * kTile, kSmLc = 7 * kTile, kSmMx = kSmLc + 2 * kT * 4,
+              kSmBar = kSmMx + 2 * kT * 4;
+constexpr int kSmemBytes = kSmBar + 256;
 constexpr float kMaxSlack = 8.f;              // log2 units a score may exceed the running maximum before it is raised
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
@@ -66,16 +68,20 @@ __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v <<
 __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
 __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_constant__ Params p) {
-    extern __shared__ unsigned char smem_raw[];
+    extern __shared__ __align__(1024) unsigned char smem[];   // the swizzle pattern repeats every 1024 bytes
     const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
     const int G = p.Hq / p.Hkv, bh = b * p.Hkv + h;
     const int rows_total = G * p.m;                           // query rows of this (sequence, KV head)
     const int len = max(min(p.core_len[bh], p.cap), 0);
     const int nt = (len + kT - 1) / kT;                       // key tiles
     const long long q_row0 = ((long long)b * p.Hq + (long long)h * G) * p.m + (long long)qt * kT;
-    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    unsigned char* smem = smem_raw + (sbase - smem_u32(smem_raw));
+    const uint32_t sbase = smem_u32(smem);
+    if ((sbase & 1023u) != 0u) {   // the swizzled addressing assumes this; uniform over the block
+        if (threadIdx.x == 0) set_status(p.status, SC_ERR_CUDA);
+        return;
+    }
     float* lc_s = reinterpret_cast<float*>(smem + kSmLc);     // [2][128] log2(count) of the tile's keys
+    float* mx_s = reinterpret_cast<float*>(smem + kSmMx);     // [2][128] each half's row maximum (at the end the row sums)
     const uint32_t bar0 = sbase + kSmBar;
     const uint32_t q_full = bar0, kv_full0 = bar0 + 8, kv_empty0 = bar0 + 24, s_full0 = bar0 + 40, s_empty0 = bar0 + 56,
                    p_full = bar0 + 72, p_empty = bar0 + 80;
@@ -91,9 +97,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
             mbar_init(kv_full0 + 8 * s, 1);
             mbar_init(kv_empty0 + 8 * s, 1);
             mbar_init(s_full0 + 8 * s, 1);
-            mbar_init(s_empty0 + 8 * s, 4);
+            mbar_init(s_empty0 + 8 * s, 8);
         }
-        mbar_init(p_full, 4);
+        mbar_init(p_full, 8);
         mbar_init(p_empty, 1);
         mbar_fence_init();
         *sh_fail = 0; *sh_fail_sm = 0; *sh_issued = 0;
@@ -167,60 +173,62 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
             if (!ok) *sh_fail = 1;
         }
     } else {
-        // ---- softmax: thread = one query row ----
-        const int q = warp & 3, r = q * 32 + lane;
+        // ---- softmax: two threads per query row (= tensor-memory lane), each owning 64 of a tile's 128 keys
+        //      and 64 of the accumulator's 128 columns; warps 2-5 take the first halves, warps 6-9 the second ----
+        const int q = warp & 3, r = q * 32 + lane, wg = (warp - 2) >> 2;
         const int row = qt * kT + r;                          // row among the G*m of this head group
         const bool row_ok = row < rows_total;
         const int qi = row % p.m;                             // which of the m queries
         const int vis = p.causal ? len - (p.m - 1 - qi) : len;   // keys this row sees: [0, vis)
         const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
         const int32_t* cnt = p.count ? p.count + (size_t)bh * p.cap : nullptr;
-        float m_run = -INFINITY, l_run = 0.f;
+        float m_run = -INFINITY, l_run = 0.f;                 // l_run: this thread's keys only
         bool failed = false;
         for (int t = 0; t < nt; ++t) {
-            const int s = t & 1, j0 = t * kT;
-            lc_s[s * kT + r] = (cnt != nullptr && j0 + r < len) ? lg2((float)max(cnt[j0 + r], 1)) : 0.f;
+            const int s = t & 1, j0 = t * kT, jw = j0 + wg * 64;   // jw: first key of this thread's half
+            if (wg == 0) lc_s[s * kT + r] = (cnt != nullptr && j0 + r < len) ? lg2((float)max(cnt[j0 + r], 1)) : 0.f;
             if (!mbar_wait(s_full0 + 8 * s, (t >> 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
             fence_after_sync();
-            asm volatile("bar.sync 1, 128;\n" ::: "memory");   // the four softmax warps: log2(count) is in place
+            asm volatile("bar.sync 1, 256;\n" ::: "memory");   // the eight softmax warps: log2(count) is in place
             if (*sh_fail_sm) { failed = true; break; }
             // Rows of the stage past the head's end hold whatever lies behind the cores (0 * NaN would poison
-            // the second product): this row's thread clears its V row.  K rows need nothing, their scores are masked.
+            // the second product): this row's threads clear its V row.  K rows need nothing, their scores are masked.
             if (j0 + r >= len) {
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    *reinterpret_cast<uint4*>(smem + kSmV + s * kTile + r * 128 + u * 16) = make_uint4(0u, 0u, 0u, 0u);
-                    *reinterpret_cast<uint4*>(smem + kSmV + s * kTile + kHalf + r * 128 + u * 16) = make_uint4(0u, 0u, 0u, 0u);
-                }
+                for (int u = 0; u < 8; ++u)
+                    *reinterpret_cast<uint4*>(smem + kSmV + s * kTile + wg * kHalf + r * 128 + u * 16) = make_uint4(0u, 0u, 0u, 0u);
             }
-            // pass 1: the row's largest score in this tile
+            // pass 1: the row's largest score in this tile (each thread its half, then the two are exchanged)
             float mx = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t g[32];
-                tmem_ld32(lane_addr + kColS + s * kT + c * 32, g);
+                tmem_ld32(lane_addr + kColS + s * kT + wg * 64 + c * 32, g);
                 tmem_ld_wait();
 #pragma unroll
                 for (int k = 0; k < 32; ++k) {
-                    const float x = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + c * 32 + k]);
-                    if (j0 + c * 32 + k < vis) mx = fmaxf(mx, x);
+                    const float x = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k]);
+                    if (jw + c * 32 + k < vis) mx = fmaxf(mx, x);
                 }
             }
+            mx_s[wg * kT + r] = mx;
             // P and O belong to the previous tile's second product until it is complete
             if (t > 0 && !mbar_wait(p_empty, (t - 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
             fence_after_sync();
-            const bool raise = mx > m_run + kMaxSlack;      // also the first finite score (m_run = -inf)
+            asm volatile("bar.sync 2, 256;\n" ::: "memory");   // both halves' maxima are in place
+            mx = fmaxf(mx, mx_s[(wg ^ 1) * kT + r]);
+            const bool raise = mx > m_run + kMaxSlack;      // also the first finite score (m_run = -inf); same in both threads
             if (__any_sync(kFull, raise)) {
                 const float f = raise ? ex2(m_run - mx) : 1.f;   // 0 when nothing had been seen
                 if (t > 0) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < 2; ++c) {
                         uint32_t o[32];
-                        tmem_ld32(lane_addr + kColO + c * 32, o);
+                        tmem_ld32(lane_addr + kColO + wg * 64 + c * 32, o);
                         tmem_ld_wait();
 #pragma unroll
                         for (int k = 0; k < 32; ++k) o[k] = __float_as_uint(__uint_as_float(o[k]) * f);
-                        tmem_st32(lane_addr + kColO + c * 32, o);
+                        tmem_st32(lane_addr + kColO + wg * 64 + c * 32, o);
                     }
                     tmem_st_wait();
                 }
@@ -230,49 +238,52 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
             // pass 2: weights, as bf16 pairs (leading part + remainder), into the swizzled K-major P tiles
             const float mref = m_run == -INFINITY ? 0.f : m_run;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t g[32];
-                tmem_ld32(lane_addr + kColS + s * kT + c * 32, g);
+                tmem_ld32(lane_addr + kColS + s * kT + wg * 64 + c * 32, g);
                 tmem_ld_wait();
                 uint32_t hi[16], lo[16];
 #pragma unroll
                 for (int k = 0; k < 32; k += 2) {
-                    const float x0 = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + c * 32 + k]);
-                    const float x1 = fmaf(__uint_as_float(g[k + 1]), p.scale_log2, lc_s[s * kT + c * 32 + k + 1]);
-                    const float w0 = (j0 + c * 32 + k < vis) ? ex2(x0 - mref) : 0.f;
-                    const float w1 = (j0 + c * 32 + k + 1 < vis) ? ex2(x1 - mref) : 0.f;
+                    const float x0 = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k]);
+                    const float x1 = fmaf(__uint_as_float(g[k + 1]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k + 1]);
+                    const float w0 = (jw + c * 32 + k < vis) ? ex2(x0 - mref) : 0.f;
+                    const float w1 = (jw + c * 32 + k + 1 < vis) ? ex2(x1 - mref) : 0.f;
                     const uint32_t ph = pack2(w0, w1);
                     const uint32_t pl = pack2(w0 - bf_lo(ph), w1 - bf_hi(ph));
                     l_run += (bf_lo(ph) + bf_lo(pl)) + (bf_hi(ph) + bf_hi(pl));
                     hi[k >> 1] = ph; lo[k >> 1] = pl;
                 }
                 // 32 keys = four 16-byte chunks of this row; chunk cc of the 64-key half sits at cc ^ (row & 7)
-                const int half = c >> 1;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int cc = (c & 1) * 4 + u;
-                    const uint32_t off = half * kHalf + r * 128 + ((cc ^ (r & 7)) << 4);
+                    const int cc = c * 4 + u;
+                    const uint32_t off = wg * kHalf + r * 128 + ((cc ^ (r & 7)) << 4);
                     *reinterpret_cast<uint4*>(smem + kSmP + off) = make_uint4(hi[4 * u], hi[4 * u + 1], hi[4 * u + 2], hi[4 * u + 3]);
                     *reinterpret_cast<uint4*>(smem + kSmP + kTile + off) = make_uint4(lo[4 * u], lo[4 * u + 1], lo[4 * u + 2], lo[4 * u + 3]);
                 }
             }
             fence_before_sync();      // this thread's reads of the score buffer
-            fence_async_proxy();      // this thread's P stores, for the tensor core's reads
+            fence_async_proxy();      // this thread's P (and V) stores, for the tensor core's reads
             __syncwarp();
             if (lane == 0) { mbar_arrive(s_empty0 + 8 * s); mbar_arrive(p_full); }
         }
-        // ---- O / l -> bf16 -> global ----
+        // ---- O / l -> bf16 -> global: each thread its 64 columns; l is the sum of the row's two partial sums ----
         if (!failed && nt > 0) {
             if (!mbar_wait(p_empty, (nt - 1) & 1)) { *sh_fail = 1; failed = true; }
             fence_after_sync();
         }
-        __nv_bfloat16* orow = p.out + (size_t)(q_row0 + r) * 128;
-        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+        asm volatile("bar.sync 2, 256;\n" ::: "memory");   // nobody still reads the last tile's maxima
+        mx_s[wg * kT + r] = l_run;
+        asm volatile("bar.sync 1, 256;\n" ::: "memory");
+        const float l_row = l_run + mx_s[(wg ^ 1) * kT + r];
+        __nv_bfloat16* orow = p.out + (size_t)(q_row0 + r) * 128 + wg * 64;
+        const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < 2; ++c) {
             uint32_t o[32];
             if (nt > 0 && !failed) {
-                tmem_ld32(lane_addr + kColO + c * 32, o);
+                tmem_ld32(lane_addr + kColO + wg * 64 + c * 32, o);
                 tmem_ld_wait();
             } else {
 #pragma unroll

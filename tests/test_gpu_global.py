@@ -91,6 +91,24 @@ def test_global_clustering_extremes_and_capacity():
     compare_compressed(got, ref, K.dtype, check_assign=True)
 
 
+@pytest.mark.parametrize("n", [40, 700, 1500])
+def test_cluster_sizes_across_the_pooling_paths(n):
+    """Clusters of up to 32 members are ordered in registers, up to 1024 by repeated selection, larger ones by
+    walking the assignment array: one big cluster (everything similar to token 0 except a few strangers that
+    found their own) exercises each in turn, in both dtypes."""
+    rng = np.random.default_rng(n)
+    for dt in (torch.bfloat16, torch.float32):
+        base = rng.normal(size=128)
+        K = torch.from_numpy(base + 0.05 * rng.normal(size=(1, 2, n, 128))).float()
+        strangers = rng.choice(np.arange(1, n), size=5, replace=False)
+        K[0, :, strangers] = torch.from_numpy(rng.normal(size=(2, 5, 128))).float()
+        V = torch.from_numpy(rng.normal(size=(1, 2, n, 128))).float()
+        ref, got, status = _both(K.to(dt), V.to(dt), 0.8)
+        assert status == 0 and ref["margin"] > 1e-4
+        assert int(ref["count"][0, 0, 0]) >= n - 6
+        compare_compressed(got, ref, dt)
+
+
 def test_decode_over_globally_clustered_cores():
     w = synth.config(0, n=1500, B=1)
     ids, run_id, run_lens = synth.token_ids(w)
