@@ -388,7 +388,7 @@ def run_ours(args):
             **modes}
         line["decode_serial"] = modes["serial"]
         line["decode_independent_overlap"] = modes["independent"]
-    if args.gpus == 1:
+    if args.gpus == 1 and not args.no_append:
         line["append"] = measure_append(pipe)
     del pipe
     torch.cuda.empty_cache()
@@ -807,6 +807,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-overlap", action="store_true", help="time the step with plain stream-ordered decode launches")
     ap.add_argument("--no-modes", action="store_true", help="skip the side measurements of the other decode launch modes")
+    ap.add_argument("--no-append", action="store_true", help="skip the sc_append side measurement")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short passes over the other workloads and sweeps")
     ap.add_argument("--extras-only", action="store_true",
                     help="run only the measurements of sc_prefill_attn, the ablation arms and the budget search (a small case for profiling)")
