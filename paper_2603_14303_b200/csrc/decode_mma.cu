@@ -330,12 +330,6 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
         slab[(2 * tig + 1) * kD + d0 + 8] = o[mt][3] * f1;
     }
     __syncthreads();
-    // Nothing has been written to global memory so far.  Under an overlapped launch every write of
-    // this kernel (partials, arrival counters, out) is ordered behind the completion of the kernel
-    // before it, which ordered its own writes behind its predecessor in the same way: completion is
-    // transitive along a run of overlapped launches, and they may share workspace and out buffers.
-    // (A no-op for an ordinary launch and after the wait above.)
-    asm volatile("griddepcontrol.wait;\n" ::: "memory");
     // ---- block partial (m, l, O) into this block's shared memory, behind the warps' slabs ----
     const float* slabs = reinterpret_cast<const float*>(smem);
     float* blk = reinterpret_cast<float*>(smem) + kWarps * (8 * kD);   // [8][128] O, [8] m, [8] l
@@ -373,6 +367,12 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
     const bool direct = n_clusters == 1;   // this cluster holds the whole head: its fold is the result
     const int slice = (G * (kD / 4) + csize - 1) / csize;
     cluster.sync();
+    // Nothing has been written to global memory so far (the block partials live in shared memory).  Under
+    // an overlapped launch every global write of this kernel (out, cluster partials, arrival counters) is
+    // ordered behind the completion of the kernel before it, which ordered its own writes behind its
+    // predecessor in the same way: completion is transitive along a run of overlapped launches, and they
+    // may share workspace and out buffers.  (A no-op for an ordinary launch and after the wait above.)
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
     for (int i = threadIdx.x; i < slice; i += kWarps * 32) {
         const int e4 = crank * slice + i;
         if (e4 >= G * (kD / 4)) break;
