@@ -430,6 +430,7 @@ def measure_cell(w: synth.Workload, full_L: int, dev, sampler, peak, label: dict
         "achieved_reduction": round(1.0 / kept, 3) if kept > 0 else None,
         "decode_tokens_per_s": w.B / (us_launch * 1e-6 * full_L), "decode_bytes_per_step": dbytes / w.L * full_L,
         "decode_us_per_launch": us_launch, "decode_gbs": dgbs, "decode_frac": dgbs / peak,
+        "decode_frac_of_nominal_8tbs": dgbs / 8000.0, "compress_frac_of_nominal_8tbs": cgbs / 8000.0,
         "compress_ms_per_32k_ctx": ms_c / w.L * full_L * 32768 / (w.B * w.n), "compress_us_per_layer": ms_c * 1e3 / w.L,
         "compress_gbs": cgbs, "compress_frac": cgbs / peak})
     if raw:

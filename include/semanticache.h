@@ -317,9 +317,12 @@ SC_API sc_status sc_prefill_attn(const void* q, sc_dtype dt, int32_t B, int32_t 
  *   - a delimiter finishes the open chunk (if any) and then becomes a core of its own with
  *     count 1 and its K/V bits unchanged.
  * A finished chunk is clustered (Algorithm 1 on Eq. 2) and mean-pooled (Eq. 3) where it lies,
- * its cores replacing its first rows, with the same arithmetic as sc_compress (fp32 sums in
- * token order, one rounding); core_len grows by the number of clusters and tail_len returns
- * to 0.  The cache therefore ends up as if the generated tokens had been a second prompt.
+ * its cores replacing its first rows, with the arithmetic of sc_compress's generic kernels (Sim as
+ * the quotient of Eq. 2, fp32 sums in token order, one divide, one rounding; the fused bf16 path of
+ * sc_compress decides G > tau*|k_i|*|k_j| and multiplies by 1/|S|, so the two can differ by one unit
+ * in the last place of a core and on pairs within rounding of tau); core_len grows by the number of
+ * clusters and tail_len returns to 0.  The cache therefore ends up, within the storage type's
+ * tolerance, as if the generated tokens had been a second prompt.
  *
  *   k_new, v_new  [B, Hkv, d] contiguous, dtype dt: this layer's K/V of the new tokens
  *   token_ids     [B] int32 (device): the new token of each sequence
