@@ -657,8 +657,44 @@ def measure_append(pipe, m: int = 256, layers: int = 4):
     e1.record()
     torch.cuda.synchronize()
     b.check_status(status, "sc_append")
+    # every layer of a token in one launch (sc_append_layers): all of the workload's layers, the same stream
     med = lambda a: float(np.median(a)) if a else None
-    return {"what": "sc_append: one call per layer and generated token",
+    Lall = w.L
+    gids, gK, gV = synth.generated_stream(w, m, 0)
+    gids, gK, gV = gids.to(dev), gK.to(dev), gV.to(dev)
+    k_new = torch.zeros((w.B, w.Hkv, w.d), dtype=gK.dtype, device=dev)
+    v_new = torch.zeros_like(k_new)
+    tok = torch.zeros(w.B, **i32)
+    tails = [torch.zeros((w.B, w.Hkv), **i32) for _ in range(Lall)]
+    alens = [torch.zeros((w.B, w.Hkv), **i32) for _ in range(Lall)]
+    pipe.run_compress()        # every layer starts from its compressed prompt again (rows behind core_len are free)
+    torch.cuda.synchronize()
+    table = b.append_table([(k_new, v_new, pipe.layers[l].core_k, pipe.layers[l].core_v, pipe.layers[l].count,
+                             pipe.layers[l].core_len, tails[l], alens[l]) for l in range(Lall)])
+    gb = torch.cuda.CUDAGraph()
+    steps_b = min(m, 64)       # stays far below the free rows of every head
+    with torch.cuda.graph(gb):
+        for t in range(steps_b):
+            k_new.copy_(gK[:, :, t]); v_new.copy_(gV[:, :, t]); tok.copy_(gids[:, t])
+            b.sc_append_layers(table, k_new, tok, w.delims, w.max_chunk_len, w.tau, pipe.cap, status)
+    gb.replay()
+    torch.cuda.synchronize()
+    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2.record(); gb.replay(); e3.record()
+    torch.cuda.synchronize()
+    gc = torch.cuda.CUDAGraph()    # the three small copies alone, to take them out of the figure
+    with torch.cuda.graph(gc):
+        for t in range(steps_b):
+            k_new.copy_(gK[:, :, t]); v_new.copy_(gV[:, :, t]); tok.copy_(gids[:, t])
+    gc.replay()
+    e4, e5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e4.record(); gc.replay(); e5.record()
+    torch.cuda.synchronize()
+    b.check_status(status, "sc_append_layers")
+    batched_us = (e2.elapsed_time(e3) - e4.elapsed_time(e5)) * 1e3 / steps_b
+    return {"what": "sc_append: one call per layer and generated token; sc_append_layers: one call per generated token",
+            "all_layers_one_launch": {"layers": Lall, "us_per_token_device": batched_us,
+                                      "note": "CUDA graph of 64 tokens, the three staging copies per token timed alone and subtracted"},
             "tokens": m, "layers": layers, "us_per_call_device": e0.elapsed_time(e1) * 1e3 / len(calls),
             "calls_finishing_a_chunk_fraction": len(closing) / max(len(closing) + len(plain), 1),
             "host_bound_us_per_call_storing": med(plain), "host_bound_us_per_call_finishing_a_chunk": med(closing)}

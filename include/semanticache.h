@@ -343,6 +343,30 @@ SC_API sc_status sc_append(const void* k_new, const void* v_new, sc_dtype dt, in
                     int32_t* core_len, int32_t* tail_len, int32_t* attn_len, int32_t* status, void* stream);
 
 /*
+ * sc_append for every layer of a model in one launch (same reading, same arithmetic, same results).
+ * For loops that have the new token's K/V of all layers at hand before the caches are updated --
+ * accepting speculated tokens after verification, replaying a stored stream, a pipeline that defers
+ * cache maintenance to the end of a step -- one call per generated token replaces L of them.
+ *
+ *   layers     DEVICE array of L rows; row l holds the pointers sc_append takes for layer l
+ *              (k_new, v_new: [B, Hkv, d]; core_k, core_v, count, core_len, tail_len, attn_len as
+ *              there).  The table is read by the kernel, so it may be filled once and reused as long
+ *              as the buffers stay where they are.  Layers must not share any buffer.
+ *   L          1..65535;  all layers share dt, B, Hkv, d, cap, token_ids, the delimiter set,
+ *              max_chunk_len and tau
+ *   status     as for sc_append (first error of any layer wins)
+ */
+typedef struct {
+    const void* k_new; const void* v_new;
+    void* core_k; void* core_v; int32_t* count;
+    int32_t* core_len; int32_t* tail_len; int32_t* attn_len;
+} sc_append_layer;
+
+SC_API sc_status sc_append_layers(const sc_append_layer* layers /*DEVICE [L]*/, int32_t L, sc_dtype dt, int32_t B, int32_t Hkv,
+                           int32_t d, const int32_t* token_ids, const int32_t* delim_ids /*HOST*/, int32_t n_delim,
+                           int32_t max_chunk_len, float tau, int32_t cap, int32_t* status, void* stream);
+
+/*
  * sc_decode_attn for callers that cannot allocate device memory.  (A convenience of this
  * library; the paper has no counterpart.)
  *

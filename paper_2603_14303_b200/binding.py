@@ -25,7 +25,7 @@ _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CA
 EXPORTS = ["sc_version", "sc_launch_counter", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
            "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn",
            "sc_decode_attn_static", "sc_append", "sc_compress_budget_workspace_bytes", "sc_compress_budget",
-           "sc_compress_global_workspace_bytes", "sc_compress_global", "sc_prefill_attn"]
+           "sc_compress_global_workspace_bytes", "sc_compress_global", "sc_prefill_attn", "sc_append_layers"]
 SC_BUDGET_MAX_GRID = 65
 SC_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -90,6 +90,9 @@ def lib() -> ctypes.CDLL:
         L.sc_decode_attn.restype = _i32
         L.sc_decode_attn.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, ctypes.c_float,
                                      ctypes.c_uint32, _vp, _vp, _sz, _vp, _vp]
+        L.sc_append_layers.restype = _i32
+        L.sc_append_layers.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _vp, ctypes.POINTER(_i32), _i32, _i32,
+                                       ctypes.c_float, _i32, _vp, _vp]
         L.sc_prefill_attn.restype = _i32
         L.sc_prefill_attn.argtypes = [_vp, _i32, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _vp, ctypes.c_float,
                                       ctypes.c_uint32, _vp, _vp, _vp]
@@ -267,6 +270,28 @@ def sc_append(k_new, v_new, token_ids, delim_ids, max_chunk_len, tau, core_k, co
                            int(max_chunk_len), float(tau), _ptr(core_k), _ptr(core_v), _ptr(count), cap,
                            _ptr(core_len), _ptr(tail_len), _ptr(attn_len), _ptr(status), _stream(k_new))
     _check("sc_append", code)
+
+
+def append_table(layers) -> torch.Tensor:
+    """Device table for sc_append_layers: ``layers`` is a list of (k_new, v_new, core_k, core_v, count, core_len,
+    tail_len, attn_len) tensor tuples, one per layer.  Returns an int64 tensor [L, 8] of their addresses;
+    keep the tensors alive (and where they are) for as long as the table is used."""
+    rows = [[t.data_ptr() for t in row] for row in layers]
+    dev = layers[0][2].device
+    return torch.tensor(rows, dtype=torch.int64).to(dev)
+
+
+def sc_append_layers(table, k_new0, token_ids, delim_ids, max_chunk_len, tau, cap, status=None):
+    """Raw sc_append_layers: one generated token per sequence joins every layer's cache in one launch.
+    ``table`` from append_table; ``k_new0`` any one layer's k_new (for dtype and shape [B, Hkv, d])."""
+    _need_cuda(table, k_new0, token_ids, status)
+    B, Hkv, d = k_new0.shape
+    assert table.dtype == torch.int64 and table.dim() == 2 and table.shape[1] == 8 and table.is_contiguous()
+    delims = (_i32 * max(len(delim_ids), 1))(*[int(x) for x in delim_ids])
+    code = lib().sc_append_layers(_ptr(table), table.shape[0], _dt(k_new0), B, Hkv, d, _ptr(token_ids), delims,
+                                  len(delim_ids), int(max_chunk_len), float(tau), int(cap), _ptr(status),
+                                  _stream(k_new0))
+    _check("sc_append_layers", code)
 
 
 # ------------------------------------------------------------------------- convenience wrappers

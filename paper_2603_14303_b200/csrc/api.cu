@@ -275,4 +275,21 @@ sc_status sc_append(const void* k_new, const void* v_new, sc_dtype dt, int32_t B
     return launch_append(a, (cudaStream_t)stream) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
 
+sc_status sc_append_layers(const sc_append_layer* layers, int32_t L, sc_dtype dt, int32_t B, int32_t Hkv, int32_t d,
+                           const int32_t* token_ids, const int32_t* delim_ids, int32_t n_delim, int32_t max_chunk_len,
+                           float tau, int32_t cap, int32_t* status, void* stream) {
+    if (B < 0 || Hkv <= 0 || d <= 0 || cap < 0 || L < 0 || L > 65535) return SC_ERR_INVALID_ARG;
+    if (dt != SC_BF16 && dt != SC_F32) return SC_ERR_UNSUPPORTED;
+    if (n_delim < 0 || n_delim > SC_MAX_DELIMS || (n_delim > 0 && !delim_ids)) return SC_ERR_INVALID_ARG;
+    if (max_chunk_len < 1 || max_chunk_len > SC_MAX_CHUNK_LEN) return SC_ERR_INVALID_ARG;
+    if (!(tau == tau)) return SC_ERR_INVALID_ARG;
+    if (B == 0 || L == 0) return SC_OK;
+    if (!layers || !token_ids) return SC_ERR_INVALID_ARG;
+    AppendArgs a = {};
+    a.dt = dt; a.B = B; a.Hkv = Hkv; a.d = d; a.token_ids = token_ids;
+    for (int i = 0; i < n_delim; ++i) a.delim[i] = delim_ids[i];
+    a.n_delim = n_delim; a.max_chunk_len = max_chunk_len; a.tau = tau; a.cap = cap; a.status = status;
+    return launch_append_layers(a, layers, L, (cudaStream_t)stream) == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
 }  // extern "C"

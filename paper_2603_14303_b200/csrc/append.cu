@@ -20,8 +20,16 @@ constexpr int kAppendThreads = 256;
 constexpr int kAppendWarps = kAppendThreads / 32;
 constexpr int kWords = SC_MAX_CHUNK_LEN / 32;
 
+// The pointers of one layer, as sc_append_layers reads them from its device table.
+struct LayerPtrs {
+    const void* k_new; const void* v_new; void* core_k; void* core_v; int32_t* count;
+    int32_t* core_len; int32_t* tail_len; int32_t* attn_len;
+};
+
+// One block = one (sequence, KV head) of one layer.  `a` carries the sizes, the delimiter set, tau and the
+// token ids (its own pointers are not used), `p` the layer's buffers.
 template <typename T>
-__global__ void __launch_bounds__(kAppendThreads) append_kernel(const AppendArgs a) {
+__device__ __forceinline__ void append_block(const AppendArgs& a, const LayerPtrs& p) {
     __shared__ float norms[SC_MAX_CHUNK_LEN];
     __shared__ uint32_t assigned[kWords];                    // tokens of the tail that have a cluster
     __shared__ uint32_t members[SC_MAX_CHUNK_LEN][kWords];   // row c: the tokens of cluster c
@@ -29,13 +37,13 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(const AppendArgs
     const int bh = blockIdx.x, b = bh / a.Hkv;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int d = a.d;
-    T* ck = static_cast<T*>(a.core_k) + (int64_t)bh * a.cap * d;
-    T* cv = static_cast<T*>(a.core_v) + (int64_t)bh * a.cap * d;
-    int32_t* cnt = a.count + (int64_t)bh * a.cap;
-    const T* kn = static_cast<const T*>(a.k_new) + (int64_t)bh * d;
-    const T* vn = static_cast<const T*>(a.v_new) + (int64_t)bh * d;
+    T* ck = static_cast<T*>(p.core_k) + (int64_t)bh * a.cap * d;
+    T* cv = static_cast<T*>(p.core_v) + (int64_t)bh * a.cap * d;
+    int32_t* cnt = p.count + (int64_t)bh * a.cap;
+    const T* kn = static_cast<const T*>(p.k_new) + (int64_t)bh * d;
+    const T* vn = static_cast<const T*>(p.v_new) + (int64_t)bh * d;
 
-    int cl = a.core_len[bh], tl = a.tail_len[bh];
+    int cl = p.core_len[bh], tl = p.tail_len[bh];
     const int tok = a.token_ids[b];
     bool is_delim = false;
     for (int i = 0; i < a.n_delim; ++i) is_delim |= (a.delim[i] == tok);
@@ -43,7 +51,7 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(const AppendArgs
     if (cl < 0 || tl < 0 || tl >= a.max_chunk_len || cl + tl >= a.cap) {   // no room (or a corrupt state): leave it as it is
         if (tid == 0) {
             set_status(a.status, (cl + tl >= a.cap && cl >= 0 && tl >= 0) ? SC_ERR_CAPACITY : SC_ERR_INVALID_ARG);
-            a.attn_len[bh] = max(0, min(cl + tl, a.cap));
+            p.attn_len[bh] = max(0, min(cl + tl, a.cap));
         }
         return;
     }
@@ -138,13 +146,41 @@ __global__ void __launch_bounds__(kAppendThreads) append_kernel(const AppendArgs
         ++cl;
     }
     if (tid == 0) {
-        a.core_len[bh] = cl;
-        a.tail_len[bh] = tl;
-        a.attn_len[bh] = cl + tl;
+        p.core_len[bh] = cl;
+        p.tail_len[bh] = tl;
+        p.attn_len[bh] = cl + tl;
     }
 }
 
+template <typename T>
+__global__ void __launch_bounds__(kAppendThreads) append_kernel(const AppendArgs a) {
+    LayerPtrs p;
+    p.k_new = a.k_new; p.v_new = a.v_new; p.core_k = a.core_k; p.core_v = a.core_v; p.count = a.count;
+    p.core_len = a.core_len; p.tail_len = a.tail_len; p.attn_len = a.attn_len;
+    append_block<T>(a, p);
+}
+
+// Every layer of one generated token in one launch: blockIdx.y picks the layer's row of the table.
+template <typename T>
+__global__ void __launch_bounds__(kAppendThreads) append_layers_kernel(const AppendArgs a, const sc_append_layer* __restrict__ table) {
+    const sc_append_layer t = table[blockIdx.y];
+    LayerPtrs p;
+    p.k_new = t.k_new; p.v_new = t.v_new; p.core_k = t.core_k; p.core_v = t.core_v; p.count = t.count;
+    p.core_len = t.core_len; p.tail_len = t.tail_len; p.attn_len = t.attn_len;
+    append_block<T>(a, p);
+}
+
 }  // namespace
+
+cudaError_t launch_append_layers(const AppendArgs& a, const sc_append_layer* table, int32_t L, cudaStream_t st) {
+    const int blocks = a.B * a.Hkv;
+    if (blocks == 0 || L == 0) return cudaSuccess;
+    const dim3 grid(blocks, L);
+    if (a.dt == SC_BF16) append_layers_kernel<__nv_bfloat16><<<grid, kAppendThreads, 0, st>>>(a, table);
+    else append_layers_kernel<float><<<grid, kAppendThreads, 0, st>>>(a, table);
+    note_launches(1);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t st) {
     const int blocks = a.B * a.Hkv;

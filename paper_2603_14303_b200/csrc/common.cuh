@@ -130,5 +130,6 @@ struct AppendArgs {
     int32_t* core_len; int32_t* tail_len; int32_t* attn_len; int32_t* status;
 };
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t st);
+cudaError_t launch_append_layers(const AppendArgs& a, const sc_append_layer* table, int32_t L, cudaStream_t st);
 
 }  // namespace sc

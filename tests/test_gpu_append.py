@@ -161,3 +161,41 @@ def test_append_refuses_lengths_that_cannot_be_its_own_state():
                       0.7, both.ck, both.cv, both.cnt, both.clen, both.tlen, both.alen, both.status)
     assert int(both.status.item()) == binding.SC_ERR_INVALID_ARG
     assert int(both.clen.abs().max()) == 0 and (both.tlen == 5).all() and int(both.cnt.abs().max()) == 0
+
+
+@pytest.mark.parametrize("dtype,d", [(torch.bfloat16, 128), (torch.float32, 64)])
+def test_all_layers_in_one_launch_equal_one_launch_per_layer(dtype, d):
+    """sc_append_layers: every layer of a generated token in one launch.  Each layer has its own keys and
+    values (so chunks cluster differently per layer); after every token the batched caches must equal, bit
+    for bit, caches maintained by one sc_append per layer, and layer 0 must match the oracle's state."""
+    B, Hkv, m, L, max_len = 2, 2, 160, 3, 24
+    streams = [_stream(40 + l, B, Hkv, m, d, 0.07, dtype) for l in range(L)]
+    ids = streams[0][0]                       # the token ids are the model's, the same for every layer
+    single = [Both(B, Hkv, m, d, dtype) for _ in range(L)]
+    batched = [Both(B, Hkv, m, d, dtype) for _ in range(L)]
+    k_new = [torch.zeros((B, Hkv, d), dtype=dtype, device=DEV) for _ in range(L)]
+    v_new = [torch.zeros((B, Hkv, d), dtype=dtype, device=DEV) for _ in range(L)]
+    table = binding.append_table([(k_new[l], v_new[l], x.ck, x.cv, x.cnt, x.clen, x.tlen, x.alen)
+                                  for l, x in enumerate(batched)])
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    tok = torch.zeros(B, dtype=torch.int32, device=DEV)
+    for t in range(m):
+        for l in range(L):
+            single[l].step(ids[:, t], streams[l][1][:, :, t], streams[l][2][:, :, t], 0.7, max_len)
+            k_new[l].copy_(streams[l][1][:, :, t])
+            v_new[l].copy_(streams[l][2][:, :, t])
+        tok.copy_(ids[:, t])
+        binding.sc_append_layers(table, k_new[0], tok, DELIM, max_len, 0.7, m, status)
+        if t % 40 == 39 or t == m - 1:
+            binding.check_status(status, "sc_append_layers")
+            for l in range(L):
+                a, b = single[l], batched[l]
+                for x, y in ((a.clen, b.clen), (a.tlen, b.tlen), (a.alen, b.alen), (a.cnt, b.cnt), (a.ck, b.ck), (a.cv, b.cv)):
+                    assert torch.equal(x, y), f"layer {l}, token {t}"
+    single[0].compare("layer 0 after the stream")
+    # a full cache in one layer is reported and leaves that layer alone
+    batched[1].clen.fill_(m)
+    batched[1].tlen.zero_()
+    before = batched[1].ck.clone()
+    binding.sc_append_layers(table, k_new[0], tok, DELIM, max_len, 0.7, m, status)
+    assert int(status.item()) == binding.SC_ERR_CAPACITY and torch.equal(before, batched[1].ck)
