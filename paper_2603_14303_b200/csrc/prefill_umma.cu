@@ -4,16 +4,18 @@
 // step this is a dense contraction: the G query heads that share a KV head times the m queries give
 // G*m rows against the same cores, so it runs on the tcgen05 tensor cores (bf16, d = 128):
 //   one CTA = 128 query rows of one (sequence, KV head), walking the head's cores 128 at a time;
-//   warp 0     TMA: the query tile once, then K and V tiles into a two-stage ring (128-byte swizzle);
-//   warp 1     issues the MMAs: S = Q K^T into one of two score buffers in tensor memory (so the next
-//              tile's scores are computed while this tile's are being exponentiated), then O += P V,
-//              V read as an MN-major operand straight from its [keys x dims] tile;
+//   warp 0     TMA: the query tile once, then K and V tiles into a three-stage ring (128-byte swizzle);
+//   warp 1     issues the MMAs: S = Q K^T into one of two score buffers in tensor memory (two tiles ahead
+//              of the weighted sum), then O += P V with P read from tensor memory and V as an MN-major
+//              operand straight from its [keys x dims] tile;
 //   warps 2-9  softmax, two threads per query row (= tensor-memory lane; each owns half of a tile's keys and
 //              half of the accumulator's columns, the row maximum is exchanged through shared memory):
 //              x = S * scale*log2(e) + log2(count), masks (head length, optional causal tail), running
 //              maximum raised lazily (the accumulator row is rescaled in tensor memory only then),
-//              P = 2^(x - m) written to shared memory as a bf16 pair (leading part + remainder) in
-//              the swizzled K-major layout the second MMA reads; finally O / l -> bf16 -> global.
+//              P = 2^(x - m) as a bf16 pair (leading part + remainder) written back over the scores it
+//              came from: the 32 fp32 columns of a chunk of scores become 16 columns of packed leading
+//              parts and 16 of remainders, so P is double-buffered like S and never touches shared
+//              memory; finally O / l -> bf16 -> global.
 // Every wait is bounded; a wait that gives up is reported through the status word.
 // A CUDA-core kernel (one warp per query) serves other dtypes and head sizes.
 #include "common.cuh"
@@ -29,9 +31,10 @@ constexpr int kT = 128;                       // query rows per CTA, keys per ti
 constexpr int kHalf = kT * 128;               // 16384 bytes: one 64-column half of a [128 x 128] bf16 tile
 constexpr int kTile = 2 * kHalf;              // 32768
 constexpr int kThreads = 320;                 // warp 0: TMA, warp 1: MMA + tensor memory, warps 2-9: softmax
-constexpr int kTmemCols = 512;                // S0 | S1 | O (128 columns each), rounded up to a power of two
+constexpr int kTmemCols = 512;                // S0 | S1 | O (128 columns each; P overwrites S in place), rounded up to a power of two
 constexpr int kColS = 0, kColO = 256;
-constexpr int kSmQ = 0, kSmK = kTile, kSmV = 3 * kTile, kSmP = 5 * kTile, kSmLc = 7 * kTile, kSmMx = kSmLc + 2 * kT * 4,
+constexpr int kStages = 3;                    // K/V ring
+constexpr int kSmQ = 0, kSmK = kTile, kSmV = (1 + kStages) * kTile, kSmLc = (1 + 2 * kStages) * kTile, kSmMx = kSmLc + 2 * kT * 4,
               kSmBar = kSmMx + 2 * kT * 4;
 constexpr int kSmemBytes = kSmBar + 256;
 constexpr float kMaxSlack = 8.f;              // log2 units a score may exceed the running maximum before it is raised
@@ -59,6 +62,20 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]: A's rows are tensor-memory lanes, two 16-bit elements of the contraction
+// axis per 32-bit column; one thread issues.
+__device__ __forceinline__ void mma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+                 ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -83,28 +100,29 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
     float* lc_s = reinterpret_cast<float*>(smem + kSmLc);     // [2][128] log2(count) of the tile's keys
     float* mx_s = reinterpret_cast<float*>(smem + kSmMx);     // [2][128] each half's row maximum (at the end the row sums)
     const uint32_t bar0 = sbase + kSmBar;
-    const uint32_t q_full = bar0, kv_full0 = bar0 + 8, kv_empty0 = bar0 + 24, s_full0 = bar0 + 40, s_empty0 = bar0 + 56,
-                   p_full = bar0 + 72, p_empty = bar0 + 80;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kSmBar + 96);
-    volatile int* sh_fail = reinterpret_cast<volatile int*>(smem + kSmBar + 100);
-    volatile int* sh_fail_sm = reinterpret_cast<volatile int*>(smem + kSmBar + 104);   // set by the softmax warps only
-    volatile int* sh_issued = reinterpret_cast<volatile int*>(smem + kSmBar + 108);
+    const uint32_t q_full = bar0, kv_full0 = bar0 + 8, kv_empty0 = bar0 + 32, s_full0 = bar0 + 56, p_full0 = bar0 + 72,
+                   pv_done0 = bar0 + 88;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kSmBar + 104);
+    volatile int* sh_fail = reinterpret_cast<volatile int*>(smem + kSmBar + 108);
+    volatile int* sh_fail_sm = reinterpret_cast<volatile int*>(smem + kSmBar + 112);   // set by the softmax warps only
+    volatile int* sh_issued = reinterpret_cast<volatile int*>(smem + kSmBar + 116);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
         mbar_init(q_full, 1);
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             mbar_init(kv_full0 + 8 * s, 1);
             mbar_init(kv_empty0 + 8 * s, 1);
-            mbar_init(s_full0 + 8 * s, 1);
-            mbar_init(s_empty0 + 8 * s, 8);
         }
-        mbar_init(p_full, 8);
-        mbar_init(p_empty, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(s_full0 + 8 * s, 1);
+            mbar_init(p_full0 + 8 * s, 8);
+            mbar_init(pv_done0 + 8 * s, 1);
+        }
         mbar_fence_init();
         *sh_fail = 0; *sh_fail_sm = 0; *sh_issued = 0;
     }
-    if (warp == 1) tmem_alloc(sbase + kSmBar + 96, kTmemCols);
+    if (warp == 1) tmem_alloc(sbase + kSmBar + 104, kTmemCols);
     fence_before_sync();
     __syncthreads();
     fence_after_sync();
@@ -117,8 +135,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
             tma_load_4d(sbase + kSmQ + kHalf, &p.map_q, 64, (int)q_row0, 0, 0, q_full);
             const int row_base = bh * p.cap;
             for (int t = 0; t < nt; ++t) {
-                const int s = t & 1;
-                if (t >= 2 && !mbar_wait(kv_empty0 + 8 * s, ((t >> 1) - 1) & 1)) { *sh_fail = 1; break; }
+                const int s = t % kStages;
+                if (t >= kStages && !mbar_wait(kv_empty0 + 8 * s, ((t / kStages) - 1) & 1)) { *sh_fail = 1; break; }
                 mbar_expect_tx(kv_full0 + 8 * s, 2 * kTile);
                 const uint32_t dk = sbase + kSmK + s * kTile, dv = sbase + kSmV + s * kTile;
                 tma_load_4d(dk, &p.map_k, 0, row_base + t * kT, 0, 0, kv_full0 + 8 * s);
@@ -131,44 +149,47 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
     } else if (warp == 1) {
         if (lane == 0 && nt > 0) {   // ---- MMA issuer ----
             constexpr uint32_t idesc_qk = instr_desc_bf16(kT, kT, false, false);   // Q and K both K-major
-            constexpr uint32_t idesc_pv = instr_desc_bf16(kT, kT, false, true);    // P K-major, V MN-major
+            constexpr uint32_t idesc_pv = instr_desc_bf16(kT, kT, false, true);    // P K-major (tensor memory), V MN-major
             const uint32_t aq = sbase + kSmQ;
-            auto issue_qk = [&](int t) {
-                const int s = t & 1;
-                const uint32_t bk = sbase + kSmK + s * kTile;
+            auto issue_qk = [&](int t) {   // S[t & 1] = Q K_t^T
+                const uint32_t bk = sbase + kSmK + (t % kStages) * kTile;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint32_t off = (ks >> 2) * kHalf + (ks & 3) * 32;
-                    mma_bf16_ss(tmem + kColS + s * kT, smem_desc_sw128(aq + off, 16, 1024), smem_desc_sw128(bk + off, 16, 1024),
+                    mma_bf16_ss(tmem + kColS + (t & 1) * kT, smem_desc_sw128(aq + off, 16, 1024), smem_desc_sw128(bk + off, 16, 1024),
                                 idesc_qk, ks > 0);
                 }
-                mma_commit(s_full0 + 8 * s);
+                mma_commit(s_full0 + 8 * (t & 1));
             };
             bool ok = mbar_wait(q_full, 0) && mbar_wait(kv_full0, 0);
             if (ok) { fence_after_sync(); issue_qk(0); }
+            if (ok && nt > 1) {
+                ok = mbar_wait(kv_full0 + 8, 0);
+                if (ok) { fence_after_sync(); issue_qk(1); }
+            }
             for (int t = 0; t < nt && ok; ++t) {
-                const int s = t & 1;
-                if (t + 1 < nt) {   // next tile's scores, into the other buffer
-                    const int s1 = (t + 1) & 1;
-                    ok = mbar_wait(kv_full0 + 8 * s1, ((t + 1) >> 1) & 1);
-                    if (ok && t + 1 >= 2) ok = mbar_wait(s_empty0 + 8 * s1, (((t + 1) >> 1) - 1) & 1);
-                    if (!ok) break;
-                    fence_after_sync();
-                    issue_qk(t + 1);
-                }
-                ok = mbar_wait(p_full, t & 1);
+                const int sb = t & 1;
+                ok = mbar_wait(p_full0 + 8 * sb, (t >> 1) & 1);   // the weights of tile t are in tensor memory
                 if (!ok) break;
                 fence_after_sync();
-                const uint32_t bv = sbase + kSmV + s * kTile;
+                const uint32_t bv = sbase + kSmV + (t % kStages) * kTile;
+                const uint32_t pcol = tmem + kColS + sb * kT;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {   // sixteen keys per instruction
-                    const uint32_t offp = (ks >> 2) * kHalf + (ks & 3) * 32;            // P: K-major, keys along the row
+                for (int ks = 0; ks < 8; ++ks) {   // sixteen keys per instruction: eight packed columns of P
                     const uint64_t vdesc = smem_desc_sw128(bv + ks * 16 * 128, kHalf, 1024);   // V: MN-major, 16 key rows down
-                    mma_bf16_ss(tmem + kColO, smem_desc_sw128(sbase + kSmP + offp, 16, 1024), vdesc, idesc_pv, t > 0 || ks > 0);
-                    mma_bf16_ss(tmem + kColO, smem_desc_sw128(sbase + kSmP + kTile + offp, 16, 1024), vdesc, idesc_pv, true);
+                    const uint32_t pa = pcol + (ks >> 1) * 32 + (ks & 1) * 8;                  // leading parts; remainders 16 columns on
+                    mma_bf16_ts(tmem + kColO, pa, vdesc, idesc_pv, t > 0 || ks > 0);
+                    mma_bf16_ts(tmem + kColO, pa + 16, vdesc, idesc_pv, true);
                 }
-                mma_commit(kv_empty0 + 8 * s);   // K and V of this stage are spent
-                mma_commit(p_empty);             // P may be overwritten, O may be read
+                mma_commit(kv_empty0 + 8 * (t % kStages));   // K and V of this stage are spent
+                mma_commit(pv_done0 + 8 * sb);               // P of this buffer is spent, O holds tile t
+                if (t + 2 < nt) {   // the scores two tiles ahead go where this tile's scores and weights were
+                    ok = mbar_wait(kv_full0 + 8 * ((t + 2) % kStages), ((t + 2) / kStages) & 1) &&
+                         mbar_wait(pv_done0 + 8 * sb, (t >> 1) & 1);
+                    if (!ok) break;
+                    fence_after_sync();
+                    issue_qk(t + 2);
+                }
             }
             if (!ok) *sh_fail = 1;
         }
@@ -185,7 +206,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
         float m_run = -INFINITY, l_run = 0.f;                 // l_run: this thread's keys only
         bool failed = false;
         for (int t = 0; t < nt; ++t) {
-            const int s = t & 1, j0 = t * kT, jw = j0 + wg * 64;   // jw: first key of this thread's half
+            const int s = t & 1, st = t % kStages, j0 = t * kT, jw = j0 + wg * 64;   // jw: first key of this thread's half
             if (wg == 0) lc_s[s * kT + r] = (cnt != nullptr && j0 + r < len) ? lg2((float)max(cnt[j0 + r], 1)) : 0.f;
             if (!mbar_wait(s_full0 + 8 * s, (t >> 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
             fence_after_sync();
@@ -196,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
             if (j0 + r >= len) {
 #pragma unroll
                 for (int u = 0; u < 8; ++u)
-                    *reinterpret_cast<uint4*>(smem + kSmV + s * kTile + wg * kHalf + r * 128 + u * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    *reinterpret_cast<uint4*>(smem + kSmV + st * kTile + wg * kHalf + r * 128 + u * 16) = make_uint4(0u, 0u, 0u, 0u);
             }
             // pass 1: the row's largest score in this tile (each thread its half, then the two are exchanged)
             float mx = -INFINITY;
@@ -212,14 +233,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
                 }
             }
             mx_s[wg * kT + r] = mx;
-            // P and O belong to the previous tile's second product until it is complete
-            if (t > 0 && !mbar_wait(p_empty, (t - 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
-            fence_after_sync();
             asm volatile("bar.sync 2, 256;\n" ::: "memory");   // both halves' maxima are in place
             mx = fmaxf(mx, mx_s[(wg ^ 1) * kT + r]);
             const bool raise = mx > m_run + kMaxSlack;      // also the first finite score (m_run = -inf); same in both threads
             if (__any_sync(kFull, raise)) {
                 const float f = raise ? ex2(m_run - mx) : 1.f;   // 0 when nothing had been seen
+                // the accumulator may be touched only between two weighted sums: the previous one must be complete
+                // (this tile's cannot start before this warp has handed in its weights)
+                if (t > 0 && !mbar_wait(pv_done0 + 8 * ((t - 1) & 1), ((t - 1) >> 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
+                fence_after_sync();
                 if (t > 0) {
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
@@ -235,7 +257,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
                 l_run *= f;
                 if (raise) m_run = mx;
             }
-            // pass 2: weights, as bf16 pairs (leading part + remainder), into the swizzled K-major P tiles
+            // pass 2: weights, as bf16 pairs (leading part + remainder), back into the score buffer's columns
             const float mref = m_run == -INFINITY ? 0.f : m_run;
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -254,23 +276,19 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
                     l_run += (bf_lo(ph) + bf_lo(pl)) + (bf_hi(ph) + bf_hi(pl));
                     hi[k >> 1] = ph; lo[k >> 1] = pl;
                 }
-                // 32 keys = four 16-byte chunks of this row; chunk cc of the 64-key half sits at cc ^ (row & 7)
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int cc = c * 4 + u;
-                    const uint32_t off = wg * kHalf + r * 128 + ((cc ^ (r & 7)) << 4);
-                    *reinterpret_cast<uint4*>(smem + kSmP + off) = make_uint4(hi[4 * u], hi[4 * u + 1], hi[4 * u + 2], hi[4 * u + 3]);
-                    *reinterpret_cast<uint4*>(smem + kSmP + kTile + off) = make_uint4(lo[4 * u], lo[4 * u + 1], lo[4 * u + 2], lo[4 * u + 3]);
-                }
+                // the 32 score columns just read become 16 columns of packed leading parts and 16 of remainders
+                tmem_st16(lane_addr + kColS + s * kT + wg * 64 + c * 32, hi);
+                tmem_st16(lane_addr + kColS + s * kT + wg * 64 + c * 32 + 16, lo);
             }
-            fence_before_sync();      // this thread's reads of the score buffer
-            fence_async_proxy();      // this thread's P (and V) stores, for the tensor core's reads
+            tmem_st_wait();
+            fence_before_sync();      // this thread's accesses to tensor memory
+            fence_async_proxy();      // a cleared V row, for the tensor core's reads
             __syncwarp();
-            if (lane == 0) { mbar_arrive(s_empty0 + 8 * s); mbar_arrive(p_full); }
+            if (lane == 0) mbar_arrive(p_full0 + 8 * s);
         }
         // ---- O / l -> bf16 -> global: each thread its 64 columns; l is the sum of the row's two partial sums ----
         if (!failed && nt > 0) {
-            if (!mbar_wait(p_empty, (nt - 1) & 1)) { *sh_fail = 1; failed = true; }
+            if (!mbar_wait(pv_done0 + 8 * ((nt - 1) & 1), ((nt - 1) >> 1) & 1)) { *sh_fail = 1; failed = true; }
             fence_after_sync();
         }
         asm volatile("bar.sync 2, 256;\n" ::: "memory");   // nobody still reads the last tile's maxima
@@ -308,7 +326,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
             set_status(p.status, SC_ERR_TIMEOUT);
             const int issued = *sh_issued;
             if (nt > 0) mbar_wait(q_full, 0);
-            for (int t = max(issued - 2, 0); t < issued; ++t) mbar_wait(kv_full0 + 8 * (t & 1), (t >> 1) & 1);
+            for (int t = max(issued - kStages, 0); t < issued; ++t) mbar_wait(kv_full0 + 8 * (t % kStages), (t / kStages) & 1);
         }
         __syncthreads();
     }
