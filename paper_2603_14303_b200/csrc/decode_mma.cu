@@ -192,9 +192,9 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
         soff[i] = r * kRowBytes + ((c ^ (r & 7)) << 4);
     }
 
-    // prologue: fill the ring
+    // prologue: fill the whole ring (under a chained launch this is what is in shared memory when the wait ends)
 #pragma unroll
-    for (int s = 0; s < kStages - 1; ++s) {
+    for (int s = 0; s < kStages; ++s) {
         if (s < my_tiles) issue_tile(wbase + s * kStageBytes, kh, vh, ch, (t0 + warp + s * kWarps) * kTile, len, lane, soff);
         cp_async_commit();
     }
@@ -226,11 +226,7 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
     const int v_row = lm_r + ((lm_j >> 1) << 3), v_csel = lm_j & 1;    // V^T: (r0-7,c), (r0-7,c+1), (r8-15,c), (r8-15,c+1)
 
     for (int i = 0; i < my_tiles; ++i) {
-        const int pre = i + kStages - 1;
-        if (pre < my_tiles)
-            issue_tile(wbase + (pre % kStages) * kStageBytes, kh, vh, ch, (t0 + warp + pre * kWarps) * kTile, len, lane, soff);
-        cp_async_commit();
-        cp_async_wait<kStages - 1>();
+        cp_async_wait<kStages - 1>();   // tile i has landed; tiles i+1, i+2 are on their way
         __syncwarp();
 
         const uint32_t st = wbase + (i % kStages) * kStageBytes;
@@ -300,6 +296,11 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
             mma_bf16(o[mt], a0, a1, a2, a3, rb0, rb1);
         }
         __syncwarp();
+        // the stage just consumed takes the tile three ahead
+        const int nxt = i + kStages;
+        if (nxt < my_tiles)
+            issue_tile(wbase + (i % kStages) * kStageBytes, kh, vh, ch, (t0 + warp + nxt * kWarps) * kTile, len, lane, soff);
+        cp_async_commit();
     }
     cp_async_wait<0>();
 
