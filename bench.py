@@ -164,6 +164,9 @@ class Pipeline:
         self.cstatus = torch.zeros((w.L, 1), **i32)
         self.launches_compress = 0
         self.g_compress = None
+        self.g_compress_per_layer = None
+        self.lws = None
+        self.one_launch = False
         self.g_decode, self.launches_decode = {}, {}
         # exact attention over the raw cache with the same kernel (count = NULL, every head n rows long)
         self.raw = None
@@ -173,7 +176,8 @@ class Pipeline:
             self.raw = True
 
     # the launch sequences (also what the graphs capture)
-    def run_compress(self):
+    def run_compress(self, one_launch: bool = False):
+        """sc_chunk, then the compress stage: one sc_compress per layer, or every layer in one sc_compress_layers."""
         b, w = self.b, self.w
         if self.plan is None:
             self.plan = b.chunk(self.ids_dev, w.delims, w.max_chunk_len)
@@ -182,6 +186,11 @@ class Pipeline:
             p = self.plan
             b.sc_chunk(self.ids_dev, w.delims, w.max_chunk_len, p.seg_off, p.seq_seg_off, p.n_seg, p.tile_seg,
                        p.seq_tile_cnt, self._chunk_ws, p.status)
+        if one_launch:
+            if self.lws is None:
+                self.lws = b.compress_layers_workspace(w.L, w.B, w.Hkv, w.n, self.dev)
+            b.sc_compress_layers(self.K, self.V, self.plan, w.tau, self.layers, self.lws, self.cstatus[0], 0)
+            return
         for l in range(w.L):
             ly = self.layers[l]
             b.sc_compress(self.K[l], self.V[l], self.plan, w.tau, ly.core_k, ly.core_v, ly.count, ly.core_len, None,
@@ -202,10 +211,14 @@ class Pipeline:
                     b.decode_attn(q, self.layers[l], out=self.out[s, l], workspace=self.dws[l],
                                   status=self.status[l], flags=fl)
 
-    def capture(self, modes=("chain",), short_steps: int | None = None):
+    def capture(self, modes=("chain",), short_steps: int | None = None, one_launch: bool = False):
         """Warm-up pass, then one graph for the compress stage and one per decode mode.  The first mode
-        is captured with all decode steps; the others with ``short_steps`` (they are side measurements)."""
+        is captured with all decode steps; the others with ``short_steps`` (they are side measurements).
+        ``one_launch``: the timed compress stage is sc_compress_layers; the per-layer form gets a graph of its own."""
+        self.one_launch = one_launch
         self.run_compress()   # allocates the plan outside capture
+        if one_launch:
+            self.run_compress(True)
         torch.cuda.synchronize(self.dev)
         self.b.check_status(self.plan.status, "warm-up pass")
         if int(self.cstatus.abs().max().item()) != 0:
@@ -213,8 +226,12 @@ class Pipeline:
         c0 = self.b.launch_counter()
         self.g_compress = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.g_compress):
-            self.run_compress()
+            self.run_compress(one_launch)
         self.launches_compress = self.b.launch_counter() - c0
+        if one_launch:
+            self.g_compress_per_layer = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self.g_compress_per_layer):
+                self.run_compress(False)
         self.steps_of = {}
         for i, mode in enumerate(modes):
             steps = self.w.decode_steps if (i == 0 or not short_steps) else min(short_steps, self.w.decode_steps)
@@ -289,7 +306,8 @@ def run_ours(args):
     pipe = Pipeline(w, dev)
     main_mode = "serial" if args.no_overlap else "chain"
     side_modes = [m for m in DECODE_MODES if m != main_mode] if (args.gpus == 1 and not args.no_modes) else []
-    pipe.capture([main_mode] + side_modes, short_steps=max(8, min(32, w.decode_steps // 8)))
+    one_launch = (not args.per_layer_compress) and w.L <= binding.SC_MAX_LAYERS_PER_CALL
+    pipe.capture([main_mode] + side_modes, short_steps=max(8, min(32, w.decode_steps // 8)), one_launch=one_launch)
     cbytes, dbytes, per_layer, kept = pipe.algorithmic_bytes()
     g_decode = pipe.g_decode[main_mode]
 
@@ -352,6 +370,7 @@ def run_ours(args):
         "config": {"workload": w.name, "B": w.B, "n_ctx": w.n, "layers": w.L, "kv_heads": w.Hkv, "q_heads": w.Hq,
                    "head_dim": w.d, "tau": w.tau, "decode_steps": w.decode_steps, "kept_fraction": round(kept, 4),
                    "l2": "inputs larger than L2 (every step streams all layers)", "launch": launch_text,
+                   "compress_launch": "one sc_compress_layers for all layers" if one_launch else "one sc_compress per layer",
                    "parallelism": f"replicas x{args.gpus}" if distributed else "single gpu"},
         "decode_tokens_per_s": w.B * w.decode_steps * args.gpus / (sum_d / args.steps * 1e-3),
         "decode_bytes_per_step": dbytes,
@@ -364,11 +383,13 @@ def run_ours(args):
                      "us_per_launch": dec_launch_us,
                      "traffic": args.traffic if args.traffic is not None else recorded_traffic(w.name, "decode"),
                      "traffic_source": "ncu capture recorded under profiles/ (not this run); null once the kernel source changed"},
-        "roofline_compress": {"kernel": "sc_compress (one layer per launch)", "bound": "hbm", "achieved": comp_gbs,
+        "roofline_compress": {"kernel": "sc_compress_layers (every layer in one launch, as at the end of a prefill)" if one_launch
+                              else "sc_compress (one layer per launch)", "bound": "hbm", "achieved": comp_gbs,
                               "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": comp_gbs / peak,
-                              "frac_of_nominal_8tbs": comp_gbs / 8000.0, "bytes_per_launch": cbytes / w.L,
-                              "us_per_launch": comp_ms * 1e3 / w.L,
-                              "traffic": recorded_traffic(w.name, "compress")},
+                              "frac_of_nominal_8tbs": comp_gbs / 8000.0, "bytes_per_launch": cbytes / (1 if one_launch else w.L),
+                              "us_per_launch": comp_ms * 1e3 / (1 if one_launch else w.L), "us_per_layer": comp_ms * 1e3 / w.L,
+                              "launches_per_step": 1 if one_launch else w.L,
+                              "traffic": recorded_traffic(w.name, "compress_layers" if one_launch else "compress")},
         "gpu_launches": args.steps * (pipe.launches_compress + pipe.launches_decode[main_mode]),
         "gpu_launches_per_step": {"chunk+compress": pipe.launches_compress, "decode": pipe.launches_decode[main_mode]},
         "clocks": clocks, "e2e": e2e, "wall_s": t_wall,
@@ -388,6 +409,17 @@ def run_ours(args):
             **modes}
         line["decode_serial"] = modes["serial"]
         line["decode_independent_overlap"] = modes["independent"]
+    if one_launch and args.gpus == 1:
+        # the same stage as one sc_compress per layer (the per-layer call of the scope table), graph alone
+        ms_p = pipe.time_graph(pipe.g_compress_per_layer, 5)
+        gbs_p = cbytes / (ms_p * 1e-3) / 1e9
+        line["roofline_compress_per_layer_calls"] = {
+            "kernel": "sc_compress (one layer per launch)", "bound": "hbm", "achieved": gbs_p, "peak": peak, "peak_kind": peak_kind,
+            "unit": "GB/s", "frac": gbs_p / peak, "frac_of_nominal_8tbs": gbs_p / 8000.0, "bytes_per_launch": cbytes / w.L,
+            "us_per_launch": ms_p * 1e3 / w.L, "ms_per_32k_ctx": ms_p * 32768 / (w.B * w.n),
+            "traffic": recorded_traffic(w.name, "compress")}
+        if int(pipe.cstatus.abs().max().item()) != 0:
+            raise RuntimeError("sc_compress reported a device-side error")
     if args.gpus == 1 and not args.no_append:
         line["append"] = measure_append(pipe)
     del pipe
@@ -845,6 +877,8 @@ def main():
     ap.add_argument("--no-overlap", action="store_true", help="time the step with plain stream-ordered decode launches")
     ap.add_argument("--no-modes", action="store_true", help="skip the side measurements of the other decode launch modes")
     ap.add_argument("--no-append", action="store_true", help="skip the sc_append side measurement")
+    ap.add_argument("--per-layer-compress", action="store_true",
+                    help="time the step with one sc_compress per layer instead of one sc_compress_layers for all")
     ap.add_argument("--no-sweep", action="store_true", help="skip the short passes over the other workloads and sweeps")
     ap.add_argument("--extras-only", action="store_true",
                     help="run only the measurements of sc_prefill_attn, the ablation arms and the budget search (a small case for profiling)")

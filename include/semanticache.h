@@ -180,6 +180,37 @@ SC_API sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides
                       int32_t* status, void* stream);
 
 /*
+ * sc_compress for several layers of a model in one launch (same results, layer by layer).  At the end of
+ * a prefill every layer's K and V exist, and all layers share the chunk plan (it depends on token ids
+ * only): one call then replaces L, and the kernel has L times as many independent (layer, sequence, head)
+ * units to interleave, which matters when a layer alone has few of them.
+ *
+ *   layers      HOST array of L rows of DEVICE pointers: K, V (both with kv_strides), core_k, core_v,
+ *               count, core_len, assign (or NULL) as sc_compress takes them for that layer.  Layers must
+ *               not share outputs.  The array is read during the call only.
+ *   L           1..SC_MAX_LAYERS_PER_CALL
+ *   the rest    as for sc_compress; params->flags may hold SC_FLAG_GENERIC only (the generic kernels then
+ *               run layer after layer)
+ *   workspace   at least sc_compress_layers_workspace_bytes(L, B, Hkv, n) bytes, zeroed once after
+ *               allocation and left zeroed by every call
+ */
+typedef struct {
+    const void* K; const void* V;
+    void* core_k; void* core_v; int32_t* count; int32_t* core_len; int32_t* assign;
+} sc_compress_layer;
+
+#define SC_MAX_LAYERS_PER_CALL 64
+
+SC_API size_t sc_compress_layers_workspace_bytes(int32_t L, int32_t B, int32_t Hkv, int32_t n);
+
+SC_API sc_status sc_compress_layers(const sc_compress_layer* layers /*HOST [L]*/, int32_t L, sc_strides kv_strides,
+                             sc_dtype dt, int32_t B, int32_t Hkv, int32_t n, int32_t d,
+                             const int32_t* seg_off, const int32_t* seq_seg_off, const int32_t* n_seg,
+                             const int32_t* tile_seg, const int32_t* seq_tile_cnt, int32_t n_tile_cap,
+                             const sc_gsc_params* params /*HOST*/, int32_t cap,
+                             void* workspace, size_t workspace_bytes, int32_t* status, void* stream);
+
+/*
  * Compress one layer to a KV budget (the paper evaluates budgets of 20 / 35 / 50 % kept, Table 1, and
  * shows that a lower threshold keeps fewer entries, Table 4b; how a budget is turned into a threshold
  * it does not say).  This library's reading: the threshold of Algorithm 1 is searched on a grid

@@ -25,7 +25,9 @@ _STATUS_NAMES = ["SC_OK", "SC_ERR_INVALID_ARG", "SC_ERR_UNSUPPORTED", "SC_ERR_CA
 EXPORTS = ["sc_version", "sc_launch_counter", "sc_chunk_bounds", "sc_chunk_workspace_bytes", "sc_chunk",
            "sc_compress_workspace_bytes", "sc_compress", "sc_decode_workspace_bytes", "sc_decode_attn",
            "sc_decode_attn_static", "sc_append", "sc_compress_budget_workspace_bytes", "sc_compress_budget",
-           "sc_compress_global_workspace_bytes", "sc_compress_global", "sc_prefill_attn", "sc_append_layers"]
+           "sc_compress_global_workspace_bytes", "sc_compress_global", "sc_prefill_attn", "sc_append_layers",
+           "sc_compress_layers_workspace_bytes", "sc_compress_layers"]
+SC_MAX_LAYERS_PER_CALL = 64
 SC_BUDGET_MAX_GRID = 65
 SC_STATIC_SCRATCH_BYTES = 8 << 20
 
@@ -43,6 +45,10 @@ class _GscParams(ctypes.Structure):
 class _Budget(ctypes.Structure):
     _fields_ = [("target_kept", ctypes.c_float), ("tau_lo", ctypes.c_float), ("tau_hi", ctypes.c_float),
                 ("n_grid", ctypes.c_int32)]
+
+
+class _CompressLayer(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_void_p) for k in ("K", "V", "core_k", "core_v", "count", "core_len", "assign")]
 
 
 class _Strides(ctypes.Structure):
@@ -76,6 +82,11 @@ def lib() -> ctypes.CDLL:
         L.sc_compress.restype = _i32
         L.sc_compress.argtypes = [_vp, _vp, _Strides, _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32,
                                   ctypes.POINTER(_GscParams), _vp, _vp, _vp, _i32, _vp, _vp, _vp, _sz, _vp, _vp]
+        L.sc_compress_layers_workspace_bytes.restype = _sz
+        L.sc_compress_layers_workspace_bytes.argtypes = [_i32, _i32, _i32, _i32]
+        L.sc_compress_layers.restype = _i32
+        L.sc_compress_layers.argtypes = [ctypes.POINTER(_CompressLayer), _i32, _Strides, _i32, _i32, _i32, _i32, _i32,
+                                         _vp, _vp, _vp, _vp, _vp, _i32, ctypes.POINTER(_GscParams), _i32, _vp, _sz, _vp, _vp]
         L.sc_compress_budget_workspace_bytes.restype = _sz
         L.sc_compress_budget_workspace_bytes.argtypes = [_i32, _i32, _i32]
         L.sc_compress_budget.restype = _i32
@@ -178,6 +189,36 @@ def sc_compress(K, V, plan: "ChunkPlan", tau, core_k, core_v, count, core_len, a
                              _ptr(assign), _ptr(workspace), workspace.numel() * workspace.element_size(),
                              _ptr(status), _stream(K))
     _check("sc_compress", code)
+
+
+def compress_layers_workspace(L, B, Hkv, n, device) -> torch.Tensor:
+    """Zero-initialised workspace for sc_compress_layers."""
+    return torch.zeros(lib().sc_compress_layers_workspace_bytes(L, B, Hkv, n), dtype=torch.uint8, device=device)
+
+
+def sc_compress_layers(Ks, Vs, plan: "ChunkPlan", tau, outs, workspace, status=None, flags=0):
+    """Raw sc_compress_layers: ``Ks``/``Vs`` lists of [B, Hkv, n, d] tensors (same shape, dtype and strides),
+    ``outs`` a list of CompressedLayer (same capacity), one per layer; every layer in one launch."""
+    L = len(Ks)
+    K0 = Ks[0]
+    B, Hkv, n, d = K0.shape
+    cap = outs[0].core_k.shape[2]
+    rows = (_CompressLayer * L)()
+    for l in range(L):
+        K, V, o = Ks[l], Vs[l], outs[l]
+        _need_cuda(K, V, o.core_k, o.core_v, o.count, o.core_len, o.assign)
+        assert K.shape == K0.shape and V.shape == K0.shape and K.stride() == K0.stride() and V.stride() == K0.stride()
+        assert K.dtype == K0.dtype and V.dtype == K0.dtype and K.stride(3) == 1 and o.core_k.shape[2] == cap
+        assert o.core_k.is_contiguous() and o.core_v.is_contiguous() and o.count.is_contiguous()
+        rows[l] = _CompressLayer(_ptr(K), _ptr(V), _ptr(o.core_k), _ptr(o.core_v), _ptr(o.count), _ptr(o.core_len),
+                                 _ptr(o.assign))
+    prm = _GscParams(float(tau), int(plan.max_chunk_len), int(flags))
+    st = _Strides(K0.stride(0), K0.stride(1), K0.stride(2))
+    code = lib().sc_compress_layers(rows, L, st, _dt(K0), B, Hkv, n, d, _ptr(plan.seg_off), _ptr(plan.seq_seg_off),
+                                    _ptr(plan.n_seg), _ptr(plan.tile_seg), _ptr(plan.seq_tile_cnt), plan.n_tile_cap,
+                                    ctypes.byref(prm), cap, _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _ptr(status), _stream(K0))
+    _check("sc_compress_layers", code)
 
 
 def sc_compress_budget(K, V, plan: "ChunkPlan", target_kept, tau_lo, tau_hi, n_grid, core_k, core_v, count, core_len,

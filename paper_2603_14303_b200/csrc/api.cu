@@ -125,6 +125,59 @@ sc_status sc_compress(const void* K, const void* V, sc_strides kv_strides, sc_dt
     return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
 
+size_t sc_compress_layers_workspace_bytes(int32_t L, int32_t B, int32_t Hkv, int32_t n) {
+    if (L <= 0 || B <= 0 || Hkv <= 0 || n <= 0) return 256;
+    // [status words and counters of the fused kernel for all layers] [scratch of the generic kernels, one layer at a time]
+    return (compress_fused_layers_ws_bytes(L, B, Hkv, n) + 255) / 256 * 256 + compress_generic_ws_bytes(B, Hkv, n);
+}
+
+sc_status sc_compress_layers(const sc_compress_layer* layers, int32_t L, sc_strides kv_strides, sc_dtype dt, int32_t B,
+                             int32_t Hkv, int32_t n, int32_t d, const int32_t* seg_off, const int32_t* seq_seg_off,
+                             const int32_t* n_seg, const int32_t* tile_seg, const int32_t* seq_tile_cnt,
+                             int32_t n_tile_cap, const sc_gsc_params* params, int32_t cap, void* workspace,
+                             size_t workspace_bytes, int32_t* status, void* stream) {
+    if (L < 0 || L > SC_MAX_LAYERS_PER_CALL || B <= 0 || Hkv <= 0 || n <= 0 || cap < 0 || !params) return SC_ERR_INVALID_ARG;
+    if (dt != SC_BF16 && dt != SC_F32) return SC_ERR_UNSUPPORTED;
+    if (d < 8 || d > 256 || (d % 8) != 0) return SC_ERR_UNSUPPORTED;
+    if (params->max_chunk_len < 1 || params->max_chunk_len > SC_MAX_CHUNK_LEN) return SC_ERR_INVALID_ARG;
+    if (!(params->tau == params->tau) || (params->flags & ~SC_FLAG_GENERIC)) return SC_ERR_INVALID_ARG;
+    if (L == 0) return SC_OK;
+    if (!layers || !seg_off || !seq_seg_off || !n_seg || !tile_seg || !seq_tile_cnt || !workspace) return SC_ERR_INVALID_ARG;
+    const size_t esz = dt == SC_BF16 ? 2 : 4;
+    if ((kv_strides.b * esz) % 16 || (kv_strides.h * esz) % 16 || (kv_strides.n * esz) % 16) return SC_ERR_INVALID_ARG;
+    if (kv_strides.n < d || (int64_t)B * n > 0x7fffffff - 1) return SC_ERR_INVALID_ARG;
+    if (n_tile_cap < 1 || n_tile_cap > tile_cap_for(n)) return SC_ERR_INVALID_ARG;
+    if (workspace_bytes < sc_compress_layers_workspace_bytes(L, B, Hkv, n)) return SC_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l) {
+        const sc_compress_layer& y = layers[l];
+        if (!y.K || !y.V || !y.core_k || !y.core_v || !y.count || !y.core_len) return SC_ERR_INVALID_ARG;
+        if (!aligned16(y.K) || !aligned16(y.V) || !aligned16(y.core_k) || !aligned16(y.core_v)) return SC_ERR_INVALID_ARG;
+    }
+    CompressArgs a = {};
+    a.st = kv_strides; a.dt = dt; a.B = B; a.Hkv = Hkv; a.n = n; a.d = d;
+    a.seg_off = seg_off; a.seq_seg_off = seq_seg_off; a.n_seg = n_seg;
+    a.tile_seg = tile_seg; a.seq_tile_cnt = seq_tile_cnt; a.n_tile_cap = n_tile_cap;
+    a.tau = params->tau; a.max_chunk_len = params->max_chunk_len; a.flags = params->flags;
+    a.cap = cap; a.ws = workspace; a.status = status;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaErrorNotSupported;
+    if (!(a.flags & SC_FLAG_GENERIC)) {
+        CompressArgs probe = a;   // what compress_fused_supported looks at is shared by the layers
+        if (compress_fused_supported(probe)) e = launch_compress_fused_layers(a, layers, L, st);
+    }
+    if (e == cudaErrorNotSupported) {   // forced, or a shape / layout the fused kernel does not take: layer after layer
+        a.ws = (char*)workspace + (compress_fused_layers_ws_bytes(L, B, Hkv, n) + 255) / 256 * 256;
+        e = cudaSuccess;
+        for (int l = 0; l < L && e == cudaSuccess; ++l) {
+            CompressArgs g = a;
+            g.K = layers[l].K; g.V = layers[l].V; g.core_k = layers[l].core_k; g.core_v = layers[l].core_v;
+            g.count = layers[l].count; g.core_len = layers[l].core_len; g.assign = layers[l].assign;
+            e = launch_compress_generic(g, st);
+        }
+    }
+    return e == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
 size_t sc_compress_budget_workspace_bytes(int32_t B, int32_t Hkv, int32_t n) {
     return budget_state_bytes() + sc_compress_workspace_bytes(B, Hkv, n);
 }

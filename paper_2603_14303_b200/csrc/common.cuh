@@ -97,6 +97,8 @@ struct CompressArgs {
     const float* tau_dev; const int32_t* skip; int32_t count_only;
 };
 cudaError_t launch_compress_generic(const CompressArgs& a, cudaStream_t st);
+cudaError_t launch_compress_fused_layers(const CompressArgs& a, const sc_compress_layer* layers, int32_t L, cudaStream_t st);
+size_t compress_fused_layers_ws_bytes(int32_t L, int32_t B, int32_t Hkv, int32_t n);
 size_t compress_generic_ws_bytes(int32_t B, int32_t Hkv, int32_t n);
 
 struct GlobalArgs {   // clustering of whole sequences (no chunking)

@@ -30,7 +30,12 @@
 //      The service warp draws the block's next ticket during step 2.
 // The last block to finish zeroes the status words and counters, so a workspace that was zero
 // before the call is zero again after it.
+// One launch may serve several layers (sc_compress_layers): the tickets then go round the (layer, sequence,
+// head) units, which puts L*B*Hkv tickets between consecutive tiles of a head instead of B*Hkv; with few heads
+// per layer that is what keeps one late tile from holding up every tile of its head that is in flight.
 #include <cuda.h>
+
+#include <mutex>
 
 #include "common.cuh"
 
@@ -71,7 +76,7 @@ static_assert(kBarOff % 8 == 0, "mbarrier alignment");
 static_assert(kSmemBytes <= 76800, "three blocks per SM need <= 75 KB each");
 
 enum Mode { kCountOnly = 0, kWriteWithCounts = 1, kLookBack = 2 };
-enum Geo { gB = 0, gH = 1, gT = 2, gNseg = 3, gRow0 = 4, gR = 5, gLast = 6 };
+enum Geo { gB = 0, gH = 1, gT = 2, gNseg = 3, gRow0 = 4, gR = 5, gLast = 6, gLayer = 7 };
 
 // cnts[seed row] while the cluster waits to be pooled: kPending | first row of its segment | (one past its last
 // row) << 9, the latter 0 for a segment of up to 32 tokens, whose member mask is one segment-relative word
@@ -434,21 +439,28 @@ __device__ __forceinline__ void pool_clusters(unsigned char* lane_base, const ui
     }
 }
 
+// What differs between the layers of a multi-layer launch (sc_compress_layers); a one-layer launch has one.
+struct LayerRefs {
+    CUtensorMap map_k, map_v;   // [B, Hkv, n, 128] bf16, boxes of 32 rows x 64 columns, 128-byte swizzle
+    __nv_bfloat16* core_k; __nv_bfloat16* core_v; int32_t* count; int32_t* core_len; int32_t* assign;
+};
+constexpr int kMaxLayers = 64;   // layers per launch (the launch parameters hold their tensor maps)
+
+template <int NL>
 struct Params {
-    const __nv_bfloat16* K; const __nv_bfloat16* V; sc_strides st;
-    int B, Hkv, n;
+    int B, Hkv, n, L;
     const int32_t* seg_off; const int32_t* tile_seg; const int32_t* seq_tile_cnt; int n_tile_cap;
     float tau;
-    __nv_bfloat16* core_k; __nv_bfloat16* core_v; int32_t* count; int cap; int32_t* core_len;
-    int32_t* assign;
+    int cap;
     int32_t* ctl;            // [0] ticket counter, [1] blocks finished
-    uint32_t* tile_state;    // [B*Hkv][n_tile_cap]
+    uint32_t* tile_state;    // [L][B*Hkv][n_tile_cap]
     int32_t* status;
     const float* tau_dev;    // threshold in device memory (budget search), or null: use tau
     const int32_t* skip;     // device flag: nonzero = this launch has nothing to do (budget search), or null
     int count_into_len;      // kCountOnly: add the tile's cluster count to core_len instead of recording it per tile
-    CUtensorMap map_k, map_v;   // [B, Hkv, n, 128] bf16, boxes of 32 rows x 64 columns, 128-byte swizzle
+    LayerRefs layer[NL];
 };
+
 
 
 // The service warp draws the next ticket, turns it into a tile (sequence, head, tile index, rows) and
@@ -457,19 +469,22 @@ struct Params {
 // tickets apart and a tile's predecessor has usually published its cluster count (and often its
 // prefix) by the time the tile looks back.  A pair with fewer tiles skips its surplus tickets.
 // geo[gT] = -1 when no work is left (max_nt = most tiles any sequence has).
-__device__ __forceinline__ void fetch_tile(const Params& p, int lane, int max_nt, int* geo, int16_t* segs) {
-    const int pairs = p.B * p.Hkv;
-    int b, h, t, nt;
+template <int NL>
+__device__ __forceinline__ void fetch_tile(const Params<NL>& p, int lane, int max_nt, int* geo, int16_t* segs) {
+    const int pairs = p.B * p.Hkv, units = pairs * p.L;   // (layer, sequence, head) units take the tickets in turn
+    int b, h, t, nt, ly;
     for (;;) {
         int w = 0;
         if (lane == 0) w = atomicAdd(&p.ctl[0], 1);
         w = __shfl_sync(kFull, w, 0);
-        t = w / pairs;
+        t = w / units;
         if (t >= max_nt) {
             if (lane == 0) geo[gT] = -1;
             return;
         }
-        const int bh = w - t * pairs;
+        const int unit = w - t * units;
+        ly = unit / pairs;
+        const int bh = unit - ly * pairs;
         b = bh / p.Hkv;
         h = bh - b * p.Hkv;
         nt = min(p.seq_tile_cnt[b], p.n_tile_cap);
@@ -484,6 +499,7 @@ __device__ __forceinline__ void fetch_tile(const Params& p, int lane, int max_nt
     if (lane == 0) {
         geo[gB] = b; geo[gH] = h; geo[gT] = t; geo[gNseg] = nseg; geo[gRow0] = g_row0 - b * p.n; geo[gR] = R;
         geo[gLast] = (t == nt - 1);
+        geo[gLayer] = ly;
     }
 }
 
@@ -605,8 +621,8 @@ __device__ __forceinline__ void merge_long_segment(unsigned char* lane_base, int
     }
 }
 
-template <int kMode>
-__global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __grid_constant__ Params p) {
+template <int kMode, int NL>
+__global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __grid_constant__ Params<NL> p) {
     extern __shared__ __align__(1024) unsigned char smem[];   // the swizzle pattern repeats every 1024 bytes
     uint32_t* cnts = reinterpret_cast<uint32_t*>(smem + kCntOff);
     uint32_t* adj = reinterpret_cast<uint32_t*>(smem + kAdjOff);
@@ -661,6 +677,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         if (t < 0) break;
         const int b = geo[gB], h = geo[gH], nseg = geo[gNseg], row0 = geo[gRow0], R = geo[gR];
         const int bh = b * p.Hkv + h;
+        const LayerRefs& lr = p.layer[NL == 1 ? 0 : geo[gLayer]];
+        const int unit = (NL == 1 ? 0 : geo[gLayer]) * p.B * p.Hkv + bh;   // index of this (layer, sequence, head)
         const bool long_tile = R > kShortRows;
         const bool two_tensors = (kMode != kCountOnly) && !long_tile;   // V staged beside K
         const int nrb = (R + 31) >> 5;
@@ -668,13 +686,13 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
 
         // ---- 1. stage the rows (service warp, TMA); prefetch ahead ----
         if (service) {
-            stage_rows(sbase, hs, &p.map_k, row0, R, h, b, bar_k, lane);
-            if (two_tensors) stage_rows(sbase + kVOff, hs, &p.map_v, row0, R, h, b, bar_v, lane);
+            stage_rows(sbase, hs, &lr.map_k, row0, R, h, b, bar_k, lane);
+            if (two_tensors) stage_rows(sbase + kVOff, hs, &lr.map_v, row0, R, h, b, bar_v, lane);
         }
         // end of the segment each row is in (0 past the tile)
         // also: one-token segments (delimiters, lone tokens) are clusters of their own -- no key needed;
         // the others are listed for the warps
-        int32_t* as = p.assign ? p.assign + (size_t)bh * p.n + row0 : nullptr;
+        int32_t* as = lr.assign ? lr.assign + (size_t)bh * p.n + row0 : nullptr;
         if (nseg == 1 && R > 1) {
             for (int r = tid; r < R; r += kThreads) send[r] = (uint16_t)R;
             if (R > kWarpSegMax && tid < nrb) { atomicOr(&misc[2], 1 << tid); reach[tid] = nrb - 1; }
@@ -781,10 +799,10 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         int P = 0;
 #pragma unroll
         for (int w = 0; w < kNW; ++w) P += __popc(seedmask[w]);
-        uint32_t* stt = p.tile_state + (size_t)bh * p.n_tile_cap;
+        uint32_t* stt = p.tile_state + (size_t)unit * p.n_tile_cap;
         if (kMode == kCountOnly) {
             if (tid == 0) {
-                if (p.count_into_len) atomicAdd(&p.core_len[bh], P);
+                if (p.count_into_len) atomicAdd(&lr.core_len[bh], P);
                 else stt[t] = (uint32_t)P;
             }
         } else {
@@ -848,7 +866,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 if (lane == 0) {
                     misc[0] = base;
                     if (geo[gLast]) {
-                        p.core_len[bh] = base + P;
+                        lr.core_len[bh] = base + P;
                         if (base + P > p.cap) set_status(p.status, SC_ERR_CAPACITY);
                     }
                 }
@@ -863,19 +881,19 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 if (base + row < p.cap) {
                     const size_t o = (obase + base + row) * kD + c * 8;
                     const unsigned char* src = smem + (c >> 3) * hs + tile_addr(seedrow[row], c & 7);
-                    *reinterpret_cast<uint4*>(p.core_k + o) = *reinterpret_cast<const uint4*>(src);
-                    if (!long_tile) *reinterpret_cast<uint4*>(p.core_v + o) = *reinterpret_cast<const uint4*>(src + kVOff);
+                    *reinterpret_cast<uint4*>(lr.core_k + o) = *reinterpret_cast<const uint4*>(src);
+                    if (!long_tile) *reinterpret_cast<uint4*>(lr.core_v + o) = *reinterpret_cast<const uint4*>(src + kVOff);
                 }
             }
             for (int row = tid; row < P; row += kThreads)
                 if (base + row < p.cap)
-                    p.count[obase + base + row] = (int32_t)cnts[seedrow[row]];
+                    lr.count[obase + base + row] = (int32_t)cnts[seedrow[row]];
 
             // ---- a tile longer than SC_TILE_ROWS: V takes the place of K and is pooled with the same masks ----
             if (long_tile) {
                 fence_async_proxy();   // the copies below overwrite what ordinary accesses read and wrote
                 __syncthreads();
-                if (service) stage_rows(sbase, hs, &p.map_v, row0, R, h, b, bar_v, lane);
+                if (service) stage_rows(sbase, hs, &lr.map_v, row0, R, h, b, bar_v, lane);
                 failed = !mbar_wait(bar_v, phase_v);
                 phase_v ^= 1u;
                 if (__syncthreads_or(failed)) { failed = true; break; }
@@ -884,7 +902,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 for (int idx = tid; idx < P * 16; idx += kThreads) {
                     const int row = idx >> 4, c = idx & 15;
                     if (base + row < p.cap)
-                        *reinterpret_cast<uint4*>(p.core_v + (obase + base + row) * kD + c * 8) =
+                        *reinterpret_cast<uint4*>(lr.core_v + (obase + base + row) * kD + c * 8) =
                             *reinterpret_cast<const uint4*>(smem + (c >> 3) * hs + tile_addr(seedrow[row], c & 7));
                 }
             }
@@ -918,7 +936,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     if (misc[1]) {
         __threadfence();
         if (kMode != kCountOnly) {
-            const size_t words = (size_t)p.B * p.Hkv * p.n_tile_cap;
+            const size_t words = (size_t)p.L * p.B * p.Hkv * p.n_tile_cap;
             for (size_t i = tid; i < words; i += kThreads) p.tile_state[i] = 0u;
         }
         if (tid == 0) { p.ctl[0] = 0; p.ctl[1] = 0; }
@@ -975,45 +993,65 @@ size_t compress_fused_ws_bytes(int32_t B, int32_t Hkv, int32_t n) {
     return sizeof(uint32_t) * ((size_t)B * Hkv * tiles + cf::kCtlWords) + 256;
 }
 
-cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
-    static int grid_of[64] = {0};   // per device: blocks that are resident at once
+namespace {
+
+// Blocks that are resident at once on the current device (one persistent block each), set up on first use.
+int resident_blocks() {
+    static int grid_of[64] = {0};
     int dev = 0;
     cudaGetDevice(&dev);
     dev &= 63;
     if (grid_of[dev] == 0) {
-        cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kCountOnly>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
-        cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kWriteWithCounts>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
-        cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kLookBack>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
+        cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kCountOnly, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
+        cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kWriteWithCounts, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
+        cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kLookBack, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
+        cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kLookBack, cf::kMaxLayers>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
         int sms = 0, per_sm = 0;
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cf::compress_fused_kernel<cf::kLookBack>, cf::kThreads,
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cf::compress_fused_kernel<cf::kLookBack, 1>, cf::kThreads,
                                                       cf::kSmemBytes);
         grid_of[dev] = (sms < 1 ? 1 : sms) * (per_sm < 1 ? 1 : per_sm);
     }
-    cf::Params p;
-    p.K = (const __nv_bfloat16*)a.K; p.V = (const __nv_bfloat16*)a.V; p.st = a.st;
-    p.B = a.B; p.Hkv = a.Hkv; p.n = a.n;
+    return grid_of[dev];
+}
+
+template <int NL>
+void fill_common(cf::Params<NL>& p, const CompressArgs& a, int L) {
+    p.B = a.B; p.Hkv = a.Hkv; p.n = a.n; p.L = L;
     p.seg_off = a.seg_off; p.tile_seg = a.tile_seg; p.seq_tile_cnt = a.seq_tile_cnt; p.n_tile_cap = a.n_tile_cap;
-    p.tau = a.tau;
+    p.tau = a.tau; p.cap = a.cap;
     p.tau_dev = a.tau_dev; p.skip = a.skip; p.count_into_len = a.count_only ? 1 : 0;
-    p.core_k = (__nv_bfloat16*)a.core_k; p.core_v = (__nv_bfloat16*)a.core_v; p.count = a.count; p.cap = a.cap;
-    p.core_len = a.core_len; p.assign = a.assign;
     p.ctl = (int32_t*)a.ws;
     p.tile_state = (uint32_t*)a.ws + cf::kCtlWords;
     p.status = a.status;
-    if (!make_map(&p.map_k, a.K, a.st, a.B, a.Hkv, a.n) || !make_map(&p.map_v, a.V, a.st, a.B, a.Hkv, a.n))
+}
+
+bool fill_layer(cf::LayerRefs& r, const CompressArgs& a, const void* K, const void* V, void* core_k, void* core_v,
+                int32_t* count, int32_t* core_len, int32_t* assign) {
+    r.core_k = (__nv_bfloat16*)core_k; r.core_v = (__nv_bfloat16*)core_v; r.count = count; r.core_len = core_len;
+    r.assign = assign;
+    return make_map(&r.map_k, K, a.st, a.B, a.Hkv, a.n) && make_map(&r.map_v, V, a.st, a.B, a.Hkv, a.n);
+}
+
+}  // namespace
+
+cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
+    const int resident = resident_blocks();
+    cf::Params<1> p;
+    fill_common(p, a, 1);
+    if (!fill_layer(p.layer[0], a, a.K, a.V, a.core_k, a.core_v, a.count, a.core_len, a.assign))
         return cudaErrorNotSupported;   // a layout TMA cannot describe: the caller takes the generic kernels
     // no more blocks than there can be tiles
     const int64_t max_tiles = (int64_t)a.B * a.Hkv * a.n_tile_cap;
-    const int grid = (int)(max_tiles < grid_of[dev] ? max_tiles : grid_of[dev]);
+    const int grid = (int)(max_tiles < resident ? max_tiles : resident);
     if (a.count_only) {   // budget search: per-head cluster counts only
-        cf::compress_fused_kernel<cf::kCountOnly><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
+        cf::compress_fused_kernel<cf::kCountOnly, 1><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
         note_launches(1);
     } else if (a.flags & SC_FLAG_TWO_PASS) {
-        cf::Params pc = p;
-        pc.assign = nullptr;
-        cf::compress_fused_kernel<cf::kCountOnly><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(pc);
-        cf::compress_fused_kernel<cf::kWriteWithCounts><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
+        cf::Params<1> pc = p;
+        pc.layer[0].assign = nullptr;
+        cf::compress_fused_kernel<cf::kCountOnly, 1><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(pc);
+        cf::compress_fused_kernel<cf::kWriteWithCounts, 1><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
         note_launches(2);
     } else {
         // With SC_FLAG_OVERLAP_PREV the kernel may start while the one enqueued before it on the stream is
@@ -1030,9 +1068,36 @@ cudaError_t launch_compress_fused(const CompressArgs& a, cudaStream_t st) {
         cfg.attrs = attr;
         cfg.numAttrs = (a.flags & SC_FLAG_OVERLAP_PREV) ? 1 : 0;
         note_launches(1);
-        return cudaLaunchKernelEx(&cfg, cf::compress_fused_kernel<cf::kLookBack>, p);
+        return cudaLaunchKernelEx(&cfg, cf::compress_fused_kernel<cf::kLookBack, 1>, p);
     }
     return cudaGetLastError();
+}
+
+// Several layers in one launch (sc_compress_layers): the (layer, sequence, head) units take the tickets in turn,
+// so consecutive tiles of one head are L*B*Hkv tickets apart and a tile's predecessor has usually published its
+// prefix long before the tile looks back.  `a` describes what the layers share (a.K .. a.assign are not used).
+cudaError_t launch_compress_fused_layers(const CompressArgs& a, const sc_compress_layer* layers, int32_t L, cudaStream_t st) {
+    if (L < 1 || L > cf::kMaxLayers) return cudaErrorInvalidValue;
+    const int resident = resident_blocks();
+    static cf::Params<cf::kMaxLayers> p;   // 20 KB: kept off the stack; filled and passed by value under the lock
+    static std::mutex lock;
+    std::lock_guard<std::mutex> guard(lock);
+    fill_common(p, a, L);
+    for (int l = 0; l < L; ++l)
+        if (!fill_layer(p.layer[l], a, layers[l].K, layers[l].V, layers[l].core_k, layers[l].core_v, layers[l].count,
+                        layers[l].core_len, layers[l].assign))
+            return cudaErrorNotSupported;
+    for (int l = L; l < cf::kMaxLayers; ++l) p.layer[l] = p.layer[0];
+    const int64_t max_tiles = (int64_t)L * a.B * a.Hkv * a.n_tile_cap;
+    const int grid = (int)(max_tiles < resident ? max_tiles : resident);
+    cf::compress_fused_kernel<cf::kLookBack, cf::kMaxLayers><<<grid, cf::kThreads, cf::kSmemBytes, st>>>(p);
+    note_launches(1);
+    return cudaGetLastError();
+}
+
+size_t compress_fused_layers_ws_bytes(int32_t L, int32_t B, int32_t Hkv, int32_t n) {
+    const size_t tiles = 2 * (size_t)div_up(n, SC_TILE_ROWS) + 1;
+    return sizeof(uint32_t) * ((size_t)L * B * Hkv * tiles + cf::kCtlWords) + 256;
 }
 
 }  // namespace sc

@@ -22,7 +22,8 @@ ROOT = os.path.dirname(HERE)
 RECORD = os.path.join(ROOT, "profiles", "traffic.txt")
 
 # stage -> source file whose change invalidates the record
-SOURCES = {"decode": "csrc/decode_mma.cu", "compress": "csrc/compress_fused.cu", "prefill": "csrc/prefill_umma.cu"}
+SOURCES = {"decode": "csrc/decode_mma.cu", "compress": "csrc/compress_fused.cu", "compress_layers": "csrc/compress_fused.cu",
+           "prefill": "csrc/prefill_umma.cu"}
 
 _UNITS = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9, "Tbyte": 1e12}
 

@@ -529,3 +529,37 @@ def test_overlapped_launches_two_apart_may_share_a_workspace():
                                 flags=binding.SC_FLAG_OVERLAP_PREV if l > 0 else 0)
         torch.cuda.synchronize()
         assert torch.equal(plain, fast), f"repeat {rep}"
+
+
+@pytest.mark.parametrize("L,n,flags,dtype", [(5, 3000, 0, "bf16"), (33, 700, 0, "bf16"), (3, 1500, binding.SC_FLAG_GENERIC, "bf16"),
+                                             (2, 900, 0, "f32")])
+def test_all_layers_in_one_launch_equal_one_launch_per_layer(L, n, flags, dtype):
+    """sc_compress_layers: every layer has its own K and V (so it clusters differently), all share the chunk
+    plan; the products must equal sc_compress layer by layer, bit for bit, and layer 0 the oracle."""
+    w = synth.config(0, n=n, L=L, B=2, Hkv=2, Hq=8, dtype=dtype)
+    ids, run_id, run_lens = synth.token_ids(w)
+    plan = binding.chunk(ids.to(DEV), w.delims, w.max_chunk_len)
+    Ks, Vs, single = [], [], []
+    for l in range(L):
+        K, V = synth.layer_kv(w, l, run_id, run_lens)
+        Ks.append(K.to(DEV)); Vs.append(V.to(DEV))
+        single.append(binding.compress(Ks[l], Vs[l], plan, w.tau, want_assign=True, flags=flags))
+    i32 = dict(dtype=torch.int32, device=DEV)
+    outs = [binding.CompressedLayer(torch.zeros_like(s.core_k), torch.zeros_like(s.core_v), torch.zeros_like(s.count),
+                                    torch.zeros_like(s.core_len), torch.full_like(s.assign, -1)) for s in single]
+    ws = binding.compress_layers_workspace(L, w.B, w.Hkv, n, DEV)
+    for rep in range(2):   # the workspace is left ready for the next call
+        binding.sc_compress_layers(Ks, Vs, plan, w.tau, outs, ws, plan.status, flags)
+        binding.check_status(plan.status)
+        for l in range(L):
+            a, b = single[l], outs[l]
+            assert torch.equal(a.core_len, b.core_len) and torch.equal(a.assign, b.assign), f"layer {l}"
+            for bb in range(w.B):
+                for h in range(w.Hkv):
+                    m = int(a.core_len[bb, h])
+                    assert torch.equal(a.count[bb, h, :m], b.count[bb, h, :m])
+                    assert torch.equal(a.core_k[bb, h, :m], b.core_k[bb, h, :m]) and torch.equal(a.core_v[bb, h, :m], b.core_v[bb, h, :m])
+    K0, V0 = synth.layer_kv(w, 0, run_id, run_lens)
+    compare_compressed(outs[0], oracle_compress(ids, K0, V0, w.delims, w.tau), K0.dtype)
+    fused_words = binding.lib().sc_compress_layers_workspace_bytes(L, w.B, w.Hkv, n) - binding.lib().sc_compress_workspace_bytes(w.B, w.Hkv, n)
+    assert int(ws[: max(fused_words, 256)].view(torch.int32).abs().max()) == 0, "status words and counters are left at zero"
