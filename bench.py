@@ -452,6 +452,7 @@ def measure_cell(w: synth.Workload, full_L: int, dev, sampler, peak, label: dict
     cbytes, dbytes, per_layer, kept = pipe.algorithmic_bytes()
     ms_c = pipe.time_graph(pipe.g_compress, 3)
     ms_d = pipe.time_graph(pipe.g_decode["chain"], 3)
+    ms_l = time_calls(lambda: pipe.run_compress(True), 3)   # the same layers in one sc_compress_layers launch
     layer_bytes = sum(per_layer) / len(per_layer)
     us_launch = ms_d * 1e3 / (decode_steps * w.L)
     dgbs = layer_bytes / (us_launch * 1e-6) / 1e9
@@ -464,7 +465,9 @@ def measure_cell(w: synth.Workload, full_L: int, dev, sampler, peak, label: dict
         "decode_us_per_launch": us_launch, "decode_gbs": dgbs, "decode_frac": dgbs / peak,
         "decode_frac_of_nominal_8tbs": dgbs / 8000.0, "compress_frac_of_nominal_8tbs": cgbs / 8000.0,
         "compress_ms_per_32k_ctx": ms_c / w.L * full_L * 32768 / (w.B * w.n), "compress_us_per_layer": ms_c * 1e3 / w.L,
-        "compress_gbs": cgbs, "compress_frac": cgbs / peak})
+        "compress_gbs": cgbs, "compress_frac": cgbs / peak,
+        "compress_all_layers_one_launch": {"layers": w.L, "ms_per_32k_ctx": ms_l / w.L * full_L * 32768 / (w.B * w.n),
+                                           "us_per_layer": ms_l * 1e3 / w.L, "frac": cbytes / (ms_l * 1e-3) / 1e9 / peak}})
     if raw:
         ms_r = pipe.time_graph(pipe.g_decode["raw"], 3)
         us_r = ms_r * 1e3 / (pipe.steps_of["raw"] * w.L)
@@ -615,7 +618,8 @@ def sweep_configs(args, dev, sampler, peak):
 
     Every cell runs a reduced number of layers whose cores still exceed the L2 by a wide margin (the
     toy workload excepted: it is L2-resident by definition and its fractions are informational)."""
-    out = {"what": "per cell: chained decode and compress on a reduced layer count (layers_run), rates scaled to "
+    out = {"what": "per cell: chained decode and compress (one sc_compress per layer; compress_all_layers_one_launch: the "
+                   "same layers in one sc_compress_layers) on a reduced layer count (layers_run), rates scaled to "
                    "layers_full; fractions of the measured HBM copy peak", "peak_gbs": peak}
     c0, c2, c3, c4 = (synth.config(i) for i in (0, 2, 3, 4))
     out["cfg0"] = measure_cell(c0, c0.L, dev, sampler, peak, {"workload": c0.name, "note": "L2-resident toy"},
