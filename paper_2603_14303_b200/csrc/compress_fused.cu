@@ -38,6 +38,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "umma.cuh"
 
 namespace sc {
 
@@ -70,8 +71,10 @@ constexpr int kSendOff = kNormOff + kWarps * 64 * 4; // uint16[256]: end of the 
 constexpr int kSegsOff = kSendOff + kMaxRows * 2; // 2 x int16[132]: segment starts (this tile, next tile)
 constexpr int kSegsStride = 132;
 constexpr int kMiscOff = kSegsOff + 2 * kSegsStride * 2;   // uint32 seedmask[8]; int geo[2][8]; int misc[4]
-constexpr int kBarOff = kMiscOff + 32 + 64 + 16 + 32 + 128;      // ... int reach[8]; uint8 multi[128]; two mbarriers
-constexpr int kSmemBytes = kBarOff + 16;
+constexpr int kBarOff = kMiscOff + 32 + 64 + 16 + 32 + 128 + 16;   // ... uint32 umma_rows[8]; uint8 multi[128]; tensor-memory slot, flag; three mbarriers
+constexpr int kSmemBytes = kBarOff + 24;
+constexpr int kTmemCols = 128;                    // one 128 x 128 fp32 accumulator per block (three blocks per SM: 384 of 512 columns)
+constexpr int kBlocksPerSm = 3;
 static_assert(kBarOff % 8 == 0, "mbarrier alignment");
 static_assert(kSmemBytes <= 76800, "three blocks per SM need <= 75 KB each");
 
@@ -159,95 +162,79 @@ __device__ __forceinline__ int adj_row(int i) {
     return 256 * k - 16 * k * (k - 1) + (i & 31) * (kNW - k);
 }
 
-// 32x32 block of K.K^T: rows of block rb against rows of block cb (column halves `hs` bytes apart).
-template <bool kDiag>
-__device__ __forceinline__ void gram_block(uint32_t kbase, int hs, int rb, int cb, int lane, float (&acc)[2][4][4]) {
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int nt = 0; nt < 4; ++nt) acc[mt][nt][0] = acc[mt][nt][1] = acc[mt][nt][2] = acc[mt][nt][3] = 0.f;
-    const int j = lane >> 3, r8 = lane & 7;
-    // A: matrices (r0-7,c) (r8-15,c) (r0-7,c+1) (r8-15,c+1);  B: (r0-7,c) (r0-7,c+1) (r8-15,c) (r8-15,c+1)
-    // chunk 2*ks + c of a row sits in half ks >> 2 at chunk (2*(ks & 3) + c) ^ (row & 7): XOR of a constant
-    const uint32_t a_addr = kbase + tile_addr(rb * 32 + r8 + ((j & 1) << 3), j >> 1);
-    const uint32_t b_addr = kbase + tile_addr(cb * 32 + r8 + ((j >> 1) << 3), j & 1);
+// 16 consecutive fp32 columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+
+// One 128 x 128 block of K.K^T of the staged keys: rows of 128-row block mb against rows of block nb (column
+// halves `hs` bytes apart, 128-byte-swizzled rows: what the TMA boxes wrote is the K-major layout tcgen05.mma
+// reads).  One thread issues the eight instructions; the mbarrier gets one arrival when they are complete.
+__device__ __forceinline__ void umma_gram_block(uint32_t kbase, int hs, int mb, int nb, uint32_t tmem, uint32_t bar) {
+    constexpr uint32_t idesc = umma::instr_desc_bf16(128, 128, false, false);
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks) {
-        uint32_t a[2][4], bq[2][4];
-        const uint32_t kx = (ks & 3) << 5, ko = (ks >> 2) * hs;
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-            ldmatrix_x4((a_addr ^ kx) + ko + mt * 16 * kHalfRow, a[mt][0], a[mt][1], a[mt][2], a[mt][3]);
-#pragma unroll
-        for (int p = 0; p < 2; ++p)
-            ldmatrix_x4((b_addr ^ kx) + ko + p * 16 * kHalfRow, bq[p][0], bq[p][1], bq[p][2], bq[p][3]);
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                if (kDiag && nt < 2 * mt) continue;   // wholly below the diagonal: never read
-                mma_bf16(acc[mt][nt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], bq[nt >> 1][(nt & 1) * 2], bq[nt >> 1][(nt & 1) * 2 + 1]);
-            }
+        const uint32_t off = (ks >> 2) * hs + (ks & 3) * 32;
+        umma::mma_bf16_ss(tmem, umma::smem_desc_sw128(kbase + mb * 128 * kHalfRow + off, 16, 1024),
+                          umma::smem_desc_sw128(kbase + nb * 128 * kHalfRow + off, 16, 1024), idesc, ks > 0);
     }
+    umma::mma_commit(bar);
 }
 
-// Diagonal of a diagonal Gram block = squared norms of its 32 rows.
-__device__ __forceinline__ void store_norms(const float (&acc)[2][4][4], int rb, int lane, float* norm) {
-    const int g = lane >> 2, tig = lane & 3;
-    if ((g >> 1) == tig) {
-        const int e = g & 1;
+// The diagonal of a diagonal block = squared norms: thread (quarter q, lane) of the four reading warps owns tile
+// row mb*128 + 32q + lane and finds its element in the 32 columns its warp's rows share.
+__device__ __forceinline__ void umma_norms(uint32_t tmem, int mb, int q, int lane, float* norm) {
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    float v = 0.f;
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
+    for (int c = 0; c < 2; ++c) {
+        uint32_t g[16];
+        tmem_ld16(lane_addr + q * 32 + c * 16, g);
+        umma::tmem_ld_wait();
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh)
-                norm[rb * 32 + mt * 16 + hh * 8 + g] =
-                    sqrtf(e ? acc[mt][2 * mt + hh][hh * 2 + 1] : acc[mt][2 * mt + hh][hh * 2]);
+        for (int k = 0; k < 16; ++k)
+            if (lane == c * 16 + k) v = __uint_as_float(g[k]);
     }
+    norm[mb * 128 + q * 32 + lane] = sqrtf(v);
 }
 
-// Turns a Gram block into adjacency words: bit j of word (i, cb) = Sim(i, 32cb + j) > tau, limited
-// to later tokens of i's own segment.
-template <bool kNegTau, bool kDiag>
-__device__ __forceinline__ void threshold_block(const float (&acc)[2][4][4], int rb, int cb, int lane, float tau,
-                                                const float* norm, const uint16_t* send, uint32_t* adj) {
-    const int g = lane >> 2, tig = lane & 3;
-    float tn[4][2];
+// Turns the block in tensor memory into adjacency words of the rows that belong to long segments (umma_rows):
+// bit j of word (i, cb) = Sim(i, 32cb + j) > tau, limited to later tokens of i's own segment.
+template <bool kNegTau>
+__device__ __forceinline__ void umma_threshold(uint32_t tmem, int mb, int nb, int q, int lane, float tau, const float* norm,
+                                               const uint16_t* send, const uint32_t* umma_rows, uint32_t* adj) {
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    const int i = mb * 128 + q * 32 + lane;
+    const float ni = norm[i];
+    uint32_t words[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-    for (int nt = 0; nt < 4; ++nt) {
-        const float2 nn = *reinterpret_cast<const float2*>(norm + cb * 32 + nt * 8 + 2 * tig);
-        tn[nt][0] = tau * nn.x;
-        tn[nt][1] = tau * nn.y;
-    }
+    for (int c = 0; c < 8; ++c) {
+        uint32_t g[16];
+        tmem_ld16(lane_addr + c * 16, g);
+        umma::tmem_ld_wait();
+        uint32_t w = 0u;
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-            const int i = rb * 32 + mt * 16 + hh * 8 + g;
-            const float ni = norm[i];
-            uint32_t w = 0;   // bit nt*8 + e, moved to nt*8 + 2*tig + e afterwards
-#pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                if (kDiag && nt < 2 * mt + hh) continue;   // columns before the row's own: masked out anyway
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const float thr = ni * tn[nt][e];
-                    bool hit = acc[mt][nt][hh * 2 + e] > thr;
-                    if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
-                    if (hit) w |= 1u << (nt * 8 + e);
-                }
-            }
-            w <<= 2 * tig;
-            w |= __shfl_xor_sync(kFull, w, 1);
-            w |= __shfl_xor_sync(kFull, w, 2);
-            // (a token with no later token in its segment keeps its word: a one-token segment's is already final)
-            const int e_i = (int)send[i];
-            if (tig == 0 && e_i > i + 1) adj[adj_row(i) + (cb - rb)] = w & bits_between(i + 1, e_i, cb);
+        for (int k = 0; k < 16; ++k) {
+            const float thr = ni * (tau * norm[nb * 128 + c * 16 + k]);
+            bool hit = __uint_as_float(g[k]) > thr;
+            if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
+            w |= (hit ? 1u : 0u) << k;
         }
+        words[c >> 1] |= w << ((c & 1) * 16);
+    }
+    if ((umma_rows[i >> 5] >> (i & 31)) & 1u) {
+        const int e_i = (int)send[i], rb = i >> 5;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int cb = nb * 4 + c;
+            if (cb >= rb && e_i > i + 1) adj[adj_row(i) + (cb - rb)] = words[c] & bits_between(i + 1, e_i, cb);
+        }
+    }
 }
-
-// Off-diagonal block pairs (row block << 4 | column block), nearest diagonals first.
-__constant__ uint8_t kOffDiag[28] = {0x01, 0x12, 0x23, 0x34, 0x45, 0x56, 0x67, 0x02, 0x13, 0x24, 0x35, 0x46, 0x57, 0x03,
-                                     0x14, 0x25, 0x36, 0x47, 0x04, 0x15, 0x26, 0x37, 0x05, 0x16, 0x27, 0x06, 0x17, 0x07};
 
 // Eq. 3 building blocks.  A lane owns eight consecutive columns (one 16-byte chunk) of the K row
 // (lanes 0-15) or of the V row (lanes 16-31); `lane_base` is its tensor and column half, c7 its
@@ -635,10 +622,12 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     int* misc = reinterpret_cast<int*>(smem + kMiscOff + 96);           // [0] output offset of the tile, [1] last block,
                                                                         // [2] 32-row blocks that a segment of > 32 tokens touches,
                                                                         // [3] number of segments of more than one token
-    int* reach = reinterpret_cast<int*>(smem + kMiscOff + 112);         // [8] last block such a segment spans from block k
+    uint32_t* umma_rows = reinterpret_cast<uint32_t*>(smem + kMiscOff + 112);   // [8] rows of segments of more than kWarpSegMax tokens
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kMiscOff + 272);
+    volatile int* umma_failed = reinterpret_cast<volatile int*>(smem + kMiscOff + 276);   // a wait for the tensor core gave up
     uint8_t* multi = smem + kMiscOff + 144;                             // [128] the segments of more than one token
     const uint32_t sbase = smem_u32(smem);
-    const uint32_t bar_k = sbase + kBarOff, bar_v = bar_k + 8;
+    const uint32_t bar_k = sbase + kBarOff, bar_v = bar_k + 8, bar_u = bar_k + 16;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool service = warp == kWarps;   // the ninth warp
@@ -652,22 +641,30 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     if (tid == 0) {
         mbar_init(bar_k, 1);
         mbar_init(bar_v, 1);
+        mbar_init(bar_u, 1);
+        *umma_failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         if ((sbase & 1023u) != 0u) set_status(p.status, SC_ERR_CUDA);   // the swizzled addressing assumes this
     }
     fence_async_proxy();
-    uint32_t phase_k = 0, phase_v = 0;
+    uint32_t phase_k = 0, phase_v = 0, phase_u = 0;
     bool failed = false;
+    // Tensor memory for the Gram blocks of long segments: allocated once per (persistent) block by the service warp,
+    // which then gives up the permit (a block may not allocate again after that, so it is not done per tile).
+    if (warp == kWarps) umma::tmem_alloc(sbase + kMiscOff + 272, kTmemCols);
+    umma::fence_before_sync();
 
     if (service) {
         for (int b = lane; b < p.B; b += 32) max_nt = max(max_nt, min(p.seq_tile_cnt[b], p.n_tile_cap));
         max_nt = warp_max_i(max_nt);
         fetch_tile(p, lane, max_nt, geo_buf, segs_buf);
     }
-    if (tid < kNW) reach[tid] = 0;
+    if (tid < kNW) umma_rows[tid] = 0u;
     if (tid == kNW) misc[2] = misc[3] = 0;
     if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
     __syncthreads();
+    umma::fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
 
     int buf = 0;
     for (;;) {
@@ -695,7 +692,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         int32_t* as = lr.assign ? lr.assign + (size_t)bh * p.n + row0 : nullptr;
         if (nseg == 1 && R > 1) {
             for (int r = tid; r < R; r += kThreads) send[r] = (uint16_t)R;
-            if (R > kWarpSegMax && tid < nrb) { atomicOr(&misc[2], 1 << tid); reach[tid] = nrb - 1; }
+            if (R > kWarpSegMax && tid < nrb) { atomicOr(&misc[2], 1 << tid); umma_rows[tid] = bits_between(0, R, tid); }
             if (tid == 0) { multi[0] = 0; misc[3] = 1; }
         } else {
             for (int s = tid; s < nseg; s += kThreads) {
@@ -710,7 +707,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 multi[atomicAdd(&misc[3], 1)] = (uint8_t)s;
                 if (e - a > kWarpSegMax) {   // only the block-level path reads send[] (of every row of the blocks it touches)
                     for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
-                    for (int k = a >> 5; k <= (e - 1) >> 5; ++k) { atomicOr(&misc[2], 1 << k); atomicMax(&reach[k], (e - 1) >> 5); }
+                    for (int k = a >> 5; k <= (e - 1) >> 5; ++k) { atomicOr(&misc[2], 1 << k); atomicOr(&umma_rows[k], bits_between(a, e, k)); }
                 }
             }
         }
@@ -723,28 +720,33 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         }
         if (__syncthreads_or(failed)) { failed = true; break; }
 
-        // ---- 2. segments of more than kWarpSegMax tokens: Gram blocks -> norms -> adjacency bits in shared memory ----
-        const int longblocks = misc[2];
-        if (longblocks != 0) {
-            float acc[2][4][4];
-            const bool have = warp < nrb && ((longblocks >> warp) & 1);   // nrb <= kWarps
-            if (have) {
-                gram_block<true>(sbase, hs, warp, warp, lane, acc);
-                store_norms(acc, warp, lane, norm);
+        // ---- 2. segments of more than kWarpSegMax tokens: the tile's Gram matrix on the tensor core, 128 x 128 at a
+        //         time into tensor memory (one block for a tile of up to 128 tokens; diagonal blocks first, they
+        //         give the norms), thresholded by four warps, one row per thread, into the bit rows ----
+        if (misc[2] != 0) {
+            const int npass = R > 128 ? 3 : 1;   // (0,0); (1,1), (0,1)
+            for (int ps = 0; ps < npass; ++ps) {
+                const int mb = ps == 1 ? 1 : 0, nb = ps == 0 ? 0 : 1;
+                if (service && lane == 0) {
+                    umma::fence_after_sync();
+                    umma_gram_block(sbase, hs, mb, nb, tmem, bar_u);
+                }
+                if (warp < 4) {
+                    if (!mbar_wait(bar_u, phase_u)) *umma_failed = 1;
+                    umma::fence_after_sync();
+                    if (mb == nb) umma_norms(tmem, mb, warp, lane, norm);
+                }
+                phase_u ^= 1u;
+                __syncthreads();   // the norms are in place (and a wait that gave up is known to all)
+                if (*umma_failed) break;
+                if (warp < 4) {
+                    if (tau < 0.f) umma_threshold<true>(tmem, mb, nb, warp, lane, tau, norm, send, umma_rows, adj);
+                    else umma_threshold<false>(tmem, mb, nb, warp, lane, tau, norm, send, umma_rows, adj);
+                    umma::fence_before_sync();
+                }
+                __syncthreads();   // the bit rows are written; the accumulator may be overwritten
             }
-            __syncthreads();
-            if (have) {
-                if (tau < 0.f) threshold_block<true, true>(acc, warp, warp, lane, tau, norm, send, adj);
-                else threshold_block<false, true>(acc, warp, warp, lane, tau, norm, send, adj);
-            }
-            for (int k = service ? 28 : warp; k < 28; k += kWarps) {
-                const int rb = kOffDiag[k] >> 4, cb = kOffDiag[k] & 15;
-                if (cb >= nrb || !((longblocks >> rb) & 1) || cb > reach[rb]) continue;
-                gram_block<false>(sbase, hs, rb, cb, lane, acc);
-                if (tau < 0.f) threshold_block<true, false>(acc, rb, cb, lane, tau, norm, send, adj);
-                else threshold_block<false, false>(acc, rb, cb, lane, tau, norm, send, adj);
-            }
-            __syncthreads();
+            if (*umma_failed) { failed = true; break; }
         }
 
         // ---- 3. the service warp draws the block's next ticket; compute warps: Algorithm 1 per segment,
@@ -907,7 +909,7 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 }
             }
         }
-        if (tid < kNW) reach[tid] = 0;
+        if (tid < kNW) umma_rows[tid] = 0u;
         if (tid == kNW) misc[2] = misc[3] = 0;
         if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
         fence_async_proxy();   // the next tile's copies overwrite what ordinary accesses read and wrote
@@ -923,7 +925,9 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         mbar_wait(bar_v, phase_v ^ 1u);
         mbar_wait(bar_v, phase_v);
     }
+    umma::fence_before_sync();
     __syncthreads();
+    if (warp == kWarps) umma::tmem_dealloc(tmem, kTmemCols);
     // Under an overlapped launch a block does not finish before the kernel enqueued ahead of this one has
     // completed, so completion is transitive along a run of overlapped launches (a no-op otherwise).
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
@@ -1006,11 +1010,12 @@ int resident_blocks() {
         cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kWriteWithCounts, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
         cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kLookBack, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
         cudaFuncSetAttribute(cf::compress_fused_kernel<cf::kLookBack, cf::kMaxLayers>, cudaFuncAttributeMaxDynamicSharedMemorySize, cf::kSmemBytes);
-        int sms = 0, per_sm = 0;
+        // Blocks per SM by construction: launch bounds (registers), 75 KB of shared memory and 128 of the 512
+        // tensor-memory columns each.  (The occupancy query answers 1 for a kernel that allocates tensor memory.)
+        // Launching more blocks than are resident would be harmless: a block draws its first ticket when it starts.
+        int sms = 0;
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cf::compress_fused_kernel<cf::kLookBack, 1>, cf::kThreads,
-                                                      cf::kSmemBytes);
-        grid_of[dev] = (sms < 1 ? 1 : sms) * (per_sm < 1 ? 1 : per_sm);
+        grid_of[dev] = (sms < 1 ? 1 : sms) * cf::kBlocksPerSm;
     }
     return grid_of[dev];
 }
