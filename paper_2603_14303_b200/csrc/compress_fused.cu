@@ -12,12 +12,13 @@
 //      triangle of its Gram matrix (bf16 products are exact in fp32), the diagonal gives the norms,
 //      Sim > tau is decided as G_ij > tau*|k_i|*|k_j|, each lane ends up with one row's adjacency
 //      word, and the greedy pass costs one shuffle and a few word operations per seed;
-//   3. a segment of 33..kWarpSegMax (48) tokens is still one warp's own business: it builds the bit rows of the
-//      segment in 16-row bands in shared memory and runs the greedy pass on them; beyond that
-//      the Gram matrix is cut into 32x32 blocks (exactly the block pairs the segment spans) that all
-//      warps share, and one warp runs the greedy pass with one lane per 32-token word.  The
-//      adjacency bits live in an upper triangle of 32-bit words per row; a seed's row ends up
-//      holding its member mask;
+//   3. a tile that holds a segment of more than 32 tokens gets its whole Gram matrix from the tensor core first:
+//      one thread issues eight tcgen05.mma (128 x 128 x 128, bf16) on the staged rows -- the 128-byte-swizzled
+//      layout the TMA boxes wrote is the K-major operand layout -- into tensor memory (three such blocks for a
+//      tile of 129..256 tokens, diagonal blocks first: they give the norms); four warps read the accumulator one
+//      row per thread and write the adjacency bits of the long segments' rows (an upper triangle of 32-bit words
+//      per row); one warp per segment then runs the greedy pass on the bit rows with one lane per 32-token word,
+//      and a seed's row ends up holding its member mask;
 //   4. the tile's cluster count enters a prefix sum over the tiles of its (sequence, head): a
 //      decoupled look-back over per-tile status words (tickets are handed out in order, so every
 //      predecessor is held by a running block and the bounded wait cannot starve), or, in
@@ -53,11 +54,9 @@ constexpr int kBoxRows = 32;                      // rows per TMA box
 constexpr int kBoxBytes = kBoxRows * kHalfRow;    // 4096
 constexpr int kMaxRows = SC_MAX_CHUNK_LEN;        // 256: a long tile
 constexpr int kShortRows = SC_TILE_ROWS;          // 128
-// Longest segment one warp clusters on its own; longer ones share their Gram blocks among all warps.  The
-// warp-private code handles up to 64 tokens, but a tile that waits for one warp to finish a long segment
-// also holds up the tiles that look back to it: 48 measured best on every workload (32 and 40 were slower
-// for Poisson(30) chunks, 56 and 64 for lognormal ones).
-constexpr int kWarpSegMax = 48;
+// Longest segment one warp clusters on its own, in registers; the bit rows of longer ones come from the tile's Gram
+// matrix on the tensor core.  (A warp-private mma.sync path for 33..48 tokens was 16 % slower on lognormal chunks.)
+constexpr int kWarpSegMax = 32;
 constexpr int kNW = 8;                            // 32-bit words per (full) adjacency row
 constexpr int kKvBytes = kMaxRows * kRowBytes;    // 65536: short = K | V, long = one tensor
 constexpr int kVOff = kShortRows * kRowBytes;     // 32768
@@ -505,84 +504,6 @@ __device__ __forceinline__ void stage_rows(uint32_t dst, int hs, const CUtensorM
     }
 }
 
-// Eq. 2 for one segment of 33..64 tokens [a, a + l) (the kernel sends it up to kWarpSegMax), by one warp on its own (no block-level step):
-// the upper triangle of the segment's Gram matrix in 16-row bands, last band first so that the
-// norms a band needs (its own rows', from its diagonal, and those of all later rows) are known
-// when it is thresholded.  Every row's adjacency bits (later tokens of the segment) go to its
-// words of the tile's bit rows, where the greedy pass for longer segments reads them.
-template <bool kNegTau>
-__device__ __forceinline__ void gram_mid_segment(uint32_t kbase, int hs, int a, int l, float tau, float* nrm /*[64], this warp's*/,
-                                                 uint32_t* adj, int lane) {
-    const int g = lane >> 2, tig = lane & 3;
-    const int nnt = (l + 7) >> 3, nmt = (l + 15) >> 4;   // 5..8 column tiles, 3..4 row bands
-    const int j = lane >> 3, r8 = lane & 7;
-    const int sh = a & 31, wb = a >> 5, w_end = (a + l - 1) >> 5;
-#pragma unroll
-    for (int mt = 3; mt >= 0; --mt) {
-        if (mt >= nmt) continue;
-        float acc[8][4];
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-        const uint32_t a_base = kbase + tile_addr(a + mt * 16 + r8 + ((j & 1) << 3), j >> 1);
-        const uint32_t b_base = kbase + tile_addr(a + r8 + ((j >> 1) << 3), j & 1);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t kx = (ks & 3) << 5, ko = (ks >> 2) * hs;
-            uint32_t a0, a1, a2, a3;
-            ldmatrix_x4((a_base ^ kx) + ko, a0, a1, a2, a3);
-#pragma unroll
-            for (int np = 0; np < 4; ++np) {
-                if (np < mt || 2 * np >= nnt) continue;   // left of the band's diagonal, or past the segment
-                uint32_t b0, b1, b2, b3;
-                ldmatrix_x4((b_base ^ kx) + ko + np * 16 * kHalfRow, b0, b1, b2, b3);
-                mma_bf16(acc[2 * np], a0, a1, a2, a3, b0, b1);
-                if (2 * np + 1 < nnt) mma_bf16(acc[2 * np + 1], a0, a1, a2, a3, b2, b3);
-            }
-        }
-        if ((g >> 1) == tig) {   // the band's own norms, from its diagonal
-            const int e = g & 1;
-            nrm[mt * 16 + g] = sqrtf(e ? acc[2 * mt][1] : acc[2 * mt][0]);
-            nrm[mt * 16 + 8 + g] = sqrtf(e ? acc[2 * mt + 1][3] : acc[2 * mt + 1][2]);
-        }
-        __syncwarp();
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-            const int i = mt * 16 + hh * 8 + g;        // token of the segment
-            const float ni = nrm[i];
-            uint32_t lo = 0u, hi = 0u;
-#pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                if (nt < 2 * mt + hh || nt >= nnt) continue;
-                const float2 nn = *reinterpret_cast<const float2*>(nrm + nt * 8 + 2 * tig);
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const float thr = ni * (tau * (e ? nn.y : nn.x));
-                    bool hit = acc[nt][hh * 2 + e] > thr;
-                    if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
-                    if (hit) { if (nt < 4) lo |= 1u << (nt * 8 + e); else hi |= 1u << ((nt - 4) * 8 + e); }
-                }
-            }
-            lo <<= 2 * tig; hi <<= 2 * tig;
-            lo |= __shfl_xor_sync(kFull, lo, 1); hi |= __shfl_xor_sync(kFull, hi, 1);
-            lo |= __shfl_xor_sync(kFull, lo, 2); hi |= __shfl_xor_sync(kFull, hi, 2);
-            if (tig == 0 && i < l) {
-                // later tokens of the segment only: bits (i, l)
-                const unsigned long long keep = (i >= 63 ? 0ull : (~0ull << (i + 1))) & (l >= 64 ? ~0ull : ((1ull << l) - 1ull));
-                const unsigned long long m = (((unsigned long long)hi << 32) | lo) & keep;
-                // to tile positions: shift by a; row a + i keeps words (a + i) >> 5 .. w_end
-                const uint32_t t0 = (uint32_t)(m << sh), t1 = (uint32_t)((m << sh) >> 32),
-                               t2 = sh ? (uint32_t)((m >> 32) >> (32 - sh)) : 0u;
-                const int wi = (a + i) >> 5;
-                uint32_t* row = adj + adj_row(a + i) - wi;
-                if (wb >= wi) row[wb] = t0;
-                if (wb + 1 >= wi && wb + 1 <= w_end) row[wb + 1] = t1;
-                if (wb + 2 >= wi && wb + 2 <= w_end) row[wb + 2] = t2;
-            }
-        }
-        __syncwarp();
-    }
-}
-
 // The same for the second tensor of a tile longer than SC_TILE_ROWS (V staged where K was): one
 // segment [a, e), seeds in seedmask, member masks in the seeds' adjacency rows, counts already known.
 __device__ __forceinline__ void merge_long_segment(unsigned char* lane_base, int a, int e, const uint32_t* seedmask,
@@ -763,10 +684,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                     if (tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
                     else gsc_short_segment<false>(sbase, hs, a, e - a, tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
                     continue;
-                }
-                if (e - a <= kWarpSegMax) {   // the warp builds the segment's bit rows itself
-                    if (tau < 0.f) gram_mid_segment<true>(sbase, hs, a, e - a, tau, norm + warp * 64, adj, lane);
-                    else gram_mid_segment<false>(sbase, hs, a, e - a, tau, norm + warp * 64, adj, lane);
                 }
                 const int w1 = (e - 1) >> 5;
                 uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
