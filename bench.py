@@ -798,32 +798,37 @@ def run_e2e(pipe, args, barrier, g_decode):
 # -------------------------------------------------------------------------- oracle (cpu) arm
 
 
-def oracle_sample(w: synth.Workload, n_decode: int = 2):
-    """Time the oracle on layer 0 of the workload: compress once, n_decode decode steps.
+def oracle_sample(w: synth.Workload, n_decode: int = 2, layers=(0,)):
+    """Time the oracle on some layers of the workload: compress each once, then n_decode decode steps on it.
 
-    Returns (seconds for chunk+compress of one layer, seconds per one-layer decode step)."""
+    Returns (seconds for chunk+compress of one layer, seconds per one-layer decode step), means over the layers."""
     import oracle
     ids, run_id, run_lens = synth.token_ids(w)
-    K, V = synth.layer_kv(w, 0, run_id, run_lens)
-    Kb, Vb = synth.to_numpy_bits(K), synth.to_numpy_bits(V)
-    t0 = time.perf_counter()
-    r = oracle.compress(ids.numpy(), w.delims, Kb, Vb, w.tau, w.max_chunk_len, cap=w.n)
-    t_c = time.perf_counter() - t0
-    t_d = 0.0
-    for s in range(n_decode):
-        q = synth.to_numpy_bits(synth.queries(w, s, 0))
+    t_c = t_d = 0.0
+    for l in layers:
+        K, V = synth.layer_kv(w, l, run_id, run_lens)
+        Kb, Vb = synth.to_numpy_bits(K), synth.to_numpy_bits(V)
         t0 = time.perf_counter()
-        oracle.attn(q, r["core_k"], r["core_v"], r["count"], r["core_len"])
-        t_d += time.perf_counter() - t0
-    return t_c, t_d / n_decode
+        r = oracle.compress(ids.numpy(), w.delims, Kb, Vb, w.tau, w.max_chunk_len, cap=w.n)
+        t_c += time.perf_counter() - t0
+        for s in range(n_decode):
+            q = synth.to_numpy_bits(synth.queries(w, s, l))
+            t0 = time.perf_counter()
+            oracle.attn(q, r["core_k"], r["core_v"], r["count"], r["core_len"])
+            t_d += time.perf_counter() - t0
+    return t_c / len(layers), t_d / (n_decode * len(layers))
 
 
 def cpu_baseline(w: synth.Workload, budget_s: float = 20.0):
+    """The oracle, as it stands, on a bounded sample of the workload: about budget_s / 2 seconds of timed CPU work
+    (a quick probe sizes the sample: as many layers and decode steps as fit), scaled linearly to the full step."""
     import oracle
     # shrink the batch so the sample stays bounded; the per-sequence cost is what gets scaled
     ws = w.replace(B=1) if w.B > 1 else w
-    t_c, t_d = oracle_sample(ws, n_decode=2)
-    del budget_s
+    p_c, p_d = oracle_sample(ws, n_decode=1)
+    n_layers = int(min(ws.L, 8, max(1, 0.25 * budget_s / max(p_c, 1e-6))))   # generating a layer's inputs is not free
+    n_decode = int(min(ws.decode_steps, max(2, 0.5 * budget_s / max(n_layers * p_d, 1e-6))))
+    t_c, t_d = oracle_sample(ws, n_decode=n_decode, layers=tuple(range(n_layers)))
     step_s = w.B * (w.L * t_c + w.decode_steps * w.L * t_d)
     threads = oracle.num_threads()
     # the oracle's loops run in parallel over (sequence, KV head) for chunk/GSC/merge and over (sequence, query
@@ -831,8 +836,10 @@ def cpu_baseline(w: synth.Workload, budget_s: float = 20.0):
     busy_c, busy_a = min(threads, ws.B * ws.Hkv), min(threads, ws.B * ws.Hq)
     return {"value": w.B * w.decode_steps / step_s, "unit": UNIT, "cores": max(busy_c, busy_a), "kind": "oracle",
             "threads_available": threads, "cores_with_work": {"chunk_gsc_merge": busy_c, "attention": busy_a},
-            "sample": f"layer 0 of {w.L}, sequence 0 of {w.B}: chunk+GSC+merge once ({t_c:.2f} s) and 2 of "
-                      f"{w.decode_steps} decode steps ({t_d * 1e3:.1f} ms each), scaled linearly to the full step",
+            "sample": f"layers 0..{n_layers - 1} of {w.L}, sequence 0 of {w.B}: chunk+GSC+merge of each layer "
+                      f"({t_c:.2f} s per layer) and {n_decode} of {w.decode_steps} decode steps on each "
+                      f"({t_d * 1e3:.1f} ms per layer and step): {n_layers * (t_c + n_decode * t_d):.1f} s of timed CPU "
+                      "work, scaled linearly to the full step",
             "compress_s_per_layer": t_c, "decode_s_per_layer_step": t_d}
 
 

@@ -12,13 +12,17 @@
 //      triangle of its Gram matrix (bf16 products are exact in fp32), the diagonal gives the norms,
 //      Sim > tau is decided as G_ij > tau*|k_i|*|k_j|, each lane ends up with one row's adjacency
 //      word, and the greedy pass costs one shuffle and a few word operations per seed;
-//   3. a tile that holds a segment of more than 32 tokens gets its whole Gram matrix from the tensor core first:
-//      one thread issues eight tcgen05.mma (128 x 128 x 128, bf16) on the staged rows -- the 128-byte-swizzled
-//      layout the TMA boxes wrote is the K-major operand layout -- into tensor memory (three such blocks for a
-//      tile of 129..256 tokens, diagonal blocks first: they give the norms); four warps read the accumulator one
-//      row per thread and write the adjacency bits of the long segments' rows (an upper triangle of 32-bit words
-//      per row); one warp per segment then runs the greedy pass on the bit rows with one lane per 32-token word,
-//      and a seed's row ends up holding its member mask;
+//   3. the rows of segments of more than 32 tokens get their similarities from the tensor core: one thread issues
+//      eight tcgen05.mma (128 x 128 x 128, bf16) on the staged rows -- the 128-byte-swizzled layout the TMA boxes
+//      wrote is the K-major operand layout -- into tensor memory (three such blocks for a tile of 129..256 tokens,
+//      the diagonal ones first: they give the norms); the warps that own such rows read the accumulator one row per
+//      thread and keep, as bits in registers, which EARLIER tokens of its segment each row is similar to.
+//      Algorithm 1 is then settled for all those rows at once, in rounds: a row with an earlier neighbour that is
+//      a seed is a member, a row whose earlier neighbours are all members is a seed (the lowest open row is decided
+//      in every round, so the rounds end; chunks that are unions of cliques take two).  A member joins the earliest
+//      seed among its neighbours, which is what the sequential pass does; the lanes of a warp that name the same
+//      seed are found with match.any and write that word of the seed's member mask.  Warps without such rows do
+//      the short segments meanwhile (segments are claimed from a counter, not dealt by warp number);
 //   4. the tile's cluster count enters a prefix sum over the tiles of its (sequence, head): a
 //      decoupled look-back over per-tile status words (tickets are handed out in order, so every
 //      predecessor is held by a running block and the bounded wait cannot starve), or, in
@@ -66,11 +70,11 @@ constexpr int kCntOff = kKvBytes;                 // uint32[256] per seed row: w
 constexpr int kAdjOff = kCntOff + kMaxRows * 4;
 constexpr int kAdjWords = 32 * (8 + 7 + 6 + 5 + 4 + 3 + 2 + 1);   // rows of block k keep words k..7
 constexpr int kNormOff = kAdjOff + kAdjWords * 4; // float[512]: norms (64 per warp, or one per row); later uint16 seed row per cluster
-constexpr int kSendOff = kNormOff + kWarps * 64 * 4; // uint16[256]: end of the segment a row is in
-constexpr int kSegsOff = kSendOff + kMaxRows * 2; // 2 x int16[132]: segment starts (this tile, next tile)
+constexpr int kRowNormOff = kNormOff + kWarps * 64 * 4; // float[256]: norms of the rows of long segments (from the tensor core's Gram diagonal)
+constexpr int kSegsOff = kRowNormOff + kMaxRows * 4; // 2 x int16[132]: segment starts (this tile, next tile)
 constexpr int kSegsStride = 132;
 constexpr int kMiscOff = kSegsOff + 2 * kSegsStride * 2;   // uint32 seedmask[8]; int geo[2][8]; int misc[4]
-constexpr int kBarOff = kMiscOff + 32 + 64 + 16 + 32 + 128 + 16;   // ... uint32 umma_rows[8]; uint8 multi[128]; tensor-memory slot, flag; three mbarriers
+constexpr int kBarOff = kMiscOff + 32 + 64 + 16 + 32 + 128 + 16 + 32;   // ... 8 spare words; uint8 multi[128]; tensor-memory slot, flag; uint32 membits[8]; three mbarriers
 constexpr int kSmemBytes = kBarOff + 24;
 constexpr int kTmemCols = 128;                    // one 128 x 128 fp32 accumulator per block (three blocks per SM: 384 of 512 columns)
 constexpr int kBlocksPerSm = 3;
@@ -201,38 +205,199 @@ __device__ __forceinline__ void umma_norms(uint32_t tmem, int mb, int q, int lan
     norm[mb * 128 + q * 32 + lane] = sqrtf(v);
 }
 
-// Turns the block in tensor memory into adjacency words of the rows that belong to long segments (umma_rows):
-// bit j of word (i, cb) = Sim(i, 32cb + j) > tau, limited to later tokens of i's own segment.
+// Reads this thread's row i = 128 mb + 32 q + lane of the block in tensor memory and returns, as four words over
+// the block's columns 128 nb .. 128 nb + 127, which EARLIER tokens of i's own segment [a_i, ...) are similar to it:
+// bit c of the result = Sim(c, i) > tau for a_i <= c < i, decided as G > |k_c| (tau |k_i|) -- the earlier token's
+// norm first, the product the short-segment path forms for the same pair.  Only the chunks of sixteen columns
+// that can hold a column below the warp's rows are read (`chunks`, uniform over the warp).
 template <bool kNegTau>
-__device__ __forceinline__ void umma_threshold(uint32_t tmem, int mb, int nb, int q, int lane, float tau, const float* norm,
-                                               const uint16_t* send, const uint32_t* umma_rows, uint32_t* adj) {
+__device__ __forceinline__ void umma_earlier(uint32_t tmem, int nb, int q, int i, int a_i, float tau, const float* norm,
+                                             int chunks, uint32_t (&words)[4]) {
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    const int i = mb * 128 + q * 32 + lane;
-    const float ni = norm[i];
-    uint32_t words[4] = {0u, 0u, 0u, 0u};
+    const float tni = tau * norm[i];
+    words[0] = words[1] = words[2] = words[3] = 0u;
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-        uint32_t g[16];
-        tmem_ld16(lane_addr + c * 16, g);
-        umma::tmem_ld_wait();
-        uint32_t w = 0u;
+        if (c < chunks) {
+            uint32_t g[16];
+            tmem_ld16(lane_addr + c * 16, g);
+            umma::tmem_ld_wait();
+            uint32_t w = 0u;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            const float thr = ni * (tau * norm[nb * 128 + c * 16 + k]);
-            bool hit = __uint_as_float(g[k]) > thr;
-            if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
-            w |= (hit ? 1u : 0u) << k;
-        }
-        words[c >> 1] |= w << ((c & 1) * 16);
-    }
-    if ((umma_rows[i >> 5] >> (i & 31)) & 1u) {
-        const int e_i = (int)send[i], rb = i >> 5;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const int cb = nb * 4 + c;
-            if (cb >= rb && e_i > i + 1) adj[adj_row(i) + (cb - rb)] = words[c] & bits_between(i + 1, e_i, cb);
+            for (int k = 0; k < 16; ++k) {
+                const float thr = norm[nb * 128 + c * 16 + k] * tni;
+                bool hit = __uint_as_float(g[k]) > thr;
+                if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
+                w |= (hit ? 1u : 0u) << k;
+            }
+            words[c >> 1] |= w << ((c & 1) * 16);
         }
     }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) words[c] &= bits_between(a_i, i, nb * 4 + c);
+}
+
+// One round of Algorithm 1's decisions for the 32 tokens a warp owns (tile word `word`, token 32 word + lane),
+// on each token's earlier-neighbour words `e`: a token with an earlier neighbour that is a seed is a member; a
+// token whose earlier neighbours are all members is a seed.  Both facts are final once true, so reading words
+// that other warps are updating is harmless.  `open` = not yet decided (false for tokens outside long segments);
+// the warp's new seeds and members go to the shared words with one atomic each.
+template <int NW>
+__device__ __forceinline__ void decide_round(const uint32_t (&e)[NW], int word, int lane, bool& open, bool& is_seed,
+                                             volatile uint32_t* seeds, volatile uint32_t* members) {
+    bool to_member = false, to_seed = false;
+    if (open) {
+        bool has_seed = false, all_members = true;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) {
+            if (e[w] != 0u) {
+                has_seed = has_seed || (e[w] & seeds[w]) != 0u;
+                all_members = all_members && (e[w] & ~members[w]) == 0u;
+            }
+        }
+        to_member = has_seed;
+        to_seed = !has_seed && all_members;
+        if (to_member || to_seed) open = false;
+        if (to_seed) is_seed = true;
+    }
+    const uint32_t nm = __ballot_sync(kFull, to_member), ns = __ballot_sync(kFull, to_seed);
+    if (lane == 0) {
+        if (nm) atomicOr(const_cast<uint32_t*>(members) + word, nm);
+        if (ns) atomicOr(const_cast<uint32_t*>(seeds) + word, ns);
+    }
+}
+
+// After the rounds: a member joins the earliest seed among its earlier neighbours, as Algorithm 1 would have it.
+// The lanes of a warp that name the same seed are that cluster's members in the warp's word: one of them writes
+// the word into the seed's row of the triangular store (the seed's member mask, tile positions; the seed itself
+// is in it).  Words of the row that get no member were cleared beforehand.
+template <int NW>
+__device__ __forceinline__ void settle_round(const uint32_t (&e)[NW], int word, int lane, bool active, bool is_seed,
+                                             int a_i, int e_i, const volatile uint32_t* seeds, uint32_t* adj,
+                                             uint32_t* cnts, int32_t* as, int row0) {
+    const int i = word * 32 + lane;
+    int s = active ? i : -1 - lane;   // inactive lanes: keys of their own
+    if (active && !is_seed) {
+#pragma unroll
+        for (int w = NW - 1; w >= 0; --w) {
+            const uint32_t m = e[w] & seeds[w];
+            if (m) s = w * 32 + __ffs(m) - 1;
+        }
+    }
+    const uint32_t group = __match_any_sync(kFull, s);
+    if (!active) return;
+    if (is_seed) cnts[i] = kPending | (uint32_t)a_i | ((uint32_t)e_i << 9);
+    if ((int)(__ffs(group) - 1) == lane) adj[adj_row(s) + word - (s >> 5)] = group;
+    if (as) as[i] = row0 + s;
+}
+
+// `threads` threads of the block (whole warps) meet at barrier 2 ...
+__device__ __forceinline__ void warps_sync(int threads) { asm volatile("barrier.cta.sync 2, %0;\n" ::"r"(threads) : "memory"); }
+// ... and learn whether any of them still has work.
+__device__ __forceinline__ bool warps_any(bool mine, int threads) {
+    uint32_t out;
+    asm volatile(
+        "{\n"
+        ".reg .pred p, r;\n"
+        "setp.ne.u32 p, %1, 0;\n"
+        "barrier.cta.red.or.pred r, 2, %2, p;\n"
+        "selp.u32 %0, 1, 0, r;\n"
+        "}\n"
+        : "=r"(out) : "r"(mine ? 1u : 0u), "r"(threads) : "memory");
+    return out != 0u;
+}
+
+// Step 2 for one tile: Algorithm 1 for the rows of segments of more than kWarpSegMax tokens (all threads of the
+// block call it; a wait for the tensor core that gave up is left in the tile's failure flag).  The Gram matrix comes
+// from the tensor core, 128 x 128 at a time into tensor memory: one block for a tile of up to 128 tokens, else the
+// two diagonal blocks -- they give the norms -- and the lower one.  Compute thread tid settles tile row tid: warps
+// 0..3 read the accumulator rows of block 0, warps 4..7 those of block 1 (a warp reaches the tensor-memory lanes of
+// its quarter, warp % 4), and keep which earlier tokens of its segment each row is similar to; Algorithm 1 is then
+// settled for all those rows at once in decision rounds.  `words` has a bit for every 32-row word of the tile that
+// a long segment touches: in a tile of up to 128 rows only those warps stay, the others (and the service warp, once
+// it has issued the product) leave at once for the short segments and the next ticket.  Kept out of line: its
+// registers are not the main loop's.
+__device__ __noinline__ void settle_long_segments(unsigned char* smem, int hs, const int16_t* segs, int nseg, int R,
+                                                  uint32_t words, uint32_t tmem, uint32_t phase_u, float tau,
+                                                  int32_t* as, int row0) {
+    uint32_t* cnts = reinterpret_cast<uint32_t*>(smem + kCntOff);
+    uint32_t* adj = reinterpret_cast<uint32_t*>(smem + kAdjOff);
+    float* norm = reinterpret_cast<float*>(smem + kRowNormOff);
+    uint32_t* seedmask = reinterpret_cast<uint32_t*>(smem + kMiscOff);
+    volatile int* umma_failed = reinterpret_cast<volatile int*>(smem + kMiscOff + 276);
+    uint32_t* membits = reinterpret_cast<uint32_t*>(smem + kMiscOff + 288);
+    const uint32_t sbase = smem_u32(smem), bar_u = sbase + kBarOff + 16;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, q = warp & 3;
+    const bool service = warp == kWarps;
+    const bool long_tile = R > kShortRows;
+    if (!long_tile) {
+        if (service) {
+            if (lane == 0) {
+                umma::fence_after_sync();
+                umma_gram_block(sbase, hs, 0, 0, tmem, bar_u);
+            }
+            return;
+        }
+        if (!((words >> warp) & 1u)) return;
+    }
+    const int team = long_tile ? kWarps * 32 : 32 * __popc(words & 0xffu);   // threads that meet at barrier 2
+    // the segment [beg, end) this thread's row is in: the last start that is not beyond the row
+    int beg = tid, end = tid;
+    if (tid < R) {
+        int lo = 0, hi = nseg;   // segs[lo] <= tid < segs[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if ((int)segs[mid] <= tid) lo = mid; else hi = mid;
+        }
+        beg = segs[lo]; end = segs[hi];
+    }
+    const bool act = end - beg > kWarpSegMax;   // rows of shorter segments take no part
+    uint32_t ern[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};   // earlier neighbours of the row, tile words
+    if (!long_tile) {
+        if (!mbar_wait(bar_u, phase_u)) *umma_failed = 1;   // carry on (the barriers below must be met); the tile is dropped later
+        umma::fence_after_sync();
+        umma_norms(tmem, 0, q, lane, norm);
+        warps_sync(team);   // the norms of every row of a long segment are in place
+        uint32_t w4[4];
+        if (tau < 0.f) umma_earlier<true>(tmem, 0, q, tid, beg, tau, norm, 2 * q + 2, w4);
+        else umma_earlier<false>(tmem, 0, q, tid, beg, tau, norm, 2 * q + 2, w4);
+        ern[0] = w4[0]; ern[1] = w4[1]; ern[2] = w4[2]; ern[3] = w4[3];
+        umma::fence_before_sync();
+    } else {
+        for (int ps = 0; ps < 3; ++ps) {   // (0,0); (1,1), (1,0)
+            const int mb = ps == 0 ? 0 : 1, nb = ps == 1 ? 1 : 0;
+            const bool reader = !service && (warp >> 2) == mb;
+            if (service && lane == 0) {
+                umma::fence_after_sync();
+                umma_gram_block(sbase, hs, mb, nb, tmem, bar_u);
+            }
+            if (reader) {
+                if (!mbar_wait(bar_u, phase_u)) *umma_failed = 1;
+                umma::fence_after_sync();
+                if (mb == nb) umma_norms(tmem, mb, q, lane, norm);
+            }
+            phase_u ^= 1u;
+            __syncthreads();   // the norms are in place
+            if (reader) {
+                const int chunks = mb == nb ? 2 * q + 2 : 8;   // a diagonal block: columns below the warp's rows
+                uint32_t w4[4];
+                if (tau < 0.f) umma_earlier<true>(tmem, nb, q, tid, beg, tau, norm, chunks, w4);
+                else umma_earlier<false>(tmem, nb, q, tid, beg, tau, norm, chunks, w4);
+                if (nb == 0) { ern[0] = w4[0]; ern[1] = w4[1]; ern[2] = w4[2]; ern[3] = w4[3]; }
+                else { ern[4] = w4[0]; ern[5] = w4[1]; ern[6] = w4[2]; ern[7] = w4[3]; }
+                umma::fence_before_sync();
+            }
+            if (ps < 2) __syncthreads();   // the accumulator may be overwritten
+        }
+        if (service) return;
+    }
+    // the row's place in the triangular store will hold the member mask if the row is a seed
+    if (act) for (int ww = warp; ww <= (end - 1) >> 5; ++ww) adj[adj_row(tid) + ww - warp] = 0u;
+    bool open = act, is_seed = false;
+    do {
+        decide_round<8>(ern, warp, lane, open, is_seed, seedmask, membits);
+    } while (warps_any(open, team));   // the lowest open token is decided every round
+    settle_round<8>(ern, warp, lane, act, is_seed, beg, end, seedmask, adj, cnts, as, row0);
 }
 
 // Eq. 3 building blocks.  A lane owns eight consecutive columns (one 16-byte chunk) of the K row
@@ -536,17 +701,17 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
     uint32_t* adj = reinterpret_cast<uint32_t*>(smem + kAdjOff);
     float* norm = reinterpret_cast<float*>(smem + kNormOff);
     uint16_t* seedrow = reinterpret_cast<uint16_t*>(smem + kNormOff);   // reuses the norms once they are spent
-    uint16_t* send = reinterpret_cast<uint16_t*>(smem + kSendOff);
     int16_t* segs_buf = reinterpret_cast<int16_t*>(smem + kSegsOff);
     uint32_t* seedmask = reinterpret_cast<uint32_t*>(smem + kMiscOff);
     int* geo_buf = reinterpret_cast<int*>(smem + kMiscOff + 32);        // [2][8]
     int* misc = reinterpret_cast<int*>(smem + kMiscOff + 96);           // [0] output offset of the tile, [1] last block,
                                                                         // [2] 32-row blocks that a segment of > 32 tokens touches,
                                                                         // [3] number of segments of more than one token
-    uint32_t* umma_rows = reinterpret_cast<uint32_t*>(smem + kMiscOff + 112);   // [8] rows of segments of more than kWarpSegMax tokens
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + kMiscOff + 272);
     volatile int* umma_failed = reinterpret_cast<volatile int*>(smem + kMiscOff + 276);   // a wait for the tensor core gave up
+    int* claim = reinterpret_cast<int*>(smem + kMiscOff + 112);         // next entry of multi[] to be worked on
     uint8_t* multi = smem + kMiscOff + 144;                             // [128] the segments of more than one token
+    uint32_t* membits = reinterpret_cast<uint32_t*>(smem + kMiscOff + 288);     // [8] tokens of long segments known to be members
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bar_k = sbase + kBarOff, bar_v = bar_k + 8, bar_u = bar_k + 16;
 
@@ -580,9 +745,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         max_nt = warp_max_i(max_nt);
         fetch_tile(p, lane, max_nt, geo_buf, segs_buf);
     }
-    if (tid < kNW) umma_rows[tid] = 0u;
-    if (tid == kNW) misc[2] = misc[3] = 0;
-    if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
+    if (tid == kNW) { misc[2] = misc[3] = 0; *claim = 0; }
+    if (tid >= 32 && tid < 32 + kNW) { seedmask[tid - 32] = 0u; membits[tid - 32] = 0u; }
     __syncthreads();
     umma::fence_after_sync();
     const uint32_t tmem = *tmem_slot;
@@ -599,7 +763,6 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         const int unit = (NL == 1 ? 0 : geo[gLayer]) * p.B * p.Hkv + bh;   // index of this (layer, sequence, head)
         const bool long_tile = R > kShortRows;
         const bool two_tensors = (kMode != kCountOnly) && !long_tile;   // V staged beside K
-        const int nrb = (R + 31) >> 5;
         const int hs = long_tile ? kHalfLong : kHalfShort;
 
         // ---- 1. stage the rows (service warp, TMA); prefetch ahead ----
@@ -612,27 +775,21 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         // the others are listed for the warps
         int32_t* as = lr.assign ? lr.assign + (size_t)bh * p.n + row0 : nullptr;
         if (nseg == 1 && R > 1) {
-            for (int r = tid; r < R; r += kThreads) send[r] = (uint16_t)R;
-            if (R > kWarpSegMax && tid < nrb) { atomicOr(&misc[2], 1 << tid); umma_rows[tid] = bits_between(0, R, tid); }
-            if (tid == 0) { multi[0] = 0; misc[3] = 1; }
+            if (tid == 0) { multi[0] = 0; misc[3] = 1; if (R > kWarpSegMax) misc[2] = (int)((1u << ((R + 31) >> 5)) - 1u); }
         } else {
             for (int s = tid; s < nseg; s += kThreads) {
                 const int a = segs[s], e = segs[s + 1];
                 if (e - a == 1) {
-                    send[a] = (uint16_t)e;
                     cnts[a] = 1u;
                     atomicOr(&seedmask[a >> 5], 1u << (a & 31));
                     if (as) as[a] = row0 + a;
                     continue;
                 }
                 multi[atomicAdd(&misc[3], 1)] = (uint8_t)s;
-                if (e - a > kWarpSegMax) {   // only the block-level path reads send[] (of every row of the blocks it touches)
-                    for (int r = a; r < e; ++r) send[r] = (uint16_t)e;
-                    for (int k = a >> 5; k <= (e - 1) >> 5; ++k) { atomicOr(&misc[2], 1 << k); atomicOr(&umma_rows[k], bits_between(a, e, k)); }
-                }
+                if (e - a > kWarpSegMax)   // the tile takes the tensor-core step: which 32-row words it concerns
+                    for (int k = a >> 5; k <= (e - 1) >> 5; ++k) atomicOr(&misc[2], 1 << k);
             }
         }
-        for (int r = R + tid; r < nrb * 32; r += kThreads) send[r] = (uint16_t)0;
         failed = !mbar_wait(bar_k, phase_k);   // K has landed
         phase_k ^= 1u;
         if (two_tensors && !failed) {
@@ -642,76 +799,36 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
         if (__syncthreads_or(failed)) { failed = true; break; }
 
         // ---- 2. segments of more than kWarpSegMax tokens: the tile's Gram matrix on the tensor core, 128 x 128 at a
-        //         time into tensor memory (one block for a tile of up to 128 tokens; diagonal blocks first, they
-        //         give the norms), thresholded by four warps, one row per thread, into the bit rows ----
+        //         time into tensor memory (one block for a tile of up to 128 tokens, else the two diagonal blocks --
+        //         they give the norms -- and the lower one).  Four warps read it, one row per thread, and keep which
+        //         earlier tokens of its segment each row is similar to; Algorithm 1 is then settled for all those rows
+        //         at once in decision rounds (the sequential pass visits one seed at a time) ----
         if (misc[2] != 0) {
-            const int npass = R > 128 ? 3 : 1;   // (0,0); (1,1), (0,1)
-            for (int ps = 0; ps < npass; ++ps) {
-                const int mb = ps == 1 ? 1 : 0, nb = ps == 0 ? 0 : 1;
-                if (service && lane == 0) {
-                    umma::fence_after_sync();
-                    umma_gram_block(sbase, hs, mb, nb, tmem, bar_u);
-                }
-                if (warp < 4) {
-                    if (!mbar_wait(bar_u, phase_u)) *umma_failed = 1;
-                    umma::fence_after_sync();
-                    if (mb == nb) umma_norms(tmem, mb, warp, lane, norm);
-                }
-                phase_u ^= 1u;
-                __syncthreads();   // the norms are in place (and a wait that gave up is known to all)
-                if (*umma_failed) break;
-                if (warp < 4) {
-                    if (tau < 0.f) umma_threshold<true>(tmem, mb, nb, warp, lane, tau, norm, send, umma_rows, adj);
-                    else umma_threshold<false>(tmem, mb, nb, warp, lane, tau, norm, send, umma_rows, adj);
-                    umma::fence_before_sync();
-                }
-                __syncthreads();   // the bit rows are written; the accumulator may be overwritten
-            }
-            if (*umma_failed) { failed = true; break; }
+            settle_long_segments(smem, hs, segs, nseg, R, (uint32_t)misc[2], tmem, phase_u, tau, as, row0);
+            phase_u ^= 1u;   // one or three blocks
         }
 
-        // ---- 3. the service warp draws the block's next ticket; compute warps: Algorithm 1 per segment,
-        //         one warp each, in registers up to 32 tokens, else on the bit rows ----
+        // ---- 3. the service warp draws the block's next ticket; compute warps: Algorithm 1 for the segments of up
+        //         to 32 tokens, one warp each, in registers ----
         unsigned char* lane_base = smem + (lane >> 4) * kVOff + ((lane >> 3) & 1) * hs;   // see rows_add
         if (service) {
             fetch_tile(p, lane, max_nt, geo_buf + (buf ^ 1) * 8, segs_buf + (buf ^ 1) * kSegsStride);
         } else {
             const int nmulti = misc[3];
-            for (int k = warp; k < nmulti; k += kWarps) {
+            for (;;) {   // whichever warp is free takes the next segment
+                int k = 0;
+                if (lane == 0) k = atomicAdd(claim, 1);
+                k = __shfl_sync(kFull, k, 0);
+                if (k >= nmulti) break;
                 const int s = multi[k];
                 const int a = segs[s], e = segs[s + 1];
-                if (e - a <= 32) {
-                    if (tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
-                    else gsc_short_segment<false>(sbase, hs, a, e - a, tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
-                    continue;
-                }
-                const int w1 = (e - 1) >> 5;
-                uint32_t U = (lane < kNW) ? bits_between(a, e, lane) : 0u;   // unassigned tokens of this segment
-                uint32_t seeds = 0u;
-                for (int wf = a >> 5; wf <= w1;) {   // wf: first word that may still hold unassigned tokens
-                    const uint32_t u = __shfl_sync(kFull, U, wf);
-                    if (u == 0u) { ++wf; continue; }
-                    const int i = wf * 32 + __ffs(u) - 1;   // lowest unassigned token: a seed
-                    if (lane >= wf && lane <= w1) {
-                        uint32_t* slot = adj + adj_row(i) + (lane - wf);
-                        uint32_t mem = *slot & U;
-                        if (lane == wf) {
-                            mem |= 1u << (i & 31);
-                            seeds |= 1u << (i & 31);
-                            cnts[i] = kPending | (uint32_t)a | ((uint32_t)e << 9);
-                        }
-                        *slot = mem;            // the row now lists the cluster's members
-                        U &= ~mem;
-                        if (as) {
-                            uint32_t mm = mem;
-                            while (mm) { const int j = lane * 32 + __ffs(mm) - 1; mm &= mm - 1; as[j] = row0 + i; }
-                        }
-                    }
-                }
-                if (seeds) atomicOr(&seedmask[lane], seeds);
+                if (e - a > kWarpSegMax) continue;   // settled above
+                if (tau < 0.f) gsc_short_segment<true>(sbase, hs, a, e - a, tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
+                else gsc_short_segment<false>(sbase, hs, a, e - a, tau, norm + warp * 64, seedmask, adj, cnts, as, row0, lane);
             }
         }
         __syncthreads();
+        if (*umma_failed) { failed = true; break; }   // a wait for the tensor core gave up in step 2 (known to all by now)
 
         // ---- 4. cluster count of the tile, published at once.  Service warp: output offset of the tile
         //         (look-back).  Compute warps: the seed row of every cluster, and Eq. 3 ----
@@ -826,9 +943,8 @@ __global__ void __launch_bounds__(kThreads, 3) compress_fused_kernel(const __gri
                 }
             }
         }
-        if (tid < kNW) umma_rows[tid] = 0u;
-        if (tid == kNW) misc[2] = misc[3] = 0;
-        if (tid >= 32 && tid < 32 + kNW) seedmask[tid - 32] = 0u;
+            if (tid == kNW) { misc[2] = misc[3] = 0; *claim = 0; }
+        if (tid >= 32 && tid < 32 + kNW) { seedmask[tid - 32] = 0u; membits[tid - 32] = 0u; }
         fence_async_proxy();   // the next tile's copies overwrite what ordinary accesses read and wrote
         __syncthreads();
         buf ^= 1;

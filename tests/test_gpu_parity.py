@@ -251,6 +251,38 @@ def test_compress_near_ties_are_decided_consistently():
     compare_compressed(got, dict(core_k=ck, core_v=cv, count=cnt, core_len=clen, assign=assign), torch.bfloat16)
 
 
+@pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
+def test_compress_chain_similarity_in_long_segments(flags):
+    """Keys built from random sign vectors L_t: k_t = L_t + L_{t+1} is similar to its neighbours in the sequence
+    only (cos about 1/2 against about 0), k_t = L_t + L_{t+1} + L_{t+2} to the two on either side.  Along such a
+    chain whether a token is a seed depends on the token before it, all the way down the segment: the opposite
+    of chunks that are unions of cliques, and the deepest case for any scheme that settles Algorithm 1 for many
+    tokens at once.  Segments of 33..256 tokens (several in a tile, alone in a tile, across two 128-row blocks)."""
+    rng = np.random.default_rng(77)
+    delim, plain = synth.DELIMS[0], max(synth.DELIMS) + 1
+    lengths = [200, 256, 40, 100, 33, 129, 64, 20, 255, 128, 90, 37, 5, 161]
+    ids = []
+    for l in lengths:
+        ids += [plain] * l + [delim]
+    n, d = len(ids), 128
+    ids = torch.tensor([ids], dtype=torch.int32)
+    L = rng.choice([-1.0, 1.0], size=(2, n + 2, d))
+    K = torch.empty((1, 2, n, d), dtype=torch.bfloat16)
+    K[0, 0] = torch.from_numpy(L[0, :n] + L[0, 1:n + 1])                       # entries 0, +-2, +-3: exact in bf16
+    K[0, 1] = torch.from_numpy(L[1, :n] + L[1, 1:n + 1] + L[1, 2:n + 2])
+    V = torch.empty((1, 2, n, d), dtype=torch.bfloat16)
+    V[:] = torch.from_numpy(rng.normal(size=(1, 2, n, d)))
+    tau = 0.26
+    ref = oracle_compress(ids, K, V, synth.DELIMS, tau)
+    assert oracle.gsc(synth.to_numpy_bits(K), *oracle.chunk(ids.numpy(), synth.DELIMS, 256), tau)[1] > 2e-6   # no similarity within fp32 rounding of tau
+    # the structure is what the docstring says: about every other token of a plain chain is a seed
+    seeds = (ref["assign"][0, 0] == np.arange(n)).sum()
+    assert 0.4 * n < seeds < 0.7 * n
+    plan = binding.chunk(ids.to(DEV), synth.DELIMS)
+    got = binding.compress(K.to(DEV), V.to(DEV), plan, tau, want_assign=True, flags=flags)
+    compare_compressed(got, ref, torch.bfloat16)
+
+
 @pytest.mark.parametrize("n", [1, 5, 31, 33, 130])
 def test_compress_tiny_contexts(n):
     """Contexts shorter than a TMA box / a tile, two sequences and heads."""
