@@ -215,26 +215,28 @@ __device__ __forceinline__ void umma_earlier(uint32_t tmem, int nb, int q, int i
                                              int chunks, uint32_t (&words)[4]) {
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const float tni = tau * norm[i];
-    words[0] = words[1] = words[2] = words[3] = 0u;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        if (c < chunks) {
-            uint32_t g[16];
-            tmem_ld16(lane_addr + c * 16, g);
+    for (int c = 0; c < 4; ++c) {   // 32 columns = one word at a time
+        uint32_t w = 0u;
+        if (2 * c < chunks) {
+            uint32_t g[32];
+            umma::tmem_ld32(lane_addr + c * 32, g);
             umma::tmem_ld_wait();
-            uint32_t w = 0u;
+            const float4* nc = reinterpret_cast<const float4*>(norm + nb * 128 + c * 32);
 #pragma unroll
-            for (int k = 0; k < 16; ++k) {
-                const float thr = norm[nb * 128 + c * 16 + k] * tni;
-                bool hit = __uint_as_float(g[k]) > thr;
-                if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
-                w |= (hit ? 1u : 0u) << k;
+            for (int k4 = 0; k4 < 8; ++k4) {
+                const float4 nv = nc[k4];
+                const float thr[4] = {nv.x * tni, nv.y * tni, nv.z * tni, nv.w * tni};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    bool hit = __uint_as_float(g[k4 * 4 + k]) > thr[k];
+                    if (kNegTau) hit = hit || (thr[k] == 0.f);   // a zero-norm key has Sim = 0 > tau
+                    w |= (hit ? 1u : 0u) << (k4 * 4 + k);
+                }
             }
-            words[c >> 1] |= w << ((c & 1) * 16);
         }
+        words[c] = w & bits_between(a_i, i, nb * 4 + c);
     }
-#pragma unroll
-    for (int c = 0; c < 4; ++c) words[c] &= bits_between(a_i, i, nb * 4 + c);
 }
 
 // One round of Algorithm 1's decisions for the 32 tokens a warp owns (tile word `word`, token 32 word + lane),
@@ -242,24 +244,19 @@ __device__ __forceinline__ void umma_earlier(uint32_t tmem, int nb, int q, int i
 // token whose earlier neighbours are all members is a seed.  Both facts are final once true, so reading words
 // that other warps are updating is harmless.  `open` = not yet decided (false for tokens outside long segments);
 // the warp's new seeds and members go to the shared words with one atomic each.
-template <int NW>
-__device__ __forceinline__ void decide_round(const uint32_t (&e)[NW], int word, int lane, bool& open, bool& is_seed,
+__device__ __forceinline__ void decide_round(const uint32_t (&e)[8], int word, int lane, bool& open, bool& is_seed,
                                              volatile uint32_t* seeds, volatile uint32_t* members) {
-    bool to_member = false, to_seed = false;
-    if (open) {
-        bool has_seed = false, all_members = true;
+    // all lanes read the same sixteen words (broadcast), no branch per word
+    uint32_t sd[8], mb[8];
 #pragma unroll
-        for (int w = 0; w < NW; ++w) {
-            if (e[w] != 0u) {
-                has_seed = has_seed || (e[w] & seeds[w]) != 0u;
-                all_members = all_members && (e[w] & ~members[w]) == 0u;
-            }
-        }
-        to_member = has_seed;
-        to_seed = !has_seed && all_members;
-        if (to_member || to_seed) open = false;
-        if (to_seed) is_seed = true;
-    }
+    for (int w = 0; w < 8; ++w) { sd[w] = seeds[w]; mb[w] = members[w]; }
+    uint32_t near_seed = 0u, not_member = 0u;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { near_seed |= e[w] & sd[w]; not_member |= e[w] & ~mb[w]; }
+    const bool to_member = open && near_seed != 0u;
+    const bool to_seed = open && near_seed == 0u && not_member == 0u;
+    if (to_member || to_seed) open = false;
+    if (to_seed) is_seed = true;
     const uint32_t nm = __ballot_sync(kFull, to_member), ns = __ballot_sync(kFull, to_seed);
     if (lane == 0) {
         if (nm) atomicOr(const_cast<uint32_t*>(members) + word, nm);
@@ -271,15 +268,14 @@ __device__ __forceinline__ void decide_round(const uint32_t (&e)[NW], int word, 
 // The lanes of a warp that name the same seed are that cluster's members in the warp's word: one of them writes
 // the word into the seed's row of the triangular store (the seed's member mask, tile positions; the seed itself
 // is in it).  Words of the row that get no member were cleared beforehand.
-template <int NW>
-__device__ __forceinline__ void settle_round(const uint32_t (&e)[NW], int word, int lane, bool active, bool is_seed,
+__device__ __forceinline__ void settle_round(const uint32_t (&e)[8], int word, int lane, bool active, bool is_seed,
                                              int a_i, int e_i, const volatile uint32_t* seeds, uint32_t* adj,
                                              uint32_t* cnts, int32_t* as, int row0) {
     const int i = word * 32 + lane;
     int s = active ? i : -1 - lane;   // inactive lanes: keys of their own
     if (active && !is_seed) {
 #pragma unroll
-        for (int w = NW - 1; w >= 0; --w) {
+        for (int w = 7; w >= 0; --w) {
             const uint32_t m = e[w] & seeds[w];
             if (m) s = w * 32 + __ffs(m) - 1;
         }
@@ -395,9 +391,9 @@ __device__ __noinline__ void settle_long_segments(unsigned char* smem, int hs, c
     if (act) for (int ww = warp; ww <= (end - 1) >> 5; ++ww) adj[adj_row(tid) + ww - warp] = 0u;
     bool open = act, is_seed = false;
     do {
-        decide_round<8>(ern, warp, lane, open, is_seed, seedmask, membits);
+        decide_round(ern, warp, lane, open, is_seed, seedmask, membits);
     } while (warps_any(open, team));   // the lowest open token is decided every round
-    settle_round<8>(ern, warp, lane, act, is_seed, beg, end, seedmask, adj, cnts, as, row0);
+    settle_round(ern, warp, lane, act, is_seed, beg, end, seedmask, adj, cnts, as, row0);
 }
 
 // Eq. 3 building blocks.  A lane owns eight consecutive columns (one 16-byte chunk) of the K row
