@@ -399,11 +399,17 @@ __device__ __noinline__ void settle_long_segments(unsigned char* smem, int hs, c
 // Eq. 3 building blocks.  A lane owns eight consecutive columns (one 16-byte chunk) of the K row
 // (lanes 0-15) or of the V row (lanes 16-31); `lane_base` is its tensor and column half, c7 its
 // chunk inside the half.  Sums are fp32, in token order.
+// s0 += low bf16 of v, s1 += high bf16 of v: the mixed-precision add takes the bf16 operand as it is (exact
+// widening, one fp32 rounding of the sum -- what unpacking by hand and adding gives, in half the instructions).
+__device__ __forceinline__ void add_pair(uint32_t v, float& s0, float& s1) {
+    asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\nadd.rn.f32.bf16 %0, lo, %0;\nadd.rn.f32.bf16 %1, hi, %1;\n}\n"
+        : "+f"(s0), "+f"(s1) : "r"(v));
+}
 __device__ __forceinline__ void add_chunk(const uint4& v, float (&s)[8]) {
-    s[0] += __uint_as_float(v.x << 16); s[1] += __uint_as_float(v.x & 0xffff0000u);
-    s[2] += __uint_as_float(v.y << 16); s[3] += __uint_as_float(v.y & 0xffff0000u);
-    s[4] += __uint_as_float(v.z << 16); s[5] += __uint_as_float(v.z & 0xffff0000u);
-    s[6] += __uint_as_float(v.w << 16); s[7] += __uint_as_float(v.w & 0xffff0000u);
+    add_pair(v.x, s[0], s[1]);
+    add_pair(v.y, s[2], s[3]);
+    add_pair(v.z, s[4], s[5]);
+    add_pair(v.w, s[6], s[7]);
 }
 // Adds the rows first + j for every set bit j of mem, in order; two loads are kept in flight (the
 // filler of an odd count is a row of zeros, which leaves the sums as they are).
