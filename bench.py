@@ -515,7 +515,7 @@ def measure_extras(dev, sampler, peak):
     pre = {"what": "sc_prefill_attn: a block of m queries per head over the compressed cache, one launch per layer; "
                    "flops = 4 * (G*m) * core rows * d per KV head (scores + weighted sum)", "peak_tflops": tpeak,
            "peak_kind": tkind, "cells": []}
-    for m in (128, 512, 2048):
+    for m in (8, 128, 512, 2048):
         q = torch.randn((w.L, w.B, w.Hq, m, w.d), device=dev).to(torch.bfloat16)
         o = torch.empty_like(q)
         st = torch.zeros(1, dtype=torch.int32, device=dev)

@@ -323,7 +323,8 @@ SC_API sc_status sc_decode_attn(const void* q, sc_dtype dt, int32_t B, int32_t H
  * no row gets zeros.  With m = 1 this is sc_decode_attn.
  * The G*m query rows that share a KV head are one dense contraction against that head's cores: SC_BF16
  * with d = 128 runs on the tensor cores (scores and accumulators in tensor memory), other types and
- * head sizes on a CUDA-core kernel.  No workspace.
+ * head sizes on a CUDA-core kernel.  With few query rows the keys of a head are shared out among the blocks
+ * of a thread-block cluster, which combine their partial results on chip.  No workspace.
  *
  *   q, out     [B, Hq, m, d] contiguous, dtype dt
  *   core_k/v, count (or NULL for all ones), cap, core_len, scale   as for sc_decode_attn

@@ -16,8 +16,14 @@
 //              came from: the 32 fp32 columns of a chunk of scores become 16 columns of packed leading
 //              parts and 16 of remainders, so P is double-buffered like S and never touches shared
 //              memory; finally O / l -> bf16 -> global.
+// When the launch has too few CTAs to fill the GPU (few query rows: speculative decoding, short chunks), the keys
+// of a head are split over the CTAs of a thread-block cluster: each walks its share of the key tiles, leaves its
+// unnormalised (m, l, O) in its own shared memory, and after a cluster barrier every CTA folds a slice of the
+// query rows out of all members' shared memory (distributed shared memory) and writes that slice of the output.
 // Every wait is bounded; a wait that gives up is reported through the status word.
 // A CUDA-core kernel (one warp per query) serves other dtypes and head sizes.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "umma.cuh"
 
@@ -26,6 +32,7 @@ namespace sc {
 namespace pf {
 
 using namespace umma;
+namespace cg = cooperative_groups;
 
 constexpr int kT = 128;                       // query rows per CTA, keys per tile
 constexpr int kHalf = kT * 128;               // 16384 bytes: one 64-column half of a [128 x 128] bf16 tile
@@ -37,6 +44,7 @@ constexpr int kStages = 3;                    // K/V ring
 constexpr int kSmQ = 0, kSmK = kTile, kSmV = (1 + kStages) * kTile, kSmLc = (1 + 2 * kStages) * kTile, kSmMx = kSmLc + 2 * kT * 4,
               kSmBar = kSmMx + 2 * kT * 4;
 constexpr int kSmemBytes = kSmBar + 256;
+constexpr int kMaxSplit = 8;                  // portable cluster size
 constexpr float kMaxSlack = 8.f;              // log2 units a score may exceed the running maximum before it is raised
 static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
@@ -44,7 +52,7 @@ struct Params {
     CUtensorMap map_q, map_k, map_v;          // rows x 128 bf16, boxes of 128 rows x 64 columns
     const int32_t* count; const int32_t* core_len;
     __nv_bfloat16* out;
-    int Hq, Hkv, m, cap, causal;
+    int Hq, Hkv, m, cap, causal, n_split;   // n_split: CTAs (= cluster size) that share the keys of one query tile
     float scale_log2;
     int32_t* status;
 };
@@ -86,11 +94,15 @@ __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 
 
 __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_constant__ Params p) {
     extern __shared__ __align__(1024) unsigned char smem[];   // the swizzle pattern repeats every 1024 bytes
-    const int qt = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int n_split = p.n_split, split = blockIdx.x % n_split;   // the CTAs of a cluster are consecutive in x
+    const int qt = blockIdx.x / n_split, h = blockIdx.y, b = blockIdx.z;
     const int G = p.Hq / p.Hkv, bh = b * p.Hkv + h;
     const int rows_total = G * p.m;                           // query rows of this (sequence, KV head)
     const int len = max(min(p.core_len[bh], p.cap), 0);
-    const int nt = (len + kT - 1) / kT;                       // key tiles
+    const int nt_all = (len + kT - 1) / kT;                   // key tiles of the head
+    const int per_split = (nt_all + n_split - 1) / n_split;
+    const int t_lo = min(split * per_split, nt_all);          // this CTA's tiles: [t_lo, t_lo + nt)
+    const int nt = min(t_lo + per_split, nt_all) - t_lo;
     const long long q_row0 = ((long long)b * p.Hq + (long long)h * G) * p.m + (long long)qt * kT;
     const uint32_t sbase = smem_u32(smem);
     if ((sbase & 1023u) != 0u) {   // the swizzled addressing assumes this; uniform over the block
@@ -133,7 +145,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
             mbar_expect_tx(q_full, kTile);
             tma_load_4d(sbase + kSmQ, &p.map_q, 0, (int)q_row0, 0, 0, q_full);
             tma_load_4d(sbase + kSmQ + kHalf, &p.map_q, 64, (int)q_row0, 0, 0, q_full);
-            const int row_base = bh * p.cap;
+            const int row_base = bh * p.cap + t_lo * kT;
             for (int t = 0; t < nt; ++t) {
                 const int s = t % kStages;
                 if (t >= kStages && !mbar_wait(kv_empty0 + 8 * s, ((t / kStages) - 1) & 1)) { *sh_fail = 1; break; }
@@ -206,7 +218,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
         float m_run = -INFINITY, l_run = 0.f;                 // l_run: this thread's keys only
         bool failed = false;
         for (int t = 0; t < nt; ++t) {
-            const int s = t & 1, st = t % kStages, j0 = t * kT, jw = j0 + wg * 64;   // jw: first key of this thread's half
+            const int s = t & 1, st = t % kStages, j0 = (t_lo + t) * kT, jw = j0 + wg * 64;   // jw: first key of this thread's half
             if (wg == 0) lc_s[s * kT + r] = (cnt != nullptr && j0 + r < len) ? lg2((float)max(cnt[j0 + r], 1)) : 0.f;
             if (!mbar_wait(s_full0 + 8 * s, (t >> 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
             fence_after_sync();
@@ -295,30 +307,99 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
         mx_s[wg * kT + r] = l_run;
         asm volatile("bar.sync 1, 256;\n" ::: "memory");
         const float l_row = l_run + mx_s[(wg ^ 1) * kT + r];
-        __nv_bfloat16* orow = p.out + (size_t)(q_row0 + r) * 128 + wg * 64;
-        const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
+        if (n_split == 1) {
+            __nv_bfloat16* orow = p.out + (size_t)(q_row0 + r) * 128 + wg * 64;
+            const float inv = l_row > 0.f ? 1.f / l_row : 0.f;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            uint32_t o[32];
-            if (nt > 0 && !failed) {
-                tmem_ld32(lane_addr + kColO + wg * 64 + c * 32, o);
-                tmem_ld_wait();
-            } else {
+            for (int c = 0; c < 2; ++c) {
+                uint32_t o[32];
+                if (nt > 0 && !failed) {
+                    tmem_ld32(lane_addr + kColO + wg * 64 + c * 32, o);
+                    tmem_ld_wait();
+                } else {
 #pragma unroll
-                for (int k = 0; k < 32; ++k) o[k] = 0u;
+                    for (int k = 0; k < 32; ++k) o[k] = 0u;
+                }
+                if (row_ok) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        uint4 v;
+                        v.x = pack2(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
+                        v.y = pack2(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
+                        v.z = pack2(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
+                        v.w = pack2(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + u * 8) = v;
+                    }
+                }
             }
-            if (row_ok) {
+        } else {
+            // this CTA's share of the keys: unnormalised O, m and l into its own shared memory (the K ring is spent)
+            float* part_o = reinterpret_cast<float*>(smem + kSmK);      // [128 rows][32 float4], float4 index ^ (row & 31)
+            float* part_ml = reinterpret_cast<float*>(smem + kSmV);     // [128] m, [128] l
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    uint4 v;
-                    v.x = pack2(__uint_as_float(o[8 * u]) * inv, __uint_as_float(o[8 * u + 1]) * inv);
-                    v.y = pack2(__uint_as_float(o[8 * u + 2]) * inv, __uint_as_float(o[8 * u + 3]) * inv);
-                    v.z = pack2(__uint_as_float(o[8 * u + 4]) * inv, __uint_as_float(o[8 * u + 5]) * inv);
-                    v.w = pack2(__uint_as_float(o[8 * u + 6]) * inv, __uint_as_float(o[8 * u + 7]) * inv);
-                    *reinterpret_cast<uint4*>(orow + c * 32 + u * 8) = v;
+            for (int c = 0; c < 2; ++c) {
+                uint32_t o[32];
+                if (nt > 0 && !failed) {
+                    tmem_ld32(lane_addr + kColO + wg * 64 + c * 32, o);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) o[k] = 0u;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int c4 = wg * 16 + c * 8 + u;
+                    *reinterpret_cast<uint4*>(part_o + r * 128 + ((c4 ^ (r & 31)) << 2)) = make_uint4(o[4 * u], o[4 * u + 1], o[4 * u + 2], o[4 * u + 3]);
+                }
+            }
+            if (wg == 0) { part_ml[r] = (nt > 0 && !failed) ? m_run : -INFINITY; part_ml[kT + r] = (nt > 0 && !failed) ? l_row : 0.f; }
+        }
+    }
+    if (n_split > 1) {
+        cg::cluster_group cluster = cg::this_cluster();
+        fence_before_sync();
+        cluster.sync();   // every member's partial is in its shared memory
+        if (warp >= 2) {
+            // this CTA folds query rows [split * R, (split + 1) * R) of the tile, R = 128 / n_split: one thread per
+            // (row, four output columns), reading that piece of every member's partial
+            const float* part_o = reinterpret_cast<const float*>(smem + kSmK);
+            const float* part_ml = reinterpret_cast<const float*>(smem + kSmV);
+            const int R = kT / n_split;
+            for (int it = tid - 64; it < R * 32; it += 256) {
+                const int r = split * R + (it >> 5), c4 = it & 31;
+                float mv[kMaxSplit], lv[kMaxSplit];
+                float4 ov[kMaxSplit];
+#pragma unroll
+                for (int j = 0; j < kMaxSplit; ++j) {
+                    const int src = j < n_split ? j : 0;
+                    const float* ml = cluster.map_shared_rank(part_ml, src);
+                    const float* po = cluster.map_shared_rank(part_o, src);
+                    mv[j] = j < n_split ? ml[r] : -INFINITY;
+                    lv[j] = j < n_split ? ml[kT + r] : 0.f;
+                    ov[j] = j < n_split ? *reinterpret_cast<const float4*>(po + r * 128 + ((c4 ^ (r & 31)) << 2)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                float gm = mv[0];
+#pragma unroll
+                for (int j = 1; j < kMaxSplit; ++j) gm = fmaxf(gm, mv[j]);
+                float lsum = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < kMaxSplit; ++j) {
+                    const float w = (mv[j] == -INFINITY) ? 0.f : ex2(mv[j] - gm);
+                    lsum = fmaf(w, lv[j], lsum);
+                    acc.x = fmaf(w, ov[j].x, acc.x); acc.y = fmaf(w, ov[j].y, acc.y);
+                    acc.z = fmaf(w, ov[j].z, acc.z); acc.w = fmaf(w, ov[j].w, acc.w);
+                }
+                if (qt * kT + r < rows_total) {
+                    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                    uint2 v;
+                    v.x = pack2(acc.x * inv, acc.y * inv);
+                    v.y = pack2(acc.z * inv, acc.w * inv);
+                    *reinterpret_cast<uint2*>(p.out + (size_t)(q_row0 + r) * 128 + c4 * 4) = v;
                 }
             }
         }
+        cluster.sync();   // every member's shared memory has been read: they may leave
     }
     __syncthreads();
     if (*sh_fail) {   // a wait gave up: report it and give copies still in flight one more bounded wait
@@ -398,12 +479,36 @@ cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
     const long long q_rows = (long long)a.B * a.Hq * a.m, c_rows = (long long)a.B * a.Hkv * a.cap;
     if (a.dt == SC_BF16 && a.d == 128 && !(a.flags & SC_FLAG_GENERIC) && a.cap > 0 && q_rows < 0x7fffffff &&
         c_rows < 0x7fffffff && a.Hkv <= 65535 && a.B <= 65535) {
-        static bool attr_set[64] = {false};
+        // per device: the opt-in to large dynamic shared memory, the SM count, and the largest cluster of these
+        // one-per-SM CTAs that can be scheduled
+        static int sms_of[64] = {0}, cmax_of[64] = {0};
         int dev = 0;
         cudaGetDevice(&dev);
-        if (!attr_set[dev & 63]) {
+        dev &= 63;
+        if (sms_of[dev] == 0) {
             cudaFuncSetAttribute(prefill_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-            attr_set[dev & 63] = true;
+            int v = 0;
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+            int cmax = 1;
+            for (int c = kMaxSplit; c > 1; c >>= 1) {
+                cudaLaunchConfig_t probe = {};
+                probe.gridDim = dim3(c, 1, 1);
+                probe.blockDim = dim3(kThreads);
+                probe.dynamicSmemBytes = kSmemBytes;
+                cudaLaunchAttribute pa[1];
+                pa[0].id = cudaLaunchAttributeClusterDimension;
+                pa[0].val.clusterDim.x = c; pa[0].val.clusterDim.y = 1; pa[0].val.clusterDim.z = 1;
+                probe.attrs = pa;
+                probe.numAttrs = 1;
+                int n_clusters = 0;
+                if (cudaOccupancyMaxActiveClusters(&n_clusters, prefill_umma_kernel, &probe) == cudaSuccess && n_clusters > 0) {
+                    cmax = c;
+                    break;
+                }
+            }
+            (void)cudaGetLastError();   // a refused probe is not an error of this call
+            cmax_of[dev] = cmax;
+            sms_of[dev] = v < 1 ? 1 : v;
         }
         Params p;
         p.count = a.count; p.core_len = a.core_len; p.out = (__nv_bfloat16*)a.out;
@@ -411,10 +516,24 @@ cudaError_t launch_prefill(const PrefillArgs& a, cudaStream_t st) {
         if (make_map_bf16_rows(&p.map_q, a.q, 0, 0, 128, 1, 1, q_rows, kT) &&
             make_map_bf16_rows(&p.map_k, a.core_k, 0, 0, 128, 1, 1, c_rows, kT) &&
             make_map_bf16_rows(&p.map_v, a.core_v, 0, 0, 128, 1, 1, c_rows, kT)) {
-            const dim3 grid((unsigned)((G * a.m + kT - 1) / kT), a.Hkv, a.B);
-            prefill_umma_kernel<<<grid, kThreads, kSmemBytes, st>>>(p);
+            // Few query tiles (short chunks, speculative decoding): split the keys over a cluster, as many ways as
+            // fill the GPU, but leave every CTA at least two key tiles of the capacity.
+            const long long ctas = (long long)((G * a.m + kT - 1) / kT) * a.Hkv * a.B;
+            int n_split = 1;
+            while (n_split * 2 <= cmax_of[dev] && ctas * n_split * 2 <= sms_of[dev] && (a.cap + kT - 1) / kT >= n_split * 4) n_split *= 2;
+            p.n_split = n_split;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)((G * a.m + kT - 1) / kT) * n_split, a.Hkv, a.B);
+            cfg.blockDim = dim3(kThreads);
+            cfg.dynamicSmemBytes = kSmemBytes;
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = n_split; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
             note_launches(1);
-            return cudaGetLastError();
+            return cudaLaunchKernelEx(&cfg, prefill_umma_kernel, p);
         }
     }
     const unsigned blocks = (unsigned)((q_rows + 3) / 4);

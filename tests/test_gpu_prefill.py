@@ -52,6 +52,18 @@ def test_prefill_tensor_core_path_shapes(G, m, causal):
     _check(q, ck, cv, cnt, clen, causal)
 
 
+@pytest.mark.parametrize("m,causal", [(1, False), (8, True), (33, False), (128, True)])
+def test_prefill_few_queries_split_the_keys_over_a_cluster(m, causal):
+    """Few query rows and a long cache: the keys of a head are shared out among the CTAs of a cluster (up to
+    eight), whose partial results are folded through distributed shared memory.  Heads that are empty, shorter
+    than one CTA's share, and full to capacity."""
+    rng = np.random.default_rng(500 + m)
+    B, Hkv, G, cap, d = 1, 3, 4, 4500, 128
+    ck, cv, cnt, clen = _random_cache(rng, B, Hkv, cap, d, "bf16", [[4500, 0 if not causal else m, 300]])
+    q = torch.from_numpy(rng.normal(size=(B, Hkv * G, m, d)).astype(np.float32)).to(torch.bfloat16)
+    _check(q, ck, cv, cnt, clen, causal)
+
+
 def test_prefill_sharp_scores_and_no_counts():
     """Large query norms make the softmax pick out few rows (the running maximum is raised many times);
     count = NULL is plain attention."""
