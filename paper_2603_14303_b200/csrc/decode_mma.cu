@@ -14,6 +14,9 @@
 // and fold their partials through distributed shared memory, each block its own slice of the
 // output (no partial leaves the SMs); otherwise, or when a head needs several clusters, partials go
 // to global memory and the last block of a head to arrive (atomic ticket, no waiting) merges them.
+// In such a launch of several waves the split count comes from the capacity, which the host knows; how many of
+// those blocks a head really uses is settled by each block from the head's length (about 1024 rows a block, but
+// enough blocks over the launch to fill the GPU three times): the others take their ticket and leave.
 // Every order is fixed, so results are bit-reproducible.
 //
 // Launch modes: ordinary; overlapped with the preceding kernel (programmatic stream
@@ -45,6 +48,7 @@ constexpr size_t kL2PrefetchBytes = 512 * 1024;  // per tensor and block
 constexpr float kMaxSlack = 8.f;                // log2 units a score may exceed the running maximum before it is raised
 constexpr int kMergeGroup = 16;                 // cluster partials folded per round by the merging block
 constexpr int kMaxCluster = 16;                 // blocks per cluster (more than 8 needs the non-portable opt-in)
+constexpr int kRowsPerBlock = 1024;              // rows a block should stream at least, where the head's length allows
 constexpr int kCapRowsPerSplit = 1408;           // of capacity (heads are usually half full or less): about 700 rows a block
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -137,10 +141,65 @@ __device__ __forceinline__ void issue_tile(uint32_t stage, const __nv_bfloat16* 
     }
 }
 
+// Several partials per head in global memory (one per cluster, or per block outside clusters): the last block
+// to arrive merges the first `n_parts` of them (the others belong to blocks that found no tiles).  All threads of
+// the block call it.  The cluster barrier / fence before the call orders this block's partial stores before its
+// ticket, whose release makes them visible to whoever reads the ticket with acquire (the last arrival); that
+// block's other threads are ordered behind its thread 0 by the barrier below and read the partials from L2.
+__device__ __forceinline__ void ticket_and_merge(const float* __restrict__ part, int32_t* __restrict__ tickets, int bh,
+                                                 int n_expected, int n_parts, int G, int Hq, int b, int h,
+                                                 __nv_bfloat16* __restrict__ out, int* sh_last_p) {
+    if (threadIdx.x == 0) {
+        int t;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;\n" : "=r"(t) : "l"(tickets + bh) : "memory");
+        *sh_last_p = (t == n_expected - 1);
+        if (*sh_last_p) tickets[bh] = 0;   // leave the counter ready for the next call
+    }
+    __syncthreads();
+    if (!*sh_last_p) return;
+    // One thread per (head, four output columns); the partials are folded sixteen at a time, all of a
+    // group's loads in flight together (one round trip to L2 per group).
+    const float* hp = part + (size_t)bh * n_expected * kPartStride;
+    for (int e4 = threadIdx.x; e4 < G * (kD / 4); e4 += kWarps * 32) {
+        const int hd = e4 / (kD / 4), d4 = (e4 % (kD / 4)) * 4;
+        float gm = -INFINITY, lsum = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s0 = 0; s0 < n_parts; s0 += kMergeGroup) {
+            float mv[kMergeGroup], lv[kMergeGroup];
+            float4 ov[kMergeGroup];
+#pragma unroll
+            for (int j = 0; j < kMergeGroup; ++j) {
+                const bool ok = s0 + j < n_parts;
+                const float* sp = hp + (size_t)(ok ? s0 + j : 0) * kPartStride;
+                mv[j] = ok ? __ldcg(sp + 8 * kD + hd) : -INFINITY;
+                lv[j] = ok ? __ldcg(sp + 8 * kD + 8 + hd) : 0.f;
+                ov[j] = ok ? __ldcg(reinterpret_cast<const float4*>(sp + hd * kD + d4)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            float cm = mv[0];
+#pragma unroll
+            for (int j = 1; j < kMergeGroup; ++j) cm = fmaxf(cm, mv[j]);
+            const float ngm = fmaxf(gm, cm);
+            if (ngm == -INFINITY) continue;   // nothing but empty splits so far
+            const float c = (gm == -INFINITY) ? 0.f : fast_exp2(gm - ngm);
+            lsum *= c; acc.x *= c; acc.y *= c; acc.z *= c; acc.w *= c;
+            gm = ngm;
+#pragma unroll
+            for (int j = 0; j < kMergeGroup; ++j) {
+                const float w = (mv[j] == -INFINITY) ? 0.f : fast_exp2(mv[j] - gm);
+                lsum = fmaf(w, lv[j], lsum);
+                acc.x = fmaf(w, ov[j].x, acc.x); acc.y = fmaf(w, ov[j].y, acc.y);
+                acc.z = fmaf(w, ov[j].z, acc.z); acc.w = fmaf(w, ov[j].w, acc.w);
+            }
+        }
+        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+        store_out4(out + ((size_t)b * Hq + (size_t)h * G + hd) * kD + d4, acc, inv);
+    }
+}
+
 __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
 decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __nv_bfloat16* __restrict__ core_k,
                   const __nv_bfloat16* __restrict__ core_v, const int32_t* __restrict__ count, int cap,
-                  const int32_t* __restrict__ core_len, float scale_log2, int n_split, int q_from_prev,
+                  const int32_t* __restrict__ core_len, float scale_log2, int n_split, int min_split, int q_from_prev,
                   __nv_bfloat16* __restrict__ out, float* __restrict__ part, int32_t* __restrict__ tickets) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ float sh_m[kWarps][8];
@@ -159,7 +218,17 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     const int len = max(min(core_len[bh], cap), 0);
     const int tiles_total = (len + kTile - 1) / kTile;
-    const int tiles_per_split = (tiles_total + n_split - 1) / n_split;
+    // The split count was chosen from the capacity; a head that is far from full is shared out among fewer blocks
+    // (about kRowsPerBlock rows each: shorter blocks are mostly prologue and merge), the others find no tiles and
+    // hand in an empty partial.  Not inside a cluster, whose blocks are few and fold on chip.
+    int eff_split = n_split;
+    if (cg::this_cluster().num_blocks() == 1) eff_split = min(n_split, max(min_split, (len + kRowsPerBlock - 1) / kRowsPerBlock));
+    const int tiles_per_split = (tiles_total + eff_split - 1) / eff_split;
+    if (split >= eff_split) {   // a block without tiles: it only takes its ticket (and merges, if it is the last)
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");   // no global write before the preceding kernel is complete
+        ticket_and_merge(part, tickets, bh, n_split, eff_split, G, Hq, b, h, out, &sh_last);
+        return;
+    }
     const int t0 = min(split * tiles_per_split, tiles_total);
     const int t1 = min(t0 + tiles_per_split, tiles_total);
     // this warp's tiles: t0 + warp, t0 + warp + kWarps, ...
@@ -366,6 +435,7 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
     const int n_clusters = n_split / csize, cidx = split / csize;   // clusters per head, this one's index
     float* my_part = part + ((size_t)bh * n_clusters + cidx) * kPartStride;
     const bool direct = n_clusters == 1;   // this cluster holds the whole head: its fold is the result
+    const int n_parts = csize == 1 ? eff_split : n_clusters;   // partials that hold something
     const int slice = (G * (kD / 4) + csize - 1) / csize;
     cluster.sync();
     // Nothing has been written to global memory so far (the block partials live in shared memory).  Under
@@ -411,56 +481,8 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
     cluster.sync();   // every member's shared memory has been read: they may leave
     if (direct || crank != 0) return;
 
-    // ---- several clusters per head: the last of them to arrive merges their partials ----
-    // The cluster barrier above orders every member's (fenced) partial stores before this block's
-    // ticket, whose release makes them visible to whoever reads the ticket with acquire (the last
-    // cluster); that block's other threads are ordered behind its thread 0 by the barrier below and read
-    // the partials from L2.
-    if (threadIdx.x == 0) {
-        int t;
-        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;\n" : "=r"(t) : "l"(tickets + bh) : "memory");
-        sh_last = (t == n_clusters - 1);
-        if (sh_last) tickets[bh] = 0;   // leave the counter ready for the next call
-    }
-    __syncthreads();
-    if (!sh_last) return;
-    // One thread per (head, four output columns); the partials are folded sixteen at a time, all of a
-    // group's loads in flight together (one round trip to L2 per group).
-    const float* hp = part + (size_t)bh * n_clusters * kPartStride;
-    for (int e4 = threadIdx.x; e4 < G * (kD / 4); e4 += kWarps * 32) {
-        const int hd = e4 / (kD / 4), d4 = (e4 % (kD / 4)) * 4;
-        float gm = -INFINITY, lsum = 0.f;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s0 = 0; s0 < n_clusters; s0 += kMergeGroup) {
-            float mv[kMergeGroup], lv[kMergeGroup];
-            float4 ov[kMergeGroup];
-#pragma unroll
-            for (int j = 0; j < kMergeGroup; ++j) {
-                const bool ok = s0 + j < n_clusters;
-                const float* sp = hp + (size_t)(ok ? s0 + j : 0) * kPartStride;
-                mv[j] = ok ? __ldcg(sp + 8 * kD + hd) : -INFINITY;
-                lv[j] = ok ? __ldcg(sp + 8 * kD + 8 + hd) : 0.f;
-                ov[j] = ok ? __ldcg(reinterpret_cast<const float4*>(sp + hd * kD + d4)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            float cm = mv[0];
-#pragma unroll
-            for (int j = 1; j < kMergeGroup; ++j) cm = fmaxf(cm, mv[j]);
-            const float ngm = fmaxf(gm, cm);
-            if (ngm == -INFINITY) continue;   // nothing but empty splits so far
-            const float c = (gm == -INFINITY) ? 0.f : fast_exp2(gm - ngm);
-            lsum *= c; acc.x *= c; acc.y *= c; acc.z *= c; acc.w *= c;
-            gm = ngm;
-#pragma unroll
-            for (int j = 0; j < kMergeGroup; ++j) {
-                const float w = (mv[j] == -INFINITY) ? 0.f : fast_exp2(mv[j] - gm);
-                lsum = fmaf(w, lv[j], lsum);
-                acc.x = fmaf(w, ov[j].x, acc.x); acc.y = fmaf(w, ov[j].y, acc.y);
-                acc.z = fmaf(w, ov[j].z, acc.z); acc.w = fmaf(w, ov[j].w, acc.w);
-            }
-        }
-        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-        store_out4(out + ((size_t)b * Hq + (size_t)h * G + hd) * kD + d4, acc, inv);
-    }
+    // ---- several partials per head: the last block to arrive merges them ----
+    ticket_and_merge(part, tickets, bh, n_clusters, n_parts, G, Hq, b, h, out, &sh_last);
 }
 
 // Block split of one head: how many blocks stream it, and how they are grouped into clusters.
@@ -489,7 +511,13 @@ inline SplitPlan plan_for(int B, int Hkv, int cap, int sms, int cmax) {
     // Several waves of blocks (many heads): a block that waits at a cluster barrier holds an SM slot the next
     // wave wants, and the merge is a small part of such a launch; there every block is a cluster of its own,
     // leaves its partial in global memory and goes (measured: clusters of 6 cost 7 % at 128 heads x 8K rows).
-    if ((long long)B * Hkv * s0 > 2LL * sms) return {s0, 1};
+    if ((long long)B * Hkv * s0 > 2LL * sms) {
+        // ... and the shares are cut finer (a head that is full streams kRowsPerBlock rows per block; how many of
+        // the blocks a shorter head uses is settled in the kernel, from its length)
+        const int fine = (cap + kRowsPerBlock - 1) / kRowsPerBlock;
+        const int s1 = fine > s0 ? fine : s0;
+        return {s1 > 256 ? 256 : s1, 1};
+    }
     if (s0 <= cmax + cmax / 4) { const int c = s0 < cmax ? s0 : cmax; return {c, c}; }
     const int k = (s0 + cmax - 1) / cmax, c = s0 / k;
     return {c * k, c};
@@ -507,9 +535,13 @@ size_t decode_mma_counter_bytes(int32_t B, int32_t Hkv) { return sizeof(int32_t)
 size_t decode_mma_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_t cap) {
     (void)Hq; (void)d;
     // tickets (one per (b, head), zero between calls) + partials for the largest split count
-    const int s = dm::splits_for(B, Hkv, cap, 256);
-    const int s2 = dm::splits_for(B, Hkv, cap, 132);
+    const int s = dm::plan_for(B, Hkv, cap, 256, dm::kMaxCluster).n_split;
+    const int s2 = dm::plan_for(B, Hkv, cap, 132, dm::kMaxCluster).n_split;
+    const int s3 = dm::plan_for(B, Hkv, cap, 132, 8).n_split;
     int smax = s > s2 ? s : s2;
+    if (s3 > smax) smax = s3;
+    const int fine = (cap + dm::kRowsPerBlock - 1) / dm::kRowsPerBlock;   // the finest split of a launch of several waves
+    if (fine > smax) smax = fine > 256 ? 256 : fine;
     return 256 + decode_mma_counter_bytes(B, Hkv) +
            sizeof(float) * (size_t)B * Hkv * smax * dm::kPartStride;
 }
@@ -560,10 +592,13 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
     cfg.attrs = attr;
     cfg.numAttrs = (a.flags & (SC_FLAG_OVERLAP_PREV | SC_FLAG_OVERLAP_CHAIN)) ? 2 : 1;
     const int q_from_prev = (a.flags & SC_FLAG_OVERLAP_CHAIN) ? 1 : 0;
+    // fewest blocks a head is shared out among, however short it is: three blocks per SM over the launch
+    const int heads = a.B * a.Hkv;
+    const int min_split = (3 * sms_of[dev] + heads - 1) / heads;
     note_launches(1);
     return cudaLaunchKernelEx(&cfg, dm::decode_mma_kernel, (const __nv_bfloat16*)a.q, a.Hq, a.Hkv,
                               (const __nv_bfloat16*)a.core_k, (const __nv_bfloat16*)a.core_v, a.count, a.cap,
-                              a.core_len, scale, plan.n_split, q_from_prev, (__nv_bfloat16*)a.out, part, tickets);
+                              a.core_len, scale, plan.n_split, min_split, q_from_prev, (__nv_bfloat16*)a.out, part, tickets);
 }
 
 }  // namespace sc

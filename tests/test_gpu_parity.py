@@ -403,6 +403,33 @@ def test_decode_gqa_shapes_ragged_lengths_and_plain_attention(Hkv, G, flags):
         assert torch.all(out[0, :G] == 0), "a head without cores yields zeros"
 
 
+def test_decode_many_heads_of_very_different_lengths_in_one_launch():
+    """A launch of several waves of blocks (many heads, a long capacity): the split count comes from the
+    capacity, and each head uses as many of its blocks as its own length warrants -- from none (empty head)
+    and one (a few rows) to all of them (a full head); the blocks left over only take their ticket, and any of
+    them may be the one that merges.  Two calls in a row on one workspace."""
+    rng = np.random.default_rng(4242)
+    B, Hkv, G, d, cap = 6, 8, 4, 128, 12000
+    g = torch.Generator(device=DEV)
+    g.manual_seed(99)
+    ck = torch.randn((B, Hkv, cap, d), generator=g, device=DEV).to(torch.bfloat16)
+    cv = torch.randn((B, Hkv, cap, d), generator=g, device=DEV).to(torch.bfloat16)
+    cnt = torch.randint(1, 40, (B, Hkv, cap), generator=g, device=DEV, dtype=torch.int32)
+    clen = torch.from_numpy(rng.integers(0, cap + 1, size=(B, Hkv)).astype(np.int32))
+    clen[0, 0], clen[0, 1], clen[0, 2], clen[1, 0], clen[5, 7] = 0, 1, 17, 1025, cap
+    clen[2] = torch.tensor([300, 700, 1024, 2048, 2049, 5000, 11999, 64], dtype=torch.int32)
+    q = torch.from_numpy(rng.normal(size=(B, Hkv * G, d)).astype(np.float32)).to(torch.bfloat16).to(DEV)
+    layer = binding.CompressedLayer(ck, cv, cnt, clen.to(DEV))
+    ws = binding.decode_workspace(B, Hkv * G, Hkv, d, cap, DEV)
+    want = oracle.attn(synth.to_numpy_bits(q), synth.to_numpy_bits(ck), synth.to_numpy_bits(cv), cnt.cpu().numpy(),
+                       clen.numpy())
+    first = binding.decode_attn(q, layer, workspace=ws)
+    again = binding.decode_attn(q, layer, workspace=ws)
+    assert_close_vectors(to_f64(first), want, 1e-2, "decode, heads of very different lengths")
+    assert torch.equal(first, again)
+    assert torch.all(first[0, :G] == 0), "a head without cores yields zeros"
+
+
 @pytest.mark.parametrize("flags", [0, binding.SC_FLAG_GENERIC])
 def test_decode_is_deterministic_and_scale_is_honoured(flags):
     w = synth.config(0, n=4096)
