@@ -15,7 +15,7 @@
 // output (no partial leaves the SMs); otherwise, or when a head needs several clusters, partials go
 // to global memory and the last block of a head to arrive (atomic ticket, no waiting) merges them.
 // In such a launch of several waves the split count comes from the capacity, which the host knows; how many of
-// those blocks a head really uses is settled by each block from the head's length (about 1024 rows a block, but
+// those blocks a head really uses is settled by each block from the head's length (about 1024 rows a block, 768 in the largest launches, but
 // enough blocks over the launch to fill the GPU three times): the others take their ticket and leave.
 // Every order is fixed, so results are bit-reproducible.
 //
@@ -48,7 +48,9 @@ constexpr size_t kL2PrefetchBytes = 512 * 1024;  // per tensor and block
 constexpr float kMaxSlack = 8.f;                // log2 units a score may exceed the running maximum before it is raised
 constexpr int kMergeGroup = 16;                 // cluster partials folded per round by the merging block
 constexpr int kMaxCluster = 16;                 // blocks per cluster (more than 8 needs the non-portable opt-in)
-constexpr int kRowsPerBlock = 1024;              // rows a block should stream at least, where the head's length allows
+constexpr int kRowsPerBlock = 1024;              // rows a block should stream at least, where the head's length allows ...
+constexpr int kRowsPerBlockBig = 768;            // ... in a launch over kBigLaunchRows rows of capacity (more, shorter blocks keep HBM busier there)
+constexpr long long kBigLaunchRows = 1300000;
 constexpr int kCapRowsPerSplit = 1408;           // of capacity (heads are usually half full or less): about 700 rows a block
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -199,7 +201,7 @@ __device__ __forceinline__ void ticket_and_merge(const float* __restrict__ part,
 __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
 decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __nv_bfloat16* __restrict__ core_k,
                   const __nv_bfloat16* __restrict__ core_v, const int32_t* __restrict__ count, int cap,
-                  const int32_t* __restrict__ core_len, float scale_log2, int n_split, int min_split, int q_from_prev,
+                  const int32_t* __restrict__ core_len, float scale_log2, int n_split, int min_split, int rows_block, int q_from_prev,
                   __nv_bfloat16* __restrict__ out, float* __restrict__ part, int32_t* __restrict__ tickets) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ float sh_m[kWarps][8];
@@ -219,10 +221,10 @@ decode_mma_kernel(const __nv_bfloat16* __restrict__ q, int Hq, int Hkv, const __
     const int len = max(min(core_len[bh], cap), 0);
     const int tiles_total = (len + kTile - 1) / kTile;
     // The split count was chosen from the capacity; a head that is far from full is shared out among fewer blocks
-    // (about kRowsPerBlock rows each: shorter blocks are mostly prologue and merge), the others find no tiles and
+    // (about rows_block rows each: shorter blocks are mostly prologue and merge), the others find no tiles and
     // hand in an empty partial.  Not inside a cluster, whose blocks are few and fold on chip.
     int eff_split = n_split;
-    if (cg::this_cluster().num_blocks() == 1) eff_split = min(n_split, max(min_split, (len + kRowsPerBlock - 1) / kRowsPerBlock));
+    if (cg::this_cluster().num_blocks() == 1) eff_split = min(n_split, max(min_split, (len + rows_block - 1) / rows_block));
     const int tiles_per_split = (tiles_total + eff_split - 1) / eff_split;
     if (split >= eff_split) {   // a block without tiles: it only takes its ticket (and merges, if it is the last)
         asm volatile("griddepcontrol.wait;\n" ::: "memory");   // no global write before the preceding kernel is complete
@@ -505,6 +507,8 @@ inline int splits_for(int B, int Hkv, int cap, int sms) {
 // when the whole launch is about one wave of blocks (few heads: the latency of the merge is then a large
 // part of the launch).  One cluster per head (no partial ever leaves the SMs) whenever the wanted split count is within a
 // quarter of the largest cluster; otherwise as few equal clusters as cover it.
+inline int rows_per_block(int B, int Hkv, int cap) { return (long long)B * Hkv * cap >= kBigLaunchRows ? kRowsPerBlockBig : kRowsPerBlock; }
+
 inline SplitPlan plan_for(int B, int Hkv, int cap, int sms, int cmax) {
     const int s0 = splits_for(B, Hkv, cap, sms);
     if (s0 <= 1 || cmax <= 1) return {s0, 1};
@@ -514,7 +518,8 @@ inline SplitPlan plan_for(int B, int Hkv, int cap, int sms, int cmax) {
     if ((long long)B * Hkv * s0 > 2LL * sms) {
         // ... and the shares are cut finer (a head that is full streams kRowsPerBlock rows per block; how many of
         // the blocks a shorter head uses is settled in the kernel, from its length)
-        const int fine = (cap + kRowsPerBlock - 1) / kRowsPerBlock;
+        const int rpb = rows_per_block(B, Hkv, cap);
+        const int fine = (cap + rpb - 1) / rpb;
         const int s1 = fine > s0 ? fine : s0;
         return {s1 > 256 ? 256 : s1, 1};
     }
@@ -540,7 +545,7 @@ size_t decode_mma_ws_bytes(int32_t B, int32_t Hq, int32_t Hkv, int32_t d, int32_
     const int s3 = dm::plan_for(B, Hkv, cap, 132, 8).n_split;
     int smax = s > s2 ? s : s2;
     if (s3 > smax) smax = s3;
-    const int fine = (cap + dm::kRowsPerBlock - 1) / dm::kRowsPerBlock;   // the finest split of a launch of several waves
+    const int fine = (cap + dm::kRowsPerBlockBig - 1) / dm::kRowsPerBlockBig;   // the finest split of a launch of several waves
     if (fine > smax) smax = fine > 256 ? 256 : fine;
     return 256 + decode_mma_counter_bytes(B, Hkv) +
            sizeof(float) * (size_t)B * Hkv * smax * dm::kPartStride;
@@ -598,7 +603,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, cudaStream_t st) {
     note_launches(1);
     return cudaLaunchKernelEx(&cfg, dm::decode_mma_kernel, (const __nv_bfloat16*)a.q, a.Hq, a.Hkv,
                               (const __nv_bfloat16*)a.core_k, (const __nv_bfloat16*)a.core_v, a.count, a.cap,
-                              a.core_len, scale, plan.n_split, min_split, q_from_prev, (__nv_bfloat16*)a.out, part, tickets);
+                              a.core_len, scale, plan.n_split, min_split, dm::rows_per_block(a.B, a.Hkv, a.cap), q_from_prev, (__nv_bfloat16*)a.out, part, tickets);
 }
 
 }  // namespace sc
