@@ -209,16 +209,17 @@ __device__ __forceinline__ void umma_norms(uint32_t tmem, int mb, int q, int lan
 // the block's columns 128 nb .. 128 nb + 127, which EARLIER tokens of i's own segment [a_i, ...) are similar to it:
 // bit c of the result = Sim(c, i) > tau for a_i <= c < i, decided as G > |k_c| (tau |k_i|) -- the earlier token's
 // norm first, the product the short-segment path forms for the same pair.  Only the chunks of sixteen columns
-// that can hold a column below the warp's rows are read (`chunks`, uniform over the warp).
+// that can hold a column below the warp's rows are read (`chunks`), and no word before the first (`w_lo`) that
+// holds a token of a segment one of the warp's rows is in (both uniform over the warp).
 template <bool kNegTau>
 __device__ __forceinline__ void umma_earlier(uint32_t tmem, int nb, int q, int i, int a_i, float tau, const float* norm,
-                                             int chunks, uint32_t (&words)[4]) {
+                                             int w_lo, int chunks, uint32_t (&words)[4]) {
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const float tni = tau * norm[i];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {   // 32 columns = one word at a time
         uint32_t w = 0u;
-        if (2 * c < chunks) {
+        if (c >= w_lo && 2 * c < chunks) {   // a word that holds an earlier token of some row's segment
             uint32_t g[32];
             umma::tmem_ld32(lane_addr + c * 32, g);
             umma::tmem_ld_wait();
@@ -355,8 +356,9 @@ __device__ __noinline__ void settle_long_segments(unsigned char* smem, int hs, c
         umma_norms(tmem, 0, q, lane, norm);
         warps_sync(team);   // the norms of every row of a long segment are in place
         uint32_t w4[4];
-        if (tau < 0.f) umma_earlier<true>(tmem, 0, q, tid, beg, tau, norm, 2 * q + 2, w4);
-        else umma_earlier<false>(tmem, 0, q, tid, beg, tau, norm, 2 * q + 2, w4);
+        const int w_lo = __reduce_min_sync(kFull, act ? beg >> 5 : kNW);   // first word any of the warp's rows needs
+        if (tau < 0.f) umma_earlier<true>(tmem, 0, q, tid, beg, tau, norm, w_lo, 2 * q + 2, w4);
+        else umma_earlier<false>(tmem, 0, q, tid, beg, tau, norm, w_lo, 2 * q + 2, w4);
         ern[0] = w4[0]; ern[1] = w4[1]; ern[2] = w4[2]; ern[3] = w4[3];
         umma::fence_before_sync();
     } else {
@@ -377,8 +379,8 @@ __device__ __noinline__ void settle_long_segments(unsigned char* smem, int hs, c
             if (reader) {
                 const int chunks = mb == nb ? 2 * q + 2 : 8;   // a diagonal block: columns below the warp's rows
                 uint32_t w4[4];
-                if (tau < 0.f) umma_earlier<true>(tmem, nb, q, tid, beg, tau, norm, chunks, w4);
-                else umma_earlier<false>(tmem, nb, q, tid, beg, tau, norm, chunks, w4);
+                if (tau < 0.f) umma_earlier<true>(tmem, nb, q, tid, beg, tau, norm, 0, chunks, w4);
+                else umma_earlier<false>(tmem, nb, q, tid, beg, tau, norm, 0, chunks, w4);
                 if (nb == 0) { ern[0] = w4[0]; ern[1] = w4[1]; ern[2] = w4[2]; ern[3] = w4[3]; }
                 else { ern[4] = w4[0]; ern[5] = w4[1]; ern[6] = w4[2]; ern[7] = w4[3]; }
                 umma::fence_before_sync();
