@@ -89,6 +89,13 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+// r0 = w0 - low bf16 of ph, r1 = w1 - high bf16 of ph, with the mixed-precision fma (the bf16 operands are taken
+// as they are: (-1) * h + w, one rounding -- what unpacking and subtracting gives, in half the instructions).
+__device__ __forceinline__ void remainders(uint32_t ph, float w0, float w1, float& r0, float& r1) {
+    asm("{\n.reg .b16 lo, hi, m1;\nmov.b32 {lo, hi}, %2;\nmov.b16 m1, 0xBF80;\n"
+        "fma.rn.f32.bf16 %0, lo, m1, %3;\nfma.rn.f32.bf16 %1, hi, m1, %4;\n}\n"
+        : "=f"(r0), "=f"(r1) : "r"(ph), "f"(w0), "f"(w1));
+}
 __device__ __forceinline__ float bf_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
@@ -111,6 +118,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
     }
     float* lc_s = reinterpret_cast<float*>(smem + kSmLc);     // [2][128] log2(count) of the tile's keys
     float* mx_s = reinterpret_cast<float*>(smem + kSmMx);     // [2][128] each half's row maximum (at the end the row sums)
+    int* lcm_s = reinterpret_cast<int*>(smem + kSmBar + 128);  // [2][4] largest log2(count) of a tile, per writing warp (float bits)
     const uint32_t bar0 = sbase + kSmBar;
     const uint32_t q_full = bar0, kv_full0 = bar0 + 8, kv_empty0 = bar0 + 32, s_full0 = bar0 + 56, p_full0 = bar0 + 72,
                    pv_done0 = bar0 + 88;
@@ -219,7 +227,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
         bool failed = false;
         for (int t = 0; t < nt; ++t) {
             const int s = t & 1, st = t % kStages, j0 = (t_lo + t) * kT, jw = j0 + wg * 64;   // jw: first key of this thread's half
-            if (wg == 0) lc_s[s * kT + r] = (cnt != nullptr && j0 + r < len) ? lg2((float)max(cnt[j0 + r], 1)) : 0.f;
+            if (wg == 0) {
+                const float lc = (cnt != nullptr && j0 + r < len) ? lg2((float)max(cnt[j0 + r], 1)) : 0.f;
+                lc_s[s * kT + r] = lc;
+                const int top = __reduce_max_sync(kFull, __float_as_int(lc));   // lc >= 0: the bits order like the values
+                if (lane == 0) lcm_s[s * 4 + q] = top;
+            }
             if (!mbar_wait(s_full0 + 8 * s, (t >> 1) & 1)) { *sh_fail = 1; *sh_fail_sm = 1; }
             fence_after_sync();
             asm volatile("bar.sync 1, 256;\n" ::: "memory");   // the eight softmax warps: log2(count) is in place
@@ -231,18 +244,36 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
                 for (int u = 0; u < 8; ++u)
                     *reinterpret_cast<uint4*>(smem + kSmV + st * kTile + wg * kHalf + r * 128 + u * 16) = make_uint4(0u, 0u, 0u, 0u);
             }
-            // pass 1: the row's largest score in this tile (each thread its half, then the two are exchanged)
+            // pass 1: a bound on the row's largest score in this tile (each thread its half, then the two are
+            // exchanged): the largest raw product times the scale plus the tile's largest log2(count).  Any reference
+            // at or above the true maximum serves the softmax; this one is at most log2 of the largest count above it,
+            // and costs one instruction per score.  (A scale that is not positive takes the exact form.)
             float mx = -INFINITY;
+            const bool all_seen = __all_sync(kFull, jw + 64 <= vis);   // no key of this half is masked for any row of the warp
+            const bool exact = !(p.scale_log2 > 0.f);
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t g[32];
                 tmem_ld32(lane_addr + kColS + s * kT + wg * 64 + c * 32, g);
                 tmem_ld_wait();
+                if (exact) {
 #pragma unroll
-                for (int k = 0; k < 32; ++k) {
-                    const float x = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k]);
-                    if (jw + c * 32 + k < vis) mx = fmaxf(mx, x);
+                    for (int k = 0; k < 32; ++k) {
+                        const float x = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k]);
+                        if (jw + c * 32 + k < vis) mx = fmaxf(mx, x);
+                    }
+                } else if (all_seen) {
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) mx = fmaxf(mx, __uint_as_float(g[k]));
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 32; ++k)
+                        if (jw + c * 32 + k < vis) mx = fmaxf(mx, __uint_as_float(g[k]));
                 }
+            }
+            if (!exact && mx != -INFINITY) {
+                const int top = max(max(lcm_s[s * 4], lcm_s[s * 4 + 1]), max(lcm_s[s * 4 + 2], lcm_s[s * 4 + 3]));
+                mx = fmaf(mx, p.scale_log2, __int_as_float(top));
             }
             mx_s[wg * kT + r] = mx;
             asm volatile("bar.sync 2, 256;\n" ::: "memory");   // both halves' maxima are in place
@@ -271,22 +302,39 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_umma_kernel(const __grid_
             }
             // pass 2: weights, as bf16 pairs (leading part + remainder), back into the score buffer's columns
             const float mref = m_run == -INFINITY ? 0.f : m_run;
+            // (the row sum takes the weights before the split: the pair carries sixteen bits of each, the difference
+            // is below 2^-17 of the sum)
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t g[32];
                 tmem_ld32(lane_addr + kColS + s * kT + wg * 64 + c * 32, g);
                 tmem_ld_wait();
                 uint32_t hi[16], lo[16];
+                if (all_seen) {   // no key of this half is masked for any row of the warp
 #pragma unroll
-                for (int k = 0; k < 32; k += 2) {
-                    const float x0 = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k]);
-                    const float x1 = fmaf(__uint_as_float(g[k + 1]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k + 1]);
-                    const float w0 = (jw + c * 32 + k < vis) ? ex2(x0 - mref) : 0.f;
-                    const float w1 = (jw + c * 32 + k + 1 < vis) ? ex2(x1 - mref) : 0.f;
-                    const uint32_t ph = pack2(w0, w1);
-                    const uint32_t pl = pack2(w0 - bf_lo(ph), w1 - bf_hi(ph));
-                    l_run += (bf_lo(ph) + bf_lo(pl)) + (bf_hi(ph) + bf_hi(pl));
-                    hi[k >> 1] = ph; lo[k >> 1] = pl;
+                    for (int k = 0; k < 32; k += 2) {
+                        const float x0 = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k]);
+                        const float x1 = fmaf(__uint_as_float(g[k + 1]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k + 1]);
+                        const float w0 = ex2(x0 - mref), w1 = ex2(x1 - mref);
+                        const uint32_t ph = pack2(w0, w1);
+                        float r0, r1;
+                        remainders(ph, w0, w1, r0, r1);
+                        l_run += w0 + w1;
+                        hi[k >> 1] = ph; lo[k >> 1] = pack2(r0, r1);
+                    }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 32; k += 2) {
+                        const float x0 = fmaf(__uint_as_float(g[k]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k]);
+                        const float x1 = fmaf(__uint_as_float(g[k + 1]), p.scale_log2, lc_s[s * kT + wg * 64 + c * 32 + k + 1]);
+                        const float w0 = (jw + c * 32 + k < vis) ? ex2(x0 - mref) : 0.f;
+                        const float w1 = (jw + c * 32 + k + 1 < vis) ? ex2(x1 - mref) : 0.f;
+                        const uint32_t ph = pack2(w0, w1);
+                        float r0, r1;
+                        remainders(ph, w0, w1, r0, r1);
+                        l_run += w0 + w1;
+                        hi[k >> 1] = ph; lo[k >> 1] = pack2(r0, r1);
+                    }
                 }
                 // the 32 score columns just read become 16 columns of packed leading parts and 16 of remainders
                 tmem_st16(lane_addr + kColS + s * kT + wg * 64 + c * 32, hi);
