@@ -65,6 +65,7 @@ __global__ void __launch_bounds__(256) norms_kernel(const T* __restrict__ K, sc_
 }
 
 // Step 2 on the tensor cores: block (I, chunk, head) thresholds tiles (I, J) for J in its chunk, J <= I.
+template <bool kNegTau>   // tau < 0: a zero-norm key (Sim = 0) counts as similar
 __global__ void __launch_bounds__(kThreads, 2) adj_umma_kernel(const __grid_constant__ AdjParams p) {
     extern __shared__ unsigned char smem_raw[];
     const int I = blockIdx.x, j_begin = blockIdx.y * kJChunk, bh = blockIdx.z;
@@ -142,7 +143,6 @@ __global__ void __launch_bounds__(kThreads, 2) adj_umma_kernel(const __grid_cons
         const int q = warp & 3, r = q * 32 + lane;          // warps 2..5 own lane quarters 2, 3, 0, 1
         const int i = I * kT + r;
         const float ni = i < p.n ? p.norms[(size_t)bh * p.n + i] : 0.f;
-        const bool neg = p.tau < 0.f;
         uint32_t* row = p.bits + (size_t)bh * bits_words(p.nb) + tile_row_base(I) + (size_t)r * 4 * (I + 1);
         for (int t = 0; t < nt; ++t) {
             const int s = t & 1, J = j_begin + t;
@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kThreads, 2) adj_umma_kernel(const __grid_cons
                 for (int k = 0; k < 32; ++k) {
                     const float thr = ni * nrm_s[s * kT + c * 32 + k];
                     bool hit = __uint_as_float(g[k]) > thr;
-                    if (neg) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
+                    if (kNegTau) hit = hit || (thr == 0.f);   // a zero-norm key has Sim = 0 > tau
                     w |= (hit ? 1u : 0u) << k;
                 }
                 if (J == I) {   // earlier tokens only
@@ -241,6 +241,10 @@ __global__ void __launch_bounds__(kT) adj_generic_kernel(const T* __restrict__ K
 }
 
 // Search state per call: ctl[r] = tokens still undecided when round r starts (ctl[0] = everything).
+// Words of a head's token masks (seed, member, rank base): one bit per token, the stride rounded up to whole
+// 16-byte groups so that a head's masks can be read four words at a time.
+__host__ __device__ inline int mask_words(int n) { return (((n + 31) >> 5) + 3) & ~3; }
+
 struct Masks {
     uint32_t* seed;      // [B*Hkv][nw]
     uint32_t* member;    // [B*Hkv][nw]
@@ -256,18 +260,31 @@ __global__ void init_kernel(Masks m, size_t words, long long tokens) {
 }
 
 // One warp looks at one undecided token's earlier neighbours.  Returns 1 = seed, 2 = member, 0 = still open.
+// The row's words come sixteen bytes per lane, two such reads in flight (a row of a 32K-token sequence is 4 KB: with
+// one word per lane and a vote per 128 bytes the warp spent its time waiting for loads).  `words` is rounded up to
+// the four-word groups the row is stored in; bits past the token's own position are zero there.
 __device__ __forceinline__ int decide_row(const uint32_t* __restrict__ row, int words, const uint32_t* seed,
                                           const uint32_t* member, int lane) {
+    const int groups = (words + 3) >> 2;
+    const uint4* row4 = reinterpret_cast<const uint4*>(row);
+    const uint4* seed4 = reinterpret_cast<const uint4*>(seed);
+    const uint4* member4 = reinterpret_cast<const uint4*>(member);
     bool has_seed = false, has_open = false;
-    for (int w0 = 0; w0 < words; w0 += 32) {
-        const int w = w0 + lane;
-        uint32_t x = 0u, sd = 0u, mb = 0u;
-        if (w < words) {
-            x = row[w];
-            if (x) { sd = ((volatile const uint32_t*)seed)[w]; mb = ((volatile const uint32_t*)member)[w]; }
+    for (int g0 = 0; g0 < groups; g0 += 64) {
+        const int ga = g0 + lane, gb = g0 + 32 + lane;
+        uint4 xa = make_uint4(0u, 0u, 0u, 0u), xb = xa;
+        if (ga < groups) xa = __ldg(row4 + ga);
+        if (gb < groups) xb = __ldg(row4 + gb);
+        if (xa.x | xa.y | xa.z | xa.w) {
+            const uint4 sd = __ldcg(seed4 + ga), mb = __ldcg(member4 + ga);   // through L2: other blocks add bits meanwhile
+            has_seed |= ((xa.x & sd.x) | (xa.y & sd.y) | (xa.z & sd.z) | (xa.w & sd.w)) != 0u;
+            has_open |= ((xa.x & ~(sd.x | mb.x)) | (xa.y & ~(sd.y | mb.y)) | (xa.z & ~(sd.z | mb.z)) | (xa.w & ~(sd.w | mb.w))) != 0u;
         }
-        has_seed |= (x & sd) != 0u;
-        has_open |= (x & ~(sd | mb)) != 0u;
+        if (xb.x | xb.y | xb.z | xb.w) {
+            const uint4 sd = __ldcg(seed4 + gb), mb = __ldcg(member4 + gb);
+            has_seed |= ((xb.x & sd.x) | (xb.y & sd.y) | (xb.z & sd.z) | (xb.w & sd.w)) != 0u;
+            has_open |= ((xb.x & ~(sd.x | mb.x)) | (xb.y & ~(sd.y | mb.y)) | (xb.z & ~(sd.z | mb.z)) | (xb.w & ~(sd.w | mb.w))) != 0u;
+        }
         if (__any_sync(kFull, has_seed)) return 2;   // an earlier neighbour is a seed: final
     }
     return __any_sync(kFull, has_open) ? 0 : 1;      // every earlier neighbour is a member (or there is none): a seed
@@ -276,7 +293,7 @@ __device__ __forceinline__ int decide_row(const uint32_t* __restrict__ row, int 
 __global__ void __launch_bounds__(256) round_kernel(const uint32_t* __restrict__ bits, int n, int nb, int heads, Masks m, int round) {
     if (m.ctl[round] == 0) return;   // nothing left: uniform over the grid
     const int lane = threadIdx.x & 31;
-    const int nw = (n + 31) >> 5;
+    const int nw = mask_words(n);
     const long long rows = (long long)heads * n;
     int open = 0;
     for (long long rid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); rid < rows; rid += (long long)gridDim.x * 8) {
@@ -303,7 +320,7 @@ __global__ void __launch_bounds__(1024) finish_kernel(const uint32_t* __restrict
     if (m.ctl[kRounds] == 0) return;
     __shared__ int open_s;
     const int bh = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int nw = (n + 31) >> 5;
+    const int nw = mask_words(n);
     uint32_t* seed = m.seed + (size_t)bh * nw;
     uint32_t* member = m.member + (size_t)bh * nw;
     for (int sweep = 0; sweep <= n; ++sweep) {
@@ -334,7 +351,7 @@ __global__ void __launch_bounds__(1024) rank_kernel(const uint32_t* __restrict__
                                                     int32_t* __restrict__ core_len, int cap, int32_t* status) {
     __shared__ int wsum[32];
     const int bh = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int nw = (n + 31) >> 5;
+    const int nw = mask_words(n);
     int carry = 0;
     for (int base = 0; base < nw; base += 1024) {
         const int w = base + threadIdx.x;
@@ -358,7 +375,7 @@ __global__ void __launch_bounds__(1024) rank_kernel(const uint32_t* __restrict__
 __global__ void __launch_bounds__(256) assign_kernel(const uint32_t* __restrict__ bits, int n, int nb, int heads,
                                                      const uint32_t* __restrict__ seed, int32_t* __restrict__ assign) {
     const int lane = threadIdx.x & 31;
-    const int nw = (n + 31) >> 5;
+    const int nw = mask_words(n);
     const long long rows = (long long)heads * n;
     for (long long rid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5); rid < rows; rid += (long long)gridDim.x * 8) {
         const int bh = (int)(rid / n), i = (int)(rid - (long long)bh * n);
@@ -369,16 +386,25 @@ __global__ void __launch_bounds__(256) assign_kernel(const uint32_t* __restrict_
         }
         const int I = i / kT;
         const uint32_t* row = bits + (size_t)bh * bits_words(nb) + tile_row_base(I) + (size_t)(i - I * kT) * 4 * (I + 1);
-        const int words = (i + 31) >> 5;
+        const int groups = (((i + 31) >> 5) + 3) >> 2;   // the row in its four-word groups, sixteen bytes per lane
+        const uint4* row4 = reinterpret_cast<const uint4*>(row);
+        const uint4* sd4 = reinterpret_cast<const uint4*>(sd);
         int found = -1;
-        for (int w0 = 0; w0 < words && found < 0; w0 += 32) {
-            const int w = w0 + lane;
-            const uint32_t x = w < words ? (row[w] & sd[w]) : 0u;
-            const uint32_t vote = __ballot_sync(kFull, x != 0u);
+        for (int g0 = 0; g0 < groups && found < 0; g0 += 32) {
+            const int g = g0 + lane;
+            uint4 x = make_uint4(0u, 0u, 0u, 0u);
+            if (g < groups) {
+                const uint4 rw = __ldg(row4 + g), sw = __ldg(sd4 + g);
+                x = make_uint4(rw.x & sw.x, rw.y & sw.y, rw.z & sw.z, rw.w & sw.w);
+            }
+            const uint32_t vote = __ballot_sync(kFull, (x.x | x.y | x.z | x.w) != 0u);
             if (vote) {
                 const int src = __ffs(vote) - 1;
-                const uint32_t xs = __shfl_sync(kFull, x, src);
-                found = (w0 + src) * 32 + __ffs(xs) - 1;
+                const uint32_t x0 = __shfl_sync(kFull, x.x, src), x1 = __shfl_sync(kFull, x.y, src);
+                const uint32_t x2 = __shfl_sync(kFull, x.z, src), x3 = __shfl_sync(kFull, x.w, src);
+                const int sub = x0 ? 0 : (x1 ? 1 : (x2 ? 2 : 3));
+                const uint32_t xs = x0 ? x0 : (x1 ? x1 : (x2 ? x2 : x3));
+                found = ((g0 + src) * 4 + sub) * 32 + __ffs(xs) - 1;
             }
         }
         if (lane == 0) assign[rid] = found;   // a member always has one
@@ -397,7 +423,7 @@ __global__ void __launch_bounds__(256) members_kernel(int n, int heads, const ui
                                                       const int32_t* __restrict__ rank_base, const int32_t* __restrict__ assign,
                                                       int32_t* __restrict__ csize, const int32_t* __restrict__ coff,
                                                       int32_t* __restrict__ cursor, int32_t* __restrict__ members, int phase) {
-    const int nw = (n + 31) >> 5;
+    const int nw = mask_words(n);
     const long long rows = (long long)heads * n;
     for (long long rid = (long long)blockIdx.x * blockDim.x + threadIdx.x; rid < rows; rid += (long long)gridDim.x * blockDim.x) {
         const int bh = (int)(rid / n), j = (int)(rid - (long long)bh * n);
@@ -513,7 +539,7 @@ struct Layout {   // workspace: every part 256-byte aligned
     size_t norms, bits, seed, member, rank, assign, csize, coff, members, ctl, total;
 };
 inline Layout layout_for(int B, int Hkv, int n) {
-    const size_t heads = (size_t)B * Hkv, nb = (n + kT - 1) / kT, nw = (n + 31) / 32;
+    const size_t heads = (size_t)B * Hkv, nb = (n + kT - 1) / kT, nw = mask_words(n);
     auto up = [](size_t x) { return (x + 255) / 256 * 256; };
     Layout L;
     size_t off = 0;
@@ -545,7 +571,7 @@ static cudaError_t run_global(const GlobalArgs& a, cudaStream_t st) {
     Masks m{(uint32_t*)(ws + L.seed), (uint32_t*)(ws + L.member), (int32_t*)(ws + L.ctl)};
     int32_t* rank_base = (int32_t*)(ws + L.rank);
     int32_t* assign = a.assign ? a.assign : (int32_t*)(ws + L.assign);
-    const int heads = a.B * a.Hkv, nb = (a.n + kT - 1) / kT, nw = (a.n + 31) / 32;
+    const int heads = a.B * a.Hkv, nb = (a.n + kT - 1) / kT, nw = mask_words(a.n);
     const long long rows = (long long)heads * a.n;
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
@@ -560,13 +586,15 @@ static cudaError_t run_global(const GlobalArgs& a, cudaStream_t st) {
     if (a.dt == SC_BF16 && a.d == 128 && !(a.flags & SC_FLAG_GENERIC) && heads <= 65535 && nb <= 65535) {
         static bool attr_set[64] = {false};
         if (!attr_set[dev & 63]) {
-            cudaFuncSetAttribute(adj_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+            cudaFuncSetAttribute(adj_umma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+            cudaFuncSetAttribute(adj_umma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
             attr_set[dev & 63] = true;
         }
         AdjParams p;
         p.norms = norms; p.bits = bits; p.n = a.n; p.nb = nb; p.Hkv = a.Hkv; p.tau = a.tau; p.status = a.status;
         if (make_map_bf16_rows(&p.map, a.K, a.st.b, a.st.h, a.st.n, a.B, a.Hkv, a.n, kT)) {
-            adj_umma_kernel<<<grid, kThreads, kSmemBytes, st>>>(p);
+            if (a.tau < 0.f) adj_umma_kernel<true><<<grid, kThreads, kSmemBytes, st>>>(p);
+            else adj_umma_kernel<false><<<grid, kThreads, kSmemBytes, st>>>(p);
             umma_done = true;
         }
     }
