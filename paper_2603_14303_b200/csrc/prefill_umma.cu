@@ -11,7 +11,8 @@
 //   warps 2-9  softmax, two threads per query row (= tensor-memory lane; each owns half of a tile's keys and
 //              half of the accumulator's columns, the row maximum is exchanged through shared memory):
 //              x = S * scale*log2(e) + log2(count), masks (head length, optional causal tail), running
-//              maximum raised lazily (the accumulator row is rescaled in tensor memory only then),
+//              maximum raised lazily (the accumulator row is rescaled in tensor memory only then; the tile's
+//              maximum is taken as a bound: largest raw product * scale + largest log2(count) of the tile),
 //              P = 2^(x - m) as a bf16 pair (leading part + remainder) written back over the scores it
 //              came from: the 32 fp32 columns of a chunk of scores become 16 columns of packed leading
 //              parts and 16 of remainders, so P is double-buffered like S and never touches shared
